@@ -1,0 +1,792 @@
+// gl_cartesian_dot: compute dotProd (cartProd (windows? a0) a1)   (Fig. 2a, 2b, Fig. 6)
+//
+// The pairing that cartProd describes (Section 4.2) is never stored: it is the
+// pairing of an A tile with a B tile inside a GEMM  out[m,o] = sum_k A[m,k] B[o,k].
+// Tensor-core path (sm_100a):
+//   * operands are staged in shared memory by TMA.  For a convolution the rows
+//     of A are windows of a channels-last activation tensor and the TMA unit
+//     forms them itself (im2col tensor map: window origin, filter offset, zero
+//     fill outside the image), so the im2col matrix of Section 5.3 never exists;
+//   * tcgen05.mma (bf16 x bf16 -> fp32) issued by one thread accumulates into
+//     TMEM; two accumulator buffers let the epilogue of one tile overlap the
+//     main loop of the next;
+//   * four epilogue warps read TMEM with tcgen05.ld, apply relu if asked and
+//     store fp32 rows.
+// A general SIMT kernel covers every other shape (odd K, arbitrary-rank windows).
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstring>
+#include <mutex>
+
+#include "gl_internal.h"
+
+using namespace gl;
+
+namespace {
+
+__device__ unsigned int g_status = 0;   // sticky: set when a bounded wait gives up
+
+// ------------------------------------------------------------------------
+// General SIMT kernel
+// ------------------------------------------------------------------------
+
+struct GenA {            // how to fetch A[m,k]
+  int mode;              // 0 plain [M,K]; 1 conv windows; 2 arbitrary windows
+  int64_t M, K, O;
+  // conv
+  int channels_last;
+  int64_t C, H, W, Kh, Kw, Sh, Sw, ph, pw, Ho, Wo;
+  // arbitrary windows
+  int n;
+  int64_t in_size[GL_MAX_DIMS], in_stride[GL_MAX_DIMS], out_ext[GL_MAX_DIMS];
+  int64_t w[GL_MAX_DIMS], s[GL_MAX_DIMS], pad_lo[GL_MAX_DIMS];
+  int64_t item;
+};
+
+__device__ __forceinline__ float bf16_to_f32(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }
+
+__device__ float fetch_a(const uint16_t* __restrict__ a, const GenA& g, int64_t m, int64_t k) {
+  if (g.mode == 0) return bf16_to_f32(a[m * g.K + k]);
+  if (g.mode == 1) {
+    const int64_t wo = m % g.Wo, ho = (m / g.Wo) % g.Ho, n = m / (g.Wo * g.Ho);
+    int64_t c, kh, kw;
+    if (g.channels_last) { c = k % g.C; kw = (k / g.C) % g.Kw; kh = k / (g.C * g.Kw); }
+    else { kw = k % g.Kw; kh = (k / g.Kw) % g.Kh; c = k / (g.Kw * g.Kh); }
+    const int64_t h = ho * g.Sh + kh - g.ph, w = wo * g.Sw + kw - g.pw;
+    if (h < 0 || h >= g.H || w < 0 || w >= g.W) return 0.f;
+    const int64_t off = g.channels_last ? ((n * g.H + h) * g.W + w) * g.C + c : ((n * g.C + c) * g.H + h) * g.W + w;
+    return bf16_to_f32(a[off]);
+  }
+  int64_t q[GL_MAX_DIMS], idx = k, off = 0;
+  for (int d = g.n - 1; d >= 0; --d) { q[d] = idx % g.w[d]; idx /= g.w[d]; }
+  idx = m;
+  bool inside = true;
+  for (int d = g.n - 1; d >= 0; --d) {
+    const int64_t pos = (idx % g.out_ext[d]) * g.s[d] + q[d] - g.pad_lo[d];
+    idx /= g.out_ext[d];
+    inside = inside && pos >= 0 && pos < g.in_size[d];
+    off += pos * g.in_stride[d];
+  }
+  return inside ? bf16_to_f32(a[idx * g.item + off]) : 0.f;
+}
+
+// 64x64 output tile per block, 4x4 per thread, K in steps of 16.
+__global__ void __launch_bounds__(256) dot_general(const uint16_t* __restrict__ a, const uint16_t* __restrict__ b,
+                                                   float* __restrict__ out, const GenA g, int relu) {
+  __shared__ float sa[16][64 + 1], sb[16][64 + 1];
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  const int64_t m0 = (int64_t)blockIdx.y * 64, o0 = (int64_t)blockIdx.x * 64;
+  float acc[4][4] = {};
+  for (int64_t k0 = 0; k0 < g.K; k0 += 16) {
+    for (int e = threadIdx.x; e < 16 * 64; e += 256) {
+      const int kk = e & 15, r = e >> 4;
+      const int64_t k = k0 + kk;
+      sa[kk][r] = (m0 + r < g.M && k < g.K) ? fetch_a(a, g, m0 + r, k) : 0.f;
+      sb[kk][r] = (o0 + r < g.O && k < g.K) ? bf16_to_f32(b[(o0 + r) * g.K + k]) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < 16; ++kk) {
+      float av[4], bv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { av[i] = sa[kk][ty * 4 + i]; bv[i] = sb[kk][tx * 4 + i]; }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int64_t m = m0 + ty * 4 + i, o = o0 + tx * 4 + j;
+      if (m < g.M && o < g.O) {
+        float v = acc[i][j];
+        if (relu) v = v > 0.f ? v : 0.f;
+        out[m * g.O + o] = v;
+      }
+    }
+}
+
+// ------------------------------------------------------------------------
+// Layout pre-pass for the paper's (C,H,W) item layout: channels-last copies
+// with the channel count padded to a multiple of 8 (16 bytes of bf16), which
+// is what the TMA unit can address.
+// ------------------------------------------------------------------------
+
+// X (N,C,HW) -> (N,HW,Cp), zero for c >= C.
+__global__ void __launch_bounds__(256) nchw_to_nhwc_pad(const uint16_t* __restrict__ in, uint16_t* __restrict__ out,
+                                                        int64_t C, int64_t HW, int64_t Cp) {
+  __shared__ uint16_t tile[32][34];
+  const int64_t n = blockIdx.z, c0 = (int64_t)blockIdx.y * 32, p0 = (int64_t)blockIdx.x * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int64_t c = c0 + ty + 8 * i, p = p0 + tx;
+    tile[ty + 8 * i][tx] = (c < C && p < HW) ? in[(n * C + c) * HW + p] : (uint16_t)0;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int64_t p = p0 + ty + 8 * i, c = c0 + tx;
+    if (p < HW && c < Cp) out[(n * HW + p) * Cp + c] = tile[tx][ty + 8 * i];
+  }
+}
+
+// W (O,C,T) -> (O,T,Cp) with T = Kh*Kw, zero for c >= C.
+__global__ void __launch_bounds__(256) weights_to_channels_last(const uint16_t* __restrict__ in,
+                                                                uint16_t* __restrict__ out, int64_t O, int64_t C,
+                                                                int64_t T, int64_t Cp) {
+  const int64_t total = O * T * Cp;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t c = e % Cp, t = (e / Cp) % T, o = e / (Cp * T);
+    out[e] = c < C ? in[(o * C + c) * T + t] : (uint16_t)0;
+  }
+}
+
+// ------------------------------------------------------------------------
+// tcgen05 / TMA building blocks (inline PTX)
+// ------------------------------------------------------------------------
+
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // a wait that lasts 2 s has failed
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ uint64_t global_timer() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Bounded wait.  Returns false when the block is giving up: either this wait
+// ran out of time (it then raises the block's abort flag and the device status
+// word) or another role of the block already did.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_timer();
+  uint32_t spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 0xFFu) == 0) {
+      if (*abort_flag) return false;
+      if (global_timer() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        atomicOr(&g_status, 1u);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar)
+      : "memory");
+}
+// im2col-mode load of a (pixels x channels) box: coordinates are the first
+// window origin (c, w, h, n); the filter offset (kw, kh) is added by the TMA unit.
+__device__ __forceinline__ void tma_load_im2col(uint32_t dst, const CUtensorMap* map, int c, int w, int h, int n,
+                                                uint16_t kw, uint16_t kh, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%2, %3, %4, %5}], [%6], {%7, %8};"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar), "h"(kw), "h"(kh)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, M = 128, N from the instruction descriptor, K = 16.
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_load_32cols(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major operand tile.
+//   bits  0-13 start address >> 4      bits 16-29 leading byte offset >> 4
+//   bits 32-45 stride byte offset >> 4 bits 46-47 descriptor version (1)
+//   bits 61-63 swizzle: 0 none, 2 128-byte
+// 128-byte swizzle: rows of 128 bytes, groups of 8 rows 1024 bytes apart (SBO).
+// No swizzle: 8x16-byte core matrices; LBO between cores along K, SBO along rows.
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t swz) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
+  d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;
+  d |= static_cast<uint64_t>(swz) << 61;
+  return d;
+}
+
+// Instruction descriptor, kind::f16: D fp32 (bits 4-5 = 1), A and B bf16
+// (bits 7-9, 10-12 = 1), both K-major (bits 15, 16 = 0), N >> 3 at bit 17, M >> 4 at bit 24.
+__host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
+         (static_cast<uint32_t>(m >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------
+// The GEMM kernel
+// ------------------------------------------------------------------------
+
+constexpr int kBM = 128;
+constexpr int kBK = 64;          // bf16 elements per K block = one 128-byte swizzle row
+constexpr int kTcThreads = 192;  // warp 0 TMA, warp 1 MMA + TMEM, warps 2-5 epilogue
+
+enum AMode { kDense = 0, kIm2col = 1, kIm2colGranule = 2 };
+
+struct TcParams {
+  int64_t M, O, K;        // K as laid out in B (for conv: Kh*Kw*Cp)
+  int tiles_m, tiles_n, kblocks;
+  int relu;
+  // conv only
+  int Cp, Kh, Kw, Sh, Sw, ph, pw, Ho, Wo;
+  int cchunks;            // kIm2col: 64-channel chunks per tap; kIm2colGranule: 8-channel granules per tap
+};
+
+template <int BN>
+struct TcCfg {
+  static constexpr int kStageA = kBM * kBK * 2;
+  static constexpr int kStageB = BN * kBK * 2;
+  static constexpr int kStage = kStageA + kStageB;
+  static constexpr int kStages = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
+  static constexpr int kTmemCols = 2 * BN;
+  static constexpr int kSmemBytes = kStages * kStage + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+template <int BN, int MODE>
+__global__ void __launch_bounds__(kTcThreads, 1)
+dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+       float* __restrict__ out, const TcParams p) {
+  using Cfg = TcCfg<BN>;
+  extern __shared__ unsigned char smem_raw[];
+  // operand tiles need 1024-byte alignment for the 128-byte swizzle
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;
+  unsigned char* gen_tiles = smem_raw + (tiles - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_tiles + Cfg::kStages * Cfg::kStage);
+  const uint32_t bar_full = smem_u32(bars);                          // [kStages]
+  const uint32_t bar_empty = bar_full + 8 * Cfg::kStages;            // [kStages]
+  const uint32_t bar_tfull = bar_empty + 8 * Cfg::kStages;           // [2]
+  const uint32_t bar_tempty = bar_tfull + 16;                        // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * Cfg::kStages + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < Cfg::kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(static_cast<uint32_t>(Cfg::kTmemCols))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int num_tiles = p.tiles_m * p.tiles_n;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+        const int tm = t / p.tiles_n, tn = t % p.tiles_n;
+        const int m0 = tm * kBM, n0 = tn * BN;
+        int wbase = 0, hbase = 0, img = 0;
+        if (MODE != kDense) {
+          const int wo = m0 % p.Wo, ho = (m0 / p.Wo) % p.Ho;
+          img = m0 / (p.Wo * p.Ho);
+          wbase = wo * p.Sw - p.pw;
+          hbase = ho * p.Sh - p.ph;
+        }
+        for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+          const uint32_t s = it % Cfg::kStages, ph = (it / Cfg::kStages) & 1u;
+          if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+          const uint32_t full = bar_full + 8 * s;
+          const uint32_t sa = tiles + s * Cfg::kStage, sb = sa + Cfg::kStageA;
+          mbar_expect_tx(full, Cfg::kStage);
+          if (MODE == kDense) {
+            tma_load_2d(sa, &map_a, kb * kBK, m0, full);
+            tma_load_2d(sb, &map_b, kb * kBK, n0, full);
+          } else if (MODE == kIm2col) {
+            const int tap = kb / p.cchunks, c0 = (kb % p.cchunks) * kBK;
+            tma_load_im2col(sa, &map_a, c0, wbase, hbase, img, static_cast<uint16_t>(tap % p.Kw),
+                            static_cast<uint16_t>(tap / p.Kw), full);
+            tma_load_2d(sb, &map_b, tap * p.Cp + c0, n0, full);
+          } else {
+            // eight 8-channel granules per K block, each its own (pixels x 16 bytes) box
+            const int taps = p.Kh * p.Kw;
+#pragma unroll 1
+            for (int g = 0; g < 8; ++g) {
+              const int gi = kb * 8 + g;
+              const int tap = gi / p.cchunks;
+              // beyond the last tap: a box that lies outside the channel range reads as zeros
+              const int c0 = tap < taps ? (gi % p.cchunks) * 8 : p.Cp;
+              const int tp = tap < taps ? tap : 0;
+              tma_load_im2col(sa + g * (kBM * 16), &map_a, c0, wbase, hbase, img, static_cast<uint16_t>(tp % p.Kw),
+                              static_cast<uint16_t>(tp / p.Kw), full);
+            }
+            tma_load_3d(sb, &map_b, 0, n0, kb * 8, full);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(kBM, BN);
+      uint32_t it = 0, tile_it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_it) {
+        const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
+        if (!mbar_wait(bar_tempty + 8 * acc, aph ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+          const uint32_t s = it % Cfg::kStages, ph = (it / Cfg::kStages) & 1u;
+          if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = tiles + s * Cfg::kStage, sb = sa + Cfg::kStageA;
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k) {
+            uint64_t da, db;
+            if (MODE == kIm2colGranule) {
+              da = make_desc(sa + k * 2 * (kBM * 16), kBM * 16, 128, 0);
+              db = make_desc(sb + k * 2 * (BN * 16), BN * 16, 128, 0);
+            } else {
+              da = make_desc(sa + k * 32, 16, 1024, 2);
+              db = make_desc(sb + k * 32, 16, 1024, 2);
+            }
+            tc_mma_bf16(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          tc_commit(bar_empty + 8 * s);   // frees the stage once these MMAs have read it
+        }
+        if (ok) tc_commit(bar_tfull + 8 * acc);
+      }
+    }
+  } else {
+    // ---------------- epilogue: TMEM -> registers -> global ----------------
+    const int q = warp & 3;   // TMEM lane quarter this warp may read
+    uint32_t tile_it = 0;
+    bool ok = true;
+    const bool vec_ok = (p.O & 3) == 0;
+    for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_it) {
+      const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
+      const int tm = t / p.tiles_n, tn = t % p.tiles_n;
+      if (!mbar_wait(bar_tfull + 8 * acc, aph, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+      const int64_t m = static_cast<int64_t>(tm) * kBM + q * 32 + lane;
+      float* row = out + m * p.O;
+#pragma unroll 1
+      for (int c = 0; c < BN; c += 32) {
+        const int64_t n0 = static_cast<int64_t>(tn) * BN + c;
+        if (n0 >= p.O) break;   // uniform across the warp
+        uint32_t r[32];
+        tc_load_32cols(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN + c, r);
+        if (p.relu) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(fmaxf(__uint_as_float(r[i]), 0.f));
+        }
+        if (m < p.M) {
+          if (vec_ok && n0 + 32 <= p.O) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              *reinterpret_cast<uint4*>(row + n0 + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (n0 + i < p.O) row[n0 + i] = __uint_as_float(r[i]);
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+    }
+  }
+
+  // teardown: a block that gave up lets its copies in flight land before it leaves
+  __syncwarp();
+  if (*abort_flag) {
+    const uint64_t t0 = global_timer();
+    while (global_timer() - t0 < 20000000ull) { }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"(static_cast<uint32_t>(Cfg::kTmemCols))
+                 : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------
+// Host side: tensor maps, dispatch
+// ------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const int*, const int*, cuuint32_t, cuuint32_t,
+                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct DriverApi {
+  EncodeTiledFn tiled = nullptr;
+  EncodeIm2colFn im2col = nullptr;
+  bool ok = false;
+};
+
+const DriverApi& driver_api() {
+  static DriverApi api;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess || !f) return;
+    api.tiled = reinterpret_cast<EncodeTiledFn>(f);
+    f = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &f, cudaEnableDefault, &q) != cudaSuccess || !f) return;
+    api.im2col = reinterpret_cast<EncodeIm2colFn>(f);
+    api.ok = true;
+  });
+  return api;
+}
+
+int num_sms() {
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  }
+  return sms;
+}
+
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// [rows, K] bf16 row-major, box {64, box_rows}, 128-byte swizzle, zero fill outside.
+bool encode_kmajor_sw128(CUtensorMap* m, const void* base, int64_t rows, int64_t K, int box_rows) {
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * 2};
+  const cuuint32_t box[2] = {kBK, static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t estr[2] = {1, 1};
+  return driver_api().tiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// [rows, K] bf16 viewed as {8 elements, rows, K/8 granules}: one box {8, box_rows, 8}
+// lands as [granule][row][16 bytes], the un-swizzled K-major core-matrix order.
+bool encode_kmajor_granules(CUtensorMap* m, const void* base, int64_t rows, int64_t K, int box_rows) {
+  const cuuint64_t dims[3] = {8, static_cast<cuuint64_t>(rows), static_cast<cuuint64_t>(K / 8)};
+  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(K) * 2, 16};
+  const cuuint32_t box[3] = {8, static_cast<cuuint32_t>(box_rows), 8};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return driver_api().tiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Channels-last activations (N,H,W,Cp) as an im2col tensor map: 128 window
+// origins per box, `channels` channels per origin.
+bool encode_im2col(CUtensorMap* m, const void* base, const DotProblem& d, int64_t Cp, int channels, bool swizzle) {
+  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(Cp), static_cast<cuuint64_t>(d.W), static_cast<cuuint64_t>(d.H),
+                              static_cast<cuuint64_t>(d.N)};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(Cp) * 2, static_cast<cuuint64_t>(d.W * Cp) * 2,
+                                 static_cast<cuuint64_t>(d.H * d.W * Cp) * 2};
+  const int lower[2] = {static_cast<int>(-d.pw_lo), static_cast<int>(-d.ph_lo)};
+  const int upper[2] = {static_cast<int>(d.pw_hi - (d.Kw - 1)), static_cast<int>(d.ph_hi - (d.Kh - 1))};
+  const cuuint32_t estr[4] = {1, static_cast<cuuint32_t>(d.Sw), static_cast<cuuint32_t>(d.Sh), 1};
+  return driver_api().im2col(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, lower,
+                             upper, static_cast<cuuint32_t>(channels), kBM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                             swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN, int MODE>
+int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, const TcParams& p, cudaStream_t st) {
+  using Cfg = TcCfg<BN>;
+  static bool attr_set = false;   // benign race: the attribute call is idempotent
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(dot_tc<BN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) !=
+        cudaSuccess)
+      return GL_ERR_CUDA;
+    attr_set = true;
+  }
+  const int tiles = p.tiles_m * p.tiles_n;
+  const int grid = tiles < num_sms() ? tiles : num_sms();
+  dot_tc<BN, MODE><<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(ma, mb, out, p);
+  return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+}
+
+template <int MODE>
+int launch_tc_bn(int bn, const CUtensorMap& ma, const CUtensorMap& mb, float* out, const TcParams& p,
+                 cudaStream_t st) {
+  switch (bn) {
+    case 256: return launch_tc<256, MODE>(ma, mb, out, p, st);
+    case 128: return launch_tc<128, MODE>(ma, mb, out, p, st);
+    default: return launch_tc<64, MODE>(ma, mb, out, p, st);
+  }
+}
+
+// Column-tile width: the widest tile that still leaves every SM a tile.
+int pick_bn(int64_t M, int64_t O) {
+  const int64_t tiles_m = (M + kBM - 1) / kBM;
+  const int sms = num_sms();
+  for (int bn : {256, 128}) {
+    if (O > bn / 2 && tiles_m * ((O + bn - 1) / bn) >= sms) return bn;
+  }
+  return 64;
+}
+
+struct ConvPlan {
+  bool tc = false;       // tensor-core path available
+  bool prepass = false;  // needs channels-last copies in the workspace
+  int64_t Cp = 0;
+  size_t x_bytes = 0, w_bytes = 0;
+};
+
+ConvPlan plan_conv(const DotProblem& d) {
+  ConvPlan pl;
+  pl.Cp = (d.C + 7) / 8 * 8;
+  const bool fits = d.pw_lo <= 128 && d.ph_lo <= 128 && (d.Kw - 1 - d.pw_hi) <= 128 && (d.Kh - 1 - d.ph_hi) <= 128 &&
+                    d.Kw <= 256 && d.Kh <= 256 && d.Sw <= 8 && d.Sh <= 8 && d.W < (1ll << 30) && d.H < (1ll << 30) &&
+                    d.N < (1ll << 30) && d.M < (1ll << 31) && d.O < (1ll << 31) &&
+                    d.Kh * d.Kw * pl.Cp < (1ll << 31);
+  pl.tc = fits;
+  pl.prepass = !d.channels_last || pl.Cp != d.C;
+  if (pl.prepass) {
+    pl.x_bytes = round_up(static_cast<size_t>(d.N * d.H * d.W * pl.Cp) * 2, 1024);
+    pl.w_bytes = round_up(static_cast<size_t>(d.O * d.Kh * d.Kw * pl.Cp) * 2, 1024);
+  }
+  return pl;
+}
+
+bool dense_tc_ok(const DotProblem& d) {
+  return !d.conv && !d.general && d.K % 8 == 0 && d.M < (1ll << 31) && d.O < (1ll << 31) && d.K < (1ll << 31);
+}
+
+void fill_general(const gl_ap* a0, const gl_windows* w, const DotProblem& d, GenA* g) {
+  std::memset(g, 0, sizeof(*g));
+  g->M = d.M; g->K = d.K; g->O = d.O;
+  if (!w) { g->mode = 0; return; }
+  if (d.conv) {
+    g->mode = 1;
+    g->channels_last = d.channels_last;
+    g->C = d.C; g->H = d.H; g->W = d.W; g->Kh = d.Kh; g->Kw = d.Kw; g->Sh = d.Sh; g->Sw = d.Sw;
+    g->ph = d.ph_lo; g->pw = d.pw_lo; g->Ho = d.Ho; g->Wo = d.Wo;
+    return;
+  }
+  g->mode = 2;
+  g->n = w->n;
+  const int na = a0->access_ndim;
+  int64_t s = 1;
+  for (int i = w->n - 1; i >= 0; --i) {
+    const int64_t b = a0->shape[na + i];
+    g->in_size[i] = b;
+    g->in_stride[i] = s;
+    s *= b;
+    g->w[i] = w->wshape[i];
+    g->s[i] = w->stride[i];
+    g->pad_lo[i] = w->pad_lo[i];
+    g->out_ext[i] = (b + w->pad_lo[i] + w->pad_hi[i] - (w->wshape[i] - 1) + w->stride[i] - 1) / w->stride[i];
+  }
+  g->item = s;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t gl_cartesian_dot_workspace(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, uint32_t flags) {
+  DotProblem d;
+  if (classify_dot(a0, w, a1, &d) != GL_OK) return 0;
+  if ((flags & GL_DOT_GENERAL_KERNEL) || !d.conv) return 0;
+  const ConvPlan pl = plan_conv(d);
+  return pl.tc && pl.prepass ? pl.x_bytes + pl.w_bytes : 0;
+}
+
+int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_ap* out, uint32_t flags,
+                     void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_data(a0);
+  if (rc) return rc;
+  rc = check_data(a1);
+  if (rc) return rc;
+  if (!out) return GL_ERR_NULL;
+  if (a0->dtype != GL_BF16 || a1->dtype != GL_BF16) return GL_ERR_DTYPE;
+  if (flags & ~(GL_EPILOGUE_RELU | GL_DOT_GENERAL_KERNEL)) return GL_ERR_UNSUPPORTED;
+  DotProblem d;
+  rc = classify_dot(a0, w, a1, &d);
+  if (rc) return rc;
+  gl_ap want = *out;
+  rc = gl_shape_cartesian_dot(a0, w, a1, &want);
+  if (rc) return rc;
+  rc = check_same_meta(want, out);
+  if (rc) return rc;
+  rc = check_data(out);
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int relu = (flags & GL_EPILOGUE_RELU) ? 1 : 0;
+  float* dst = static_cast<float*>(out->data);
+  const uint16_t* pa = static_cast<const uint16_t*>(a0->data);
+  const uint16_t* pb = static_cast<const uint16_t*>(a1->data);
+
+  const bool force_general = (flags & GL_DOT_GENERAL_KERNEL) != 0;
+  ConvPlan pl;
+  if (d.conv) pl = plan_conv(d);
+  const bool use_tc = !force_general && ((d.conv && pl.tc) || dense_tc_ok(d));
+  if (!use_tc) {
+    GenA g;
+    fill_general(a0, w, d, &g);
+    const int64_t gx = (d.O + 63) / 64, gy = (d.M + 63) / 64;
+    if (gy > 65535 || gx > 0x7FFFFFFF) return GL_ERR_UNSUPPORTED;
+    dot_general<<<dim3(static_cast<unsigned>(gx), static_cast<unsigned>(gy)), 256, 0, st>>>(pa, pb, dst, g, relu);
+    return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+  }
+  if (!driver_api().ok) return GL_ERR_CUDA;
+
+  TcParams p;
+  std::memset(&p, 0, sizeof(p));
+  p.M = d.M; p.O = d.O; p.relu = relu;
+  const int bn = pick_bn(d.M, d.O);
+  p.tiles_m = static_cast<int>((d.M + kBM - 1) / kBM);
+  p.tiles_n = static_cast<int>((d.O + bn - 1) / bn);
+  CUtensorMap ma, mb;
+
+  if (!d.conv) {
+    p.K = d.K;
+    p.kblocks = static_cast<int>((d.K + kBK - 1) / kBK);
+    if (!encode_kmajor_sw128(&ma, pa, d.M, d.K, kBM) || !encode_kmajor_sw128(&mb, pb, d.O, d.K, bn)) return GL_ERR_CUDA;
+    return launch_tc_bn<kDense>(bn, ma, mb, dst, p, st);
+  }
+
+  const uint16_t* x = pa;
+  const uint16_t* wt = pb;
+  if (pl.prepass) {
+    const size_t need = pl.x_bytes + pl.w_bytes;
+    if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u)) return GL_ERR_WORKSPACE;
+    uint16_t* xs = static_cast<uint16_t*>(workspace);
+    uint16_t* ws = reinterpret_cast<uint16_t*>(static_cast<unsigned char*>(workspace) + pl.x_bytes);
+    const int64_t HW = d.H * d.W, T = d.Kh * d.Kw;
+    if (d.channels_last) {
+      // (N,H,W,C) with C not a multiple of 8: re-pitch the channel dim (a (N*HW, C) -> (N*HW, Cp) copy)
+      weights_to_channels_last<<<static_cast<unsigned>(std::min<int64_t>((d.N * HW * pl.Cp + 255) / 256, 1 << 20)), 256, 0,
+                                 st>>>(pa, xs, d.N * HW, d.C, 1, pl.Cp);
+      weights_to_channels_last<<<static_cast<unsigned>(std::min<int64_t>((d.O * T * pl.Cp + 255) / 256, 1 << 20)), 256, 0,
+                                 st>>>(pb, ws, d.O * T, d.C, 1, pl.Cp);
+    } else {
+      if (d.N > 65535 || (d.C + 31) / 32 > 65535) return GL_ERR_UNSUPPORTED;
+      const dim3 grid(static_cast<unsigned>((HW + 31) / 32), static_cast<unsigned>((pl.Cp + 31) / 32),
+                      static_cast<unsigned>(d.N));
+      nchw_to_nhwc_pad<<<grid, 256, 0, st>>>(pa, xs, d.C, HW, pl.Cp);
+      weights_to_channels_last<<<static_cast<unsigned>(std::min<int64_t>((d.O * T * pl.Cp + 255) / 256, 1 << 20)), 256, 0,
+                                 st>>>(pb, ws, d.O, d.C, T, pl.Cp);
+    }
+    if (cudaGetLastError() != cudaSuccess) return GL_ERR_CUDA;
+    x = xs;
+    wt = ws;
+  }
+  const int64_t Cp = pl.Cp, taps = d.Kh * d.Kw;
+  p.K = taps * Cp;
+  p.Cp = static_cast<int>(Cp);
+  p.Kh = static_cast<int>(d.Kh); p.Kw = static_cast<int>(d.Kw);
+  p.Sh = static_cast<int>(d.Sh); p.Sw = static_cast<int>(d.Sw);
+  p.ph = static_cast<int>(d.ph_lo); p.pw = static_cast<int>(d.pw_lo);
+  p.Ho = static_cast<int>(d.Ho); p.Wo = static_cast<int>(d.Wo);
+  if (Cp >= kBK) {
+    p.cchunks = static_cast<int>((Cp + kBK - 1) / kBK);
+    p.kblocks = static_cast<int>(taps) * p.cchunks;
+    if (!encode_im2col(&ma, x, d, Cp, kBK, true) || !encode_kmajor_sw128(&mb, wt, d.O, p.K, bn)) return GL_ERR_CUDA;
+    return launch_tc_bn<kIm2col>(bn, ma, mb, dst, p, st);
+  }
+  p.cchunks = static_cast<int>(Cp / 8);
+  p.kblocks = static_cast<int>((taps * p.cchunks + 7) / 8);
+  if (!encode_im2col(&ma, x, d, Cp, 8, false) || !encode_kmajor_granules(&mb, wt, d.O, p.K, bn)) return GL_ERR_CUDA;
+  return launch_tc_bn<kIm2colGranule>(bn, ma, mb, dst, p, st);
+}
+
+int gl_poll_device_status(void* stream) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  unsigned int v = 0;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return GL_ERR_CUDA;
+  if (cudaMemcpyFromSymbol(&v, g_status, sizeof(v)) != cudaSuccess) return GL_ERR_CUDA;
+  if (v) {
+    const unsigned int zero = 0;
+    if (cudaMemcpyToSymbol(g_status, &zero, sizeof(zero)) != cudaSuccess) return GL_ERR_CUDA;
+    return GL_ERR_TIMEOUT;
+  }
+  return GL_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,613 @@
+// Memory-bound access-pattern kernels: materialised `windows` (im2col),
+// `transpose`, `pad` (transformer table, Section 4.2; pad is the constant
+// border added for ML workloads), and the operators `reduceMax` and `relu`
+// under `compute` (Section 4.3).  These move or compare values, so every
+// result is bit-exact.  Each kernel is bounded by HBM bandwidth: coalesced
+// 128-bit global accesses, shared-memory staging where the access pattern
+// would otherwise scatter.
+#include <cuda_runtime.h>
+
+#include <cstring>
+
+#include "gl_internal.h"
+
+using namespace gl;
+
+namespace {
+
+constexpr int kThreads = 256;
+
+inline int launch_status() { return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA; }
+
+inline unsigned grid_for(int64_t work_items, int per_block) {
+  int64_t g = (work_items + per_block - 1) / per_block;
+  return static_cast<unsigned>(g < 1 ? 1 : g);
+}
+
+template <typename T> struct Fill;
+template <> struct Fill<uint32_t> {
+  static __host__ __device__ uint32_t value(int kind) { return kind == GL_PAD_NEG_INF ? 0xFF800000u : 0u; }
+};
+template <> struct Fill<uint16_t> {
+  static __host__ __device__ uint16_t value(int kind) { return kind == GL_PAD_NEG_INF ? 0xFF80u : 0u; }
+};
+
+// ------------------------------------------------------------------------
+// transpose
+// ------------------------------------------------------------------------
+
+struct BatchDims {
+  int n;
+  int64_t size[GL_MAX_DIMS];
+  int64_t in_stride[GL_MAX_DIMS];
+  int64_t out_stride[GL_MAX_DIMS];
+};
+
+struct TileParams {
+  int64_t sizeA, sizeB;        // A: contiguous in the input, B: contiguous in the output
+  int64_t in_strideB, out_strideA;
+  int64_t tilesA, tilesB;
+  BatchDims batch;
+};
+
+__device__ __forceinline__ void batch_offsets(const BatchDims& b, int64_t idx, int64_t& in_off, int64_t& out_off) {
+  in_off = 0;
+  out_off = 0;
+#pragma unroll 1
+  for (int d = b.n - 1; d >= 0; --d) {
+    const int64_t i = idx % b.size[d];
+    idx /= b.size[d];
+    in_off += i * b.in_stride[d];
+    out_off += i * b.out_stride[d];
+  }
+}
+
+// 2D tile transpose with 128-bit accesses on both sides.  Each thread loads a
+// VEC x VEC block (VEC rows of one 16-byte vector), transposes it in registers
+// and parks it in shared memory with an XOR swizzle on the vector index, so
+// that both the writes and the later row reads are free of bank conflicts.
+template <typename T, int VEC>
+__global__ void __launch_bounds__(kThreads) transpose_tiled_vec(const T* __restrict__ in, T* __restrict__ out,
+                                                                const TileParams p) {
+  constexpr int TILE = 16 * VEC;
+  __shared__ uint4 tile[TILE][16];
+  int64_t bid = blockIdx.x;
+  const int64_t tileA = bid % p.tilesA; bid /= p.tilesA;
+  const int64_t tileB = bid % p.tilesB; bid /= p.tilesB;
+  int64_t in_off, out_off;
+  batch_offsets(p.batch, bid, in_off, out_off);
+  const int ta = threadIdx.x & 15, tb = threadIdx.x >> 4;
+  const int64_t a0 = tileA * TILE, b0 = tileB * TILE;
+
+  union Row { uint4 v; T e[VEC]; };
+  Row blk[VEC];
+  {
+    const int64_t a = a0 + ta * VEC;
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) {
+      const int64_t b = b0 + tb * VEC + i;
+      if (a < p.sizeA && b < p.sizeB)
+        blk[i].v = *reinterpret_cast<const uint4*>(in + in_off + b * p.in_strideB + a);
+      else
+        blk[i].v = make_uint4(0, 0, 0, 0);
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < VEC; ++j) {
+    Row r;
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) r.e[i] = blk[i].e[j];
+    tile[ta * VEC + j][tb ^ ta] = r.v;
+  }
+  __syncthreads();
+#pragma unroll
+  for (int pass = 0; pass < VEC; ++pass) {
+    const int r = pass * 16 + tb;
+    const int64_t a = a0 + r, b = b0 + ta * VEC;
+    if (a < p.sizeA && b < p.sizeB)
+      *reinterpret_cast<uint4*>(out + out_off + a * p.out_strideA + b) = tile[r][ta ^ ((r / VEC) & 15)];
+  }
+}
+
+// Scalar 32x32 tile transpose for extents that are not multiples of a vector.
+template <typename T>
+__global__ void __launch_bounds__(kThreads) transpose_tiled_scalar(const T* __restrict__ in, T* __restrict__ out,
+                                                                   const TileParams p) {
+  __shared__ T tile[32][33];
+  int64_t bid = blockIdx.x;
+  const int64_t tileA = bid % p.tilesA; bid /= p.tilesA;
+  const int64_t tileB = bid % p.tilesB; bid /= p.tilesB;
+  int64_t in_off, out_off;
+  batch_offsets(p.batch, bid, in_off, out_off);
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int64_t a0 = tileA * 32, b0 = tileB * 32;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int64_t b = b0 + ty + 8 * i, a = a0 + tx;
+    if (a < p.sizeA && b < p.sizeB) tile[ty + 8 * i][tx] = in[in_off + b * p.in_strideB + a];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int64_t a = a0 + ty + 8 * i, b = b0 + tx;
+    if (a < p.sizeA && b < p.sizeB) out[out_off + a * p.out_strideA + b] = tile[tx][ty + 8 * i];
+  }
+}
+
+struct GatherParams {   // generic strided gather, innermost output dim contiguous in the input too
+  int n;                // dims, innermost last
+  int64_t size[GL_MAX_DIMS];
+  int64_t in_stride[GL_MAX_DIMS];
+  int64_t total;        // number of VEC chunks
+};
+
+template <typename V, int ELEMS_PER_V>
+__global__ void __launch_bounds__(kThreads) gather_rows(const V* __restrict__ in, V* __restrict__ out,
+                                                        const GatherParams p) {
+  // sizes and strides of the innermost dim are already counted in V units
+  for (int64_t c = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; c < p.total; c += (int64_t)gridDim.x * blockDim.x) {
+    int64_t idx = c, off = 0;
+#pragma unroll 1
+    for (int d = p.n - 1; d >= 0; --d) {
+      off += (idx % p.size[d]) * p.in_stride[d];
+      idx /= p.size[d];
+    }
+    out[c] = in[off];
+  }
+}
+
+template <typename T>
+int run_transpose(const gl_ap* in, const int32_t* perm, gl_ap* out, cudaStream_t st) {
+  constexpr int VEC = 16 / sizeof(T);
+  // out dims with their input strides; drop size-1 dims, merge runs that stay adjacent
+  int64_t istr_all[GL_MAX_DIMS];
+  {
+    int64_t s = 1;
+    for (int d = in->ndim - 1; d >= 0; --d) { istr_all[d] = s; s *= in->shape[d]; }
+  }
+  int r = 0;
+  int64_t size[GL_MAX_DIMS], istr[GL_MAX_DIMS];
+  for (int j = 0; j < in->ndim; ++j) {
+    const int64_t sz = in->shape[perm[j]], st_in = istr_all[perm[j]];
+    if (sz == 1) continue;
+    if (r > 0 && istr[r - 1] == st_in * sz) { size[r - 1] *= sz; istr[r - 1] = st_in; }
+    else { size[r] = sz; istr[r] = st_in; ++r; }
+  }
+  const int64_t total = numel(*in);
+  const T* src = static_cast<const T*>(in->data);
+  T* dst = static_cast<T*>(out->data);
+  if (r <= 1) {  // identity layout
+    return cudaMemcpyAsync(dst, src, total * sizeof(T), cudaMemcpyDeviceToDevice, st) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+  }
+  int64_t ostr[GL_MAX_DIMS];
+  {
+    int64_t s = 1;
+    for (int j = r - 1; j >= 0; --j) { ostr[j] = s; s *= size[j]; }
+  }
+  if (istr[r - 1] == 1) {  // innermost dim untouched: gather whole rows
+    GatherParams g;
+    std::memset(&g, 0, sizeof(g));
+    g.n = r;
+    const bool vec = size[r - 1] % VEC == 0;
+    for (int j = 0; j < r; ++j) { g.size[j] = size[j]; g.in_stride[j] = vec ? istr[j] / VEC : istr[j]; }
+    // (all outer input strides are multiples of the innermost extent, hence of VEC)
+    if (vec) {
+      g.size[r - 1] = size[r - 1] / VEC;
+      g.in_stride[r - 1] = 1;
+      g.total = total / VEC;
+      gather_rows<uint4, VEC><<<grid_for(g.total, kThreads), kThreads, 0, st>>>(
+          reinterpret_cast<const uint4*>(src), reinterpret_cast<uint4*>(dst), g);
+    } else {
+      g.total = total;
+      gather_rows<T, 1><<<grid_for(g.total, kThreads), kThreads, 0, st>>>(src, dst, g);
+    }
+    return launch_status();
+  }
+  // general case: tile over (A = the dim that is contiguous in the input, B = last output dim)
+  int ja = -1;
+  for (int j = 0; j < r; ++j) if (istr[j] == 1) ja = j;
+  if (ja < 0) return GL_ERR_UNSUPPORTED;  // cannot happen for a dense input
+  TileParams p;
+  std::memset(&p, 0, sizeof(p));
+  p.sizeA = size[ja];
+  p.sizeB = size[r - 1];
+  p.in_strideB = istr[r - 1];
+  p.out_strideA = ostr[ja];
+  int64_t nbatch = 1;
+  for (int j = 0; j < r - 1; ++j) {
+    if (j == ja) continue;
+    const int k = p.batch.n++;
+    p.batch.size[k] = size[j];
+    p.batch.in_stride[k] = istr[j];
+    p.batch.out_stride[k] = ostr[j];
+    nbatch *= size[j];
+  }
+  const bool vec = p.sizeA % VEC == 0 && p.sizeB % VEC == 0;
+  const int tile = vec ? 16 * VEC : 32;
+  p.tilesA = (p.sizeA + tile - 1) / tile;
+  p.tilesB = (p.sizeB + tile - 1) / tile;
+  const int64_t blocks = p.tilesA * p.tilesB * nbatch;
+  if (blocks > 0x7FFFFFFF) return GL_ERR_UNSUPPORTED;
+  if (vec) transpose_tiled_vec<T, VEC><<<static_cast<unsigned>(blocks), kThreads, 0, st>>>(src, dst, p);
+  else transpose_tiled_scalar<T><<<static_cast<unsigned>(blocks), kThreads, 0, st>>>(src, dst, p);
+  return launch_status();
+}
+
+// ------------------------------------------------------------------------
+// pad
+// ------------------------------------------------------------------------
+
+template <typename V>
+__global__ void __launch_bounds__(kThreads) pad_kernel(const V* __restrict__ in, V* __restrict__ out, int64_t outer,
+                                                       int64_t d_in, int64_t lo, int64_t d_out, int64_t inner,
+                                                       V fill) {
+  const int64_t total = outer * d_out * inner;
+  for (int64_t c = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; c < total; c += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t i = c % inner;
+    const int64_t d = (c / inner) % d_out;
+    const int64_t u = c / (inner * d_out);
+    const int64_t s = d - lo;
+    out[c] = (s >= 0 && s < d_in) ? in[(u * d_in + s) * inner + i] : fill;
+  }
+}
+
+// ------------------------------------------------------------------------
+// windows (materialised) and windows + reduceMax
+// ------------------------------------------------------------------------
+
+struct WinParams {
+  int n;                          // compute dims
+  int64_t in_size[GL_MAX_DIMS];   // b_i
+  int64_t in_stride[GL_MAX_DIMS];
+  int64_t out_ext[GL_MAX_DIMS];   // b'_i
+  int64_t w[GL_MAX_DIMS], s[GL_MAX_DIMS], pad_lo[GL_MAX_DIMS];
+  int64_t item;                   // elements of one input item
+  int64_t wcells;                 // prod w_i
+  int64_t total;                  // output elements
+};
+
+// General rank: one thread per output cell, out[a, p.., q..] = in[a, p_i s_i + q_i - pad_lo_i].
+template <typename T>
+__global__ void __launch_bounds__(kThreads) windows_generic(const T* __restrict__ in, T* __restrict__ out,
+                                                            const WinParams p, T fill) {
+  for (int64_t c = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; c < p.total; c += (int64_t)gridDim.x * blockDim.x) {
+    int64_t idx = c;
+    int64_t q[GL_MAX_DIMS];
+#pragma unroll 1
+    for (int d = p.n - 1; d >= 0; --d) { q[d] = idx % p.w[d]; idx /= p.w[d]; }
+    int64_t off = 0;
+    bool inside = true;
+#pragma unroll 1
+    for (int d = p.n - 1; d >= 0; --d) {
+      const int64_t pos = (idx % p.out_ext[d]) * p.s[d] + q[d] - p.pad_lo[d];
+      idx /= p.out_ext[d];
+      inside = inside && pos >= 0 && pos < p.in_size[d];
+      off += pos * p.in_stride[d];
+    }
+    out[c] = inside ? in[idx * p.item + off] : fill;
+  }
+}
+
+// General rank reduceMax over windows formed on the fly: one thread per window.
+__global__ void __launch_bounds__(kThreads) window_max_generic(const float* __restrict__ in, float* __restrict__ out,
+                                                               const WinParams p, int64_t nwin, float fill) {
+  for (int64_t c = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; c < nwin; c += (int64_t)gridDim.x * blockDim.x) {
+    int64_t idx = c, base[GL_MAX_DIMS];
+#pragma unroll 1
+    for (int d = p.n - 1; d >= 0; --d) { base[d] = (idx % p.out_ext[d]) * p.s[d] - p.pad_lo[d]; idx /= p.out_ext[d]; }
+    const float* item = in + idx * p.item;
+    float best = -INFINITY;
+#pragma unroll 1
+    for (int64_t cell = 0; cell < p.wcells; ++cell) {
+      int64_t cc = cell, off = 0;
+      bool inside = true;
+#pragma unroll 1
+      for (int d = p.n - 1; d >= 0; --d) {
+        const int64_t pos = base[d] + cc % p.w[d];
+        cc /= p.w[d];
+        inside = inside && pos >= 0 && pos < p.in_size[d];
+        off += pos * p.in_stride[d];
+      }
+      best = fmaxf(best, inside ? item[off] : fill);
+    }
+    out[c] = best;
+  }
+}
+
+// Convolution-style windows over ((N),(C,H,W)) items with window (C,Kh,Kw) and
+// strides (1,Sh,Sw): the im2col matrix of Section 5.3, rows (n,h',w'), columns
+// (c,kh,kw).  One block owns one (n,h'): it stages the Kh input rows of every
+// channel in shared memory (zero or -inf border included), then streams the
+// Wo x K output slab, which is contiguous in memory, with 128-bit stores.
+struct Im2colParams {
+  int64_t N, C, H, W, Kh, Kw, Sh, Sw, ph_lo, pw_lo, Ho, Wo, K;
+  int Wp;       // staged row length = W + pw_lo + pw_hi
+};
+
+template <typename T, int VEC>
+__global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in, T* __restrict__ out,
+                                                        const Im2colParams p, T fill) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  int* lut = reinterpret_cast<int*>(smem_raw);                     // K entries: staged offset of column k at w'=0
+  T* stage = reinterpret_cast<T*>(smem_raw + ((p.K * 4 + 15) / 16) * 16);   // [C][Kh][Wp]
+  const int64_t n = blockIdx.x / p.Ho, ho = blockIdx.x % p.Ho;
+  const int rows = static_cast<int>(p.C * p.Kh);
+  for (int k = threadIdx.x; k < p.K; k += blockDim.x) {
+    const int kw = k % static_cast<int>(p.Kw), ckh = k / static_cast<int>(p.Kw);
+    lut[k] = ckh * p.Wp + kw;
+  }
+  const int64_t h0 = ho * p.Sh - p.ph_lo;
+  for (int e = threadIdx.x; e < rows * p.Wp; e += blockDim.x) {
+    const int x = e % p.Wp, r = e / p.Wp;
+    const int kh = r % static_cast<int>(p.Kh), c = r / static_cast<int>(p.Kh);
+    const int64_t h = h0 + kh, w = x - p.pw_lo;
+    stage[e] = (h >= 0 && h < p.H && w >= 0 && w < p.W) ? in[((n * p.C + c) * p.H + h) * p.W + w] : fill;
+  }
+  __syncthreads();
+  T* dst = out + (n * p.Ho + ho) * p.Wo * p.K;
+  const int total = static_cast<int>(p.Wo * p.K);
+  union Chunk { uint4 v; T e[VEC]; };
+  for (int e = threadIdx.x * VEC; e < total; e += blockDim.x * VEC) {
+    const int wo = e / static_cast<int>(p.K), k = e - wo * static_cast<int>(p.K);
+    const int shift = wo * static_cast<int>(p.Sw);
+    if (VEC == 1) {
+      dst[e] = stage[lut[k] + shift];
+    } else {
+      Chunk ch;
+#pragma unroll
+      for (int i = 0; i < VEC; ++i) ch.e[i] = stage[lut[k + i] + shift];
+      *reinterpret_cast<uint4*>(dst + e) = ch.v;
+    }
+  }
+}
+
+// 2D windows + reduceMax over ((..),(H,W)) items (Fig. 2c): one thread per output.
+__global__ void __launch_bounds__(kThreads) window_max_2d(const float* __restrict__ in, float* __restrict__ out,
+                                                           int64_t planes, int H, int W, int Kh, int Kw, int Sh, int Sw,
+                                                           int ph, int pw, int Ho, int Wo, float fill) {
+  const int64_t total = planes * Ho * Wo;
+  for (int64_t c = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; c < total; c += (int64_t)gridDim.x * blockDim.x) {
+    const int y = static_cast<int>(c % Wo);
+    const int x = static_cast<int>((c / Wo) % Ho);
+    const float* plane = in + (c / ((int64_t)Wo * Ho)) * H * W;
+    float best = -INFINITY;
+    for (int dx = 0; dx < Kh; ++dx) {
+      const int h = x * Sh + dx - ph;
+      for (int dy = 0; dy < Kw; ++dy) {
+        const int w = y * Sw + dy - pw;
+        const bool inside = h >= 0 && h < H && w >= 0 && w < W;
+        best = fmaxf(best, inside ? plane[(int64_t)h * W + w] : fill);
+      }
+    }
+    out[c] = best;
+  }
+}
+
+// reduceMax of whole items (no windows): one warp per item.
+__global__ void __launch_bounds__(kThreads) item_max(const float* __restrict__ in, float* __restrict__ out,
+                                                      int64_t items, int64_t item) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+  for (int64_t a = blockIdx.x * (int64_t)(blockDim.x >> 5) + (threadIdx.x >> 5); a < items; a += warps) {
+    float best = -INFINITY;
+    for (int64_t i = lane; i < item; i += 32) best = fmaxf(best, in[a * item + i]);
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) best = fmaxf(best, __shfl_xor_sync(0xFFFFFFFFu, best, s));
+    if (lane == 0) out[a] = best;
+  }
+}
+
+__global__ void __launch_bounds__(kThreads) relu_vec(const float4* __restrict__ in, float4* __restrict__ out, int64_t n4) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+    float4 v = in[i];
+    v.x = v.x > 0.f ? v.x : 0.f;
+    v.y = v.y > 0.f ? v.y : 0.f;
+    v.z = v.z > 0.f ? v.z : 0.f;
+    v.w = v.w > 0.f ? v.w : 0.f;
+    out[i] = v;
+  }
+}
+
+__global__ void relu_tail(const float* __restrict__ in, float* __restrict__ out, int64_t from, int64_t n) {
+  const int64_t i = from + threadIdx.x;
+  if (i < n) out[i] = in[i] > 0.f ? in[i] : 0.f;
+}
+
+void fill_win_params(const gl_ap* in, const gl_windows* w, const gl_ap& A, WinParams* p) {
+  std::memset(p, 0, sizeof(*p));
+  const int na = in->access_ndim;
+  p->n = w->n;
+  int64_t s = 1;
+  p->wcells = 1;
+  for (int i = w->n - 1; i >= 0; --i) {
+    p->in_size[i] = in->shape[na + i];
+    p->in_stride[i] = s;
+    s *= in->shape[na + i];
+    p->out_ext[i] = A.shape[na + i];
+    p->w[i] = w->wshape[i];
+    p->s[i] = w->stride[i];
+    p->pad_lo[i] = w->pad_lo[i];
+    p->wcells *= w->wshape[i];
+  }
+  p->item = s;
+  p->total = numel(A);
+}
+
+int device_smem_optin() {
+  int dev = 0, v = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+  if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return 0;
+  return v;
+}
+
+template <typename T>
+int run_windows(const gl_ap* in, const gl_windows* w, const gl_ap& A, gl_ap* out, cudaStream_t st) {
+  constexpr int VEC = 16 / sizeof(T);
+  const T fill = Fill<T>::value(w->pad_kind);
+  const T* src = static_cast<const T*>(in->data);
+  T* dst = static_cast<T*>(out->data);
+  const int na = in->access_ndim;
+  const int64_t* b = in->shape + na;
+  // convolution-style fast path: window spans the whole first compute dim
+  if (w->n == 3 && w->wshape[0] == b[0] && w->pad_lo[0] == 0 && w->pad_hi[0] == 0) {
+    Im2colParams p;
+    p.N = prod(in->shape, 0, na);
+    p.C = b[0]; p.H = b[1]; p.W = b[2];
+    p.Kh = w->wshape[1]; p.Kw = w->wshape[2];
+    p.Sh = w->stride[1]; p.Sw = w->stride[2];
+    p.ph_lo = w->pad_lo[1]; p.pw_lo = w->pad_lo[2];
+    p.Ho = A.shape[na + 1]; p.Wo = A.shape[na + 2];
+    p.K = p.C * p.Kh * p.Kw;
+    const int64_t wp = p.W + w->pad_lo[2] + w->pad_hi[2];
+    const int64_t smem = ((p.K * 4 + 15) / 16) * 16 + p.C * p.Kh * wp * (int64_t)sizeof(T);
+    const int64_t blocks = p.N * p.Ho;
+    if (smem <= 160 * 1024 && smem <= device_smem_optin() && blocks <= 0x7FFFFFFF && p.Wo * p.K < (1ll << 30)) {
+      p.Wp = static_cast<int>(wp);
+      const bool vec = p.K % VEC == 0;
+      auto kern = vec ? im2col_rows<T, VEC> : im2col_rows<T, 1>;
+      if (smem > 48 * 1024 &&
+          cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
+        return GL_ERR_CUDA;
+      kern<<<static_cast<unsigned>(blocks), kThreads, static_cast<size_t>(smem), st>>>(src, dst, p, fill);
+      return launch_status();
+    }
+  }
+  WinParams p;
+  fill_win_params(in, w, A, &p);
+  windows_generic<T><<<grid_for(p.total, kThreads), kThreads, 0, st>>>(src, dst, p, fill);
+  return launch_status();
+}
+
+}  // namespace
+
+extern "C" {
+
+int gl_access_transpose(const gl_ap* in, const int32_t* perm, gl_ap* out, void* stream) {
+  int rc = check_data(in);
+  if (rc) return rc;
+  if (!out || !perm) return GL_ERR_NULL;
+  gl_ap want = *in;
+  rc = gl_shape_transpose(in, perm, &want);
+  if (rc) return rc;
+  rc = check_same_meta(want, out);
+  if (rc) return rc;
+  rc = check_data(out);
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return in->dtype == GL_F32 ? run_transpose<uint32_t>(in, perm, out, st) : run_transpose<uint16_t>(in, perm, out, st);
+}
+
+int gl_access_pad(const gl_ap* in, int32_t dim, int64_t lo, int64_t hi, int32_t pad_kind, gl_ap* out, void* stream) {
+  int rc = check_data(in);
+  if (rc) return rc;
+  if (!out) return GL_ERR_NULL;
+  if (pad_kind != GL_PAD_ZERO && pad_kind != GL_PAD_NEG_INF) return GL_ERR_SHAPE;
+  gl_ap want = *in;
+  rc = gl_shape_pad(in, dim, lo, hi, &want);
+  if (rc) return rc;
+  rc = check_same_meta(want, out);
+  if (rc) return rc;
+  rc = check_data(out);
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t outer = prod(in->shape, 0, dim), inner = prod(in->shape, dim + 1, in->ndim);
+  const int64_t d_in = in->shape[dim], d_out = d_in + lo + hi;
+  const size_t es = dtype_size(in->dtype);
+  const int vec = static_cast<int>(16 / es);
+  if (inner % vec == 0) {
+    uint4 fill;
+    const uint32_t f32 = Fill<uint32_t>::value(pad_kind);
+    const uint32_t f16 = Fill<uint16_t>::value(pad_kind) * 0x10001u;
+    fill.x = fill.y = fill.z = fill.w = (in->dtype == GL_F32 ? f32 : f16);
+    const int64_t total = outer * d_out * (inner / vec);
+    pad_kernel<uint4><<<grid_for(total, kThreads), kThreads, 0, st>>>(
+        static_cast<const uint4*>(in->data), static_cast<uint4*>(out->data), outer, d_in, lo, d_out, inner / vec, fill);
+  } else if (in->dtype == GL_F32) {
+    pad_kernel<uint32_t><<<grid_for(outer * d_out * inner, kThreads), kThreads, 0, st>>>(
+        static_cast<const uint32_t*>(in->data), static_cast<uint32_t*>(out->data), outer, d_in, lo, d_out, inner,
+        Fill<uint32_t>::value(pad_kind));
+  } else {
+    pad_kernel<uint16_t><<<grid_for(outer * d_out * inner, kThreads), kThreads, 0, st>>>(
+        static_cast<const uint16_t*>(in->data), static_cast<uint16_t*>(out->data), outer, d_in, lo, d_out, inner,
+        Fill<uint16_t>::value(pad_kind));
+  }
+  return launch_status();
+}
+
+int gl_access_windows(const gl_ap* in, const gl_windows* w, gl_ap* out, void* stream) {
+  int rc = check_data(in);
+  if (rc) return rc;
+  if (!out || !w) return GL_ERR_NULL;
+  gl_ap want = *in;
+  rc = gl_shape_windows(in, w, &want);
+  if (rc) return rc;
+  rc = check_same_meta(want, out);
+  if (rc) return rc;
+  rc = check_data(out);
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return in->dtype == GL_F32 ? run_windows<uint32_t>(in, w, want, out, st) : run_windows<uint16_t>(in, w, want, out, st);
+}
+
+int gl_compute_reduce_max(const gl_ap* in, const gl_windows* w, gl_ap* out, void* stream) {
+  int rc = check_data(in);
+  if (rc) return rc;
+  if (!out) return GL_ERR_NULL;
+  if (in->dtype != GL_F32) return GL_ERR_DTYPE;
+  gl_ap want = *in;
+  rc = gl_shape_reduce_max(in, w, &want);
+  if (rc) return rc;
+  rc = check_same_meta(want, out);
+  if (rc) return rc;
+  rc = check_data(out);
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const float* src = static_cast<const float*>(in->data);
+  float* dst = static_cast<float*>(out->data);
+  if (!w) {
+    const int64_t items = prod(in->shape, 0, in->access_ndim), item = prod(in->shape, in->access_ndim, in->ndim);
+    item_max<<<grid_for(items, kThreads / 32), kThreads, 0, st>>>(src, dst, items, item);
+    return launch_status();
+  }
+  gl_ap A = *in;
+  gl_shape_windows(in, w, &A);
+  const float fill = w->pad_kind == GL_PAD_NEG_INF ? -INFINITY : 0.0f;
+  const int64_t nwin = numel(want);
+  const int na = in->access_ndim;
+  if (w->n == 2 && in->shape[na] < (1 << 30) && in->shape[na + 1] < (1 << 30)) {
+    window_max_2d<<<grid_for(nwin, kThreads), kThreads, 0, st>>>(
+        src, dst, prod(in->shape, 0, na), (int)in->shape[na], (int)in->shape[na + 1], (int)w->wshape[0],
+        (int)w->wshape[1], (int)w->stride[0], (int)w->stride[1], (int)w->pad_lo[0], (int)w->pad_lo[1],
+        (int)A.shape[na], (int)A.shape[na + 1], fill);
+    return launch_status();
+  }
+  WinParams p;
+  fill_win_params(in, w, A, &p);
+  window_max_generic<<<grid_for(nwin, kThreads), kThreads, 0, st>>>(src, dst, p, nwin, fill);
+  return launch_status();
+}
+
+int gl_compute_relu(const gl_ap* in, gl_ap* out, void* stream) {
+  int rc = check_data(in);
+  if (rc) return rc;
+  if (!out) return GL_ERR_NULL;
+  if (in->dtype != GL_F32) return GL_ERR_DTYPE;
+  rc = check_same_meta(*in, out);
+  if (rc) return rc;
+  rc = check_data(out);
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t n = numel(*in), n4 = n / 4;
+  const float* src = static_cast<const float*>(in->data);
+  float* dst = static_cast<float*>(out->data);
+  if (n4) {
+    int64_t blocks = (n4 + kThreads - 1) / kThreads;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    relu_vec<<<static_cast<unsigned>(blocks), kThreads, 0, st>>>(reinterpret_cast<const float4*>(src),
+                                                               reinterpret_cast<float4*>(dst), n4);
+  }
+  if (n % 4) relu_tail<<<1, 4, 0, st>>>(src, dst, n4 * 4, n);
+  return launch_status();
+}
+
+}  // extern "C"

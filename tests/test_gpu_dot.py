@@ -1,0 +1,227 @@
+"""GPU parity of gl_cartesian_dot (compute dotProd over cartProd, Fig. 2a/2b and
+the im2col-rewritten form of Section 5.3) against the CPU checker.
+
+Integer-valued inputs in [-3,3]: every partial sum is an integer below 2^24, so
+fp32 accumulation in any order is exact and the comparison is bit for bit.
+N(0,1) inputs: max |g-r| / max(|r|, rms(r)) <= 2e-3 against the float64 result.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import brute
+from oracle import interp as gi
+from paper_2105_09377_b200 import synth
+from tests.gpu_util import REL_TOL, rel_err, to_bf16_device
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gl():
+    from paper_2105_09377_b200 import binding
+    return binding
+
+
+def _ok(gl):
+    assert gl.gl_poll_device_status() == 0
+
+
+def _conv_gpu(gl, x, wt, stride, pad, channels_last=False, flags=0):
+    """conv2d through the C ABI; returns the ((N,1,H',W',O),()) result as (N,H',W',O) numpy."""
+    n, c, h, w = x.shape
+    o, _, kh, kw = wt.shape
+    if channels_last:
+        xa = gl.AccessPattern(to_bf16_device(np.ascontiguousarray(x.transpose(0, 2, 3, 1))), 1)
+        wa = gl.AccessPattern(to_bf16_device(np.ascontiguousarray(wt.transpose(0, 2, 3, 1))), 1)
+        spec = gl.windows_spec((kh, kw, c), (stride[0], stride[1], 1), (pad[0], pad[1], 0), (pad[0], pad[1], 0))
+    else:
+        xa = gl.AccessPattern(to_bf16_device(x), 1)
+        wa = gl.AccessPattern(to_bf16_device(wt), 1)
+        spec = gl.windows_spec((c, kh, kw), (1, stride[0], stride[1]), (0, pad[0], pad[1]), (0, pad[0], pad[1]))
+    out = gl.gl_cartesian_dot(xa, spec, wa, flags=flags)
+    _ok(gl)
+    t = out.tensor
+    if channels_last:
+        assert t.shape[3] == 1
+        return t.squeeze(3).cpu().numpy()
+    assert t.shape[1] == 1
+    return t.squeeze(1).cpu().numpy()
+
+
+def _conv_ref(x, wt, stride, pad):
+    """float64 (N,H',W',O) from the brute-force conv2d equation."""
+    return brute.conv2d(x, wt, stride, ((pad[0], pad[0]), (pad[1], pad[1]))).transpose(0, 2, 3, 1)
+
+
+# ---- the tiny configuration: direct form, im2col-rewritten form, interpreter ----
+
+@pytest.mark.parametrize("flags", [0, 0x100])
+def test_tiny_conv_direct_and_rewritten(gl, flags):
+    cfg = synth.CONV_TINY
+    x, wt = cfg.inputs(synth.config_seed(0))
+    ref = gi.conv2d_program(x, wt, upto="dotProd")              # ((1,1,6,6,4),())
+    xa, wa = gl.AccessPattern(to_bf16_device(x), 1), gl.AccessPattern(to_bf16_device(wt), 1)
+    spec = gl.windows_spec((3, 3, 3), (1, 1, 1))
+    direct = gl.gl_cartesian_dot(xa, spec, wa, flags=flags)
+    _ok(gl)
+    assert direct.shape == ref.shape
+    assert np.array_equal(direct.tensor.cpu().numpy().astype(np.float64), ref.data)
+    # Section 5.3: windows materialised and flattened, weights flattened, plain matmul, reshape
+    cols = gl.gl_access_flatten(gl.gl_access_windows(xa, spec))
+    wflat = gl.gl_access_flatten(wa)
+    assert cols.shape == ((36,), (27,)) and wflat.shape == ((4,), (27,))
+    mm = gl.gl_cartesian_dot(cols, None, wflat, flags=flags)
+    _ok(gl)
+    assert mm.shape == ((36, 4), ())
+    assert torch.equal(mm.tensor.view(direct.tensor.shape), direct.tensor)
+    # squeeze + transpose (0 3 1 2) of Fig. 2a gives the NCHW result
+    nhwo = gl.AccessPattern(direct.tensor.view(1, 6, 6, 4), 4)
+    nchw = gl.gl_access_transpose(nhwo, (0, 3, 1, 2))
+    full = gi.conv2d_program(x, wt)
+    assert np.array_equal(nchw.tensor.cpu().numpy().astype(np.float64), full.data)
+
+
+CONV_SMALL = [
+    # n, c, h, w, o, kh, kw, sh, sw, ph, pw
+    (2, 8, 9, 10, 16, 3, 3, 1, 1, 1, 1),      # C = 8: granule path, one M tile
+    (3, 16, 12, 11, 24, 3, 2, 2, 1, 1, 0),    # lopsided window, strides and pads
+    (2, 64, 14, 14, 64, 3, 3, 1, 1, 1, 1),    # C = 64: swizzled path, 4 ragged M tiles
+    (1, 128, 9, 9, 72, 3, 3, 1, 1, 1, 1),     # two channel chunks per tap, O not a tile multiple
+    (2, 96, 8, 8, 40, 1, 1, 1, 1, 0, 0),      # C = 96: last chunk half empty
+    (2, 3, 20, 20, 8, 7, 7, 2, 2, 3, 3),      # stem-like: C = 3 padded to 8, 49 taps
+    (2, 32, 10, 10, 130, 1, 1, 2, 2, 0, 0),   # 1x1 stride 2, O spans two column tiles
+    (5, 24, 7, 7, 10, 5, 5, 1, 1, 2, 2),      # several images per tile, window 5x5
+    (1, 5, 6, 6, 3, 2, 2, 1, 1, 0, 0),        # odd everything
+]
+
+
+@pytest.mark.parametrize("layout", ["nchw", "nhwc"])
+@pytest.mark.parametrize("case", CONV_SMALL)
+def test_conv_integer_bit_exact(gl, case, layout):
+    n, c, h, w, o, kh, kw, sh, sw, ph, pw = case
+    x = synth.uniform_int(21, 1, (n, c, h, w), -3, 3)
+    wt = synth.uniform_int(21, 2, (o, c, kh, kw), -3, 3)
+    ref = _conv_ref(x, wt, (sh, sw), (ph, pw))
+    got = _conv_gpu(gl, x, wt, (sh, sw), (ph, pw), channels_last=(layout == "nhwc"))
+    assert got.shape == ref.shape
+    assert np.array_equal(got.astype(np.float64), ref)
+    again = _conv_gpu(gl, x, wt, (sh, sw), (ph, pw), channels_last=(layout == "nhwc"))
+    assert np.array_equal(got, again)                         # same bits on a second run
+
+
+@pytest.mark.parametrize("case", CONV_SMALL[:4])
+def test_conv_general_kernel_bit_exact(gl, case):
+    n, c, h, w, o, kh, kw, sh, sw, ph, pw = case
+    x = synth.uniform_int(22, 1, (n, c, h, w), -3, 3)
+    wt = synth.uniform_int(22, 2, (o, c, kh, kw), -3, 3)
+    ref = _conv_ref(x, wt, (sh, sw), (ph, pw))
+    for cl in (False, True):
+        got = _conv_gpu(gl, x, wt, (sh, sw), (ph, pw), channels_last=cl, flags=gl.GL_DOT_GENERAL_KERNEL)
+        assert np.array_equal(got.astype(np.float64), ref)
+
+
+@pytest.mark.parametrize("case", CONV_SMALL)
+def test_conv_gaussian_within_tolerance(gl, case):
+    n, c, h, w, o, kh, kw, sh, sw, ph, pw = case
+    cc = synth.ConvCase("t", n, c, h, w, o, kh, kw, sh, ph)
+    x = synth.bf16_round(synth.normal(23, 1, (n, c, h, w)))
+    wt = synth.bf16_round(synth.normal(23, 2, (o, c, kh, kw), np.sqrt(2.0 / cc.kd)))
+    ref = _conv_ref(x, wt, (sh, sw), (ph, pw))
+    got = _conv_gpu(gl, x, wt, (sh, sw), (ph, pw), channels_last=True)
+    assert rel_err(got, ref) <= REL_TOL
+
+
+def test_windows_over_other_dims_uses_general_kernel(gl):
+    # windows that also slide over the channel dim: not a conv2d, still a valid program
+    x = synth.uniform_int(24, 1, (2, 5, 6, 7), -3, 3)
+    wt = synth.uniform_int(24, 2, (4, 2, 3, 2), -3, 3)
+    a = gi.windows(gi.access(x, 1), (2, 3, 2), (2, 1, 3))
+    ref = gi.compute("dotProd", gi.cart_prod(a, gi.access(wt, 1)))
+    out = gl.gl_cartesian_dot(gl.AccessPattern(to_bf16_device(x), 1), gl.windows_spec((2, 3, 2), (2, 1, 3)),
+                              gl.AccessPattern(to_bf16_device(wt), 1))
+    _ok(gl)
+    assert out.shape == ref.shape
+    assert np.array_equal(out.tensor.cpu().numpy().astype(np.float64), ref.data)
+
+
+# ---- dense: compute dotProd (cartProd A B), both operands as row vectors ----
+
+DENSE_SMALL = [(36, 4, 27), (1, 1, 8), (128, 256, 64), (130, 70, 72), (300, 520, 200), (257, 129, 1000), (64, 48, 7)]
+
+
+@pytest.mark.parametrize("m,o,k", DENSE_SMALL)
+def test_dense_integer_bit_exact(gl, m, o, k):
+    a = synth.uniform_int(31, 1, (m, k), -3, 3)
+    b = synth.uniform_int(31, 2, (o, k), -3, 3)
+    ref = brute.rowdot(a, b)
+    for flags in (0, gl.GL_DOT_GENERAL_KERNEL):
+        out = gl.gl_cartesian_dot(gl.AccessPattern(to_bf16_device(a), 1), None, gl.AccessPattern(to_bf16_device(b), 1),
+                                  flags=flags)
+        _ok(gl)
+        assert out.shape == ((m, o), ())
+        assert np.array_equal(out.tensor.cpu().numpy().astype(np.float64), ref)
+
+
+def test_dense_interpreter_program_with_relu(gl):
+    a = synth.uniform_int(32, 1, (20, 16), -3, 3)
+    b = synth.uniform_int(32, 2, (12, 16), -3, 3)
+    ref = gi.dense_rows_program(a, b, relu=True)
+    aa, bb = gl.AccessPattern(to_bf16_device(a), 1), gl.AccessPattern(to_bf16_device(b), 1)
+    fused = gl.gl_cartesian_dot(aa, None, bb, flags=gl.GL_EPILOGUE_RELU)
+    two_step = gl.gl_compute_relu(gl.gl_cartesian_dot(aa, None, bb))
+    _ok(gl)
+    assert np.array_equal(fused.tensor.cpu().numpy().astype(np.float64), ref.data)
+    assert torch.equal(fused.tensor, two_step.tensor)
+
+
+def test_dense_gaussian_1024_full_check(gl):
+    case = synth.DenseCase("d1024", 1024, 1024, 1024)
+    a, b = case.inputs(41)
+    ref = brute.rowdot(a, b)
+    out = gl.gl_cartesian_dot(gl.AccessPattern(to_bf16_device(a), 1), None, gl.AccessPattern(to_bf16_device(b), 1))
+    _ok(gl)
+    assert rel_err(out.tensor.cpu().numpy(), ref) <= REL_TOL
+
+
+def test_dense_4096_sampled_rows_and_relu(gl):
+    case = synth.DENSE_4096
+    a, b = case.inputs(synth.config_seed(1))
+    aa, bb = gl.AccessPattern(to_bf16_device(a), 1), gl.AccessPattern(to_bf16_device(b), 1)
+    out = gl.gl_cartesian_dot(aa, None, bb, flags=gl.GL_EPILOGUE_RELU)
+    _ok(gl)
+    got = out.tensor.cpu().numpy()
+    rng = np.random.default_rng(5)
+    rows = np.unique(np.concatenate([rng.integers(0, 4096, 48), [0, 127, 128, 255, 256, 4095]]))
+    ref = np.maximum(brute.rowdot(a, b, rows), 0.0)
+    assert rel_err(got[rows], ref) <= REL_TOL
+    cols = np.unique(np.concatenate([rng.integers(0, 4096, 48), [0, 255, 256, 4095]]))
+    refc = np.maximum(brute.rowdot(b, a, cols), 0.0).T          # columns of out = rows of B against all of A
+    assert rel_err(got[:, cols], refc) <= REL_TOL
+    assert (got >= 0).all()
+
+
+# ---- the convolution sweeps at full size, on sampled outputs ----
+
+FULL_CONVS = list(synth.CONV_SWEEP_3X3) + list(synth.CONV_STRIDED_1X1)
+
+
+@pytest.mark.parametrize("cfg", FULL_CONVS, ids=[c.name for c in FULL_CONVS])
+@pytest.mark.parametrize("layout", ["nhwc", "nchw"])
+def test_full_size_conv_sampled(gl, cfg, layout):
+    x, wt = cfg.inputs(synth.config_seed(2))
+    got = _conv_gpu(gl, x, wt, (cfg.stride,) * 2, (cfg.pad,) * 2, channels_last=(layout == "nhwc"))
+    assert got.shape == (cfg.n, cfg.ho, cfg.wo, cfg.o)
+    rng = np.random.default_rng(9)
+    cnt = 4096
+    ns, os_ = rng.integers(0, cfg.n, cnt), rng.integers(0, cfg.o, cnt)
+    xs, ys = rng.integers(0, cfg.ho, cnt), rng.integers(0, cfg.wo, cnt)
+    # corners, image borders and tile seams are always in the sample
+    xs[:64] = np.where(rng.integers(0, 2, 64) == 0, 0, cfg.ho - 1)
+    ys[64:128] = np.where(rng.integers(0, 2, 64) == 0, 0, cfg.wo - 1)
+    flat = ((ns * cfg.o + os_) * cfg.ho + xs) * cfg.wo + ys
+    pads = ((cfg.pad, cfg.pad), (cfg.pad, cfg.pad))
+    ref = brute.conv2d_sampled(x, wt, flat, (cfg.stride,) * 2, pads)
+    assert rel_err(got[ns, xs, ys, os_], ref) <= REL_TOL
+    # a property that holds at any size: the last image (ragged final tile) is finite and not all zero
+    assert np.isfinite(got[-1]).all() and np.abs(got[-1]).max() > 0

@@ -1,0 +1,187 @@
+"""GPU parity of the memory-bound access operators against the CPU checker.
+They move or compare values, so every comparison is bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import brute
+from oracle import interp as gi
+from paper_2105_09377_b200 import synth
+from tests.gpu_util import to_bf16_device, to_f32_device
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gl():
+    from paper_2105_09377_b200 import binding
+    return binding
+
+
+def _same_bits(got: torch.Tensor, ref: np.ndarray):
+    g = got.float().cpu().numpy()
+    assert g.shape == ref.shape
+    np.testing.assert_array_equal(g.view(np.uint32), np.ascontiguousarray(ref, dtype=np.float32).view(np.uint32))
+
+
+TRANSPOSE_CASES = [
+    ((2, 8, 4, 12), 1, (0, 2, 3, 1)),       # NCHW -> NHWC, vector path
+    ((3, 5, 7, 9), 1, (0, 2, 3, 1)),        # odd extents: scalar tiles
+    ((2, 6, 5, 16), 2, (0, 3, 1, 2)),       # (N,H',W',O) -> (N,O,H',W') of Fig. 2a
+    ((70, 130), 1, (1, 0)),                 # plain matrix, several ragged tiles
+    ((4, 3, 200), 1, (1, 0, 2)),            # innermost kept: row gather
+    ((4, 3, 37), 1, (1, 0, 2)),
+    ((3, 4, 5, 6, 7), 2, (4, 1, 3, 0, 2)),  # rank 5, general permutation
+    ((5, 1, 6), 1, (2, 1, 0)),              # size-1 dim in the middle
+    ((24,), 1, (0,)),                       # identity
+    ((2, 3, 4), 1, (0, 1, 2)),
+    ((1, 64, 3, 3, 8, 2, 2, 5), 3, (7, 6, 5, 4, 3, 2, 1, 0)),  # rank 8 reversal
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape,na,perm", TRANSPOSE_CASES)
+def test_transpose(gl, shape, na, perm, dtype):
+    x = synth.uniform(7, 1, shape, -1.0, 1.0)
+    if dtype == "bf16":
+        x = synth.bf16_round(x)
+    ref = gi.transpose(gi.access(x, na), perm)
+    dev = to_f32_device(x) if dtype == "f32" else to_bf16_device(x)
+    out = gl.gl_access_transpose(gl.AccessPattern(dev, na), perm)
+    assert out.shape == ref.shape
+    _same_bits(out.tensor, ref.data.astype(np.float32))
+
+
+def test_transpose_full_size_nchw_to_nhwc(gl):
+    cfg = synth.MEM_TRANSPOSE
+    x = cfg.inputs(synth.config_seed(4))
+    out = gl.gl_access_transpose(gl.AccessPattern(to_f32_device(x), 1), cfg.perm).tensor
+    n, c, h, w = cfg.shape
+    ref = brute.transpose_021(x.reshape(n, c, h * w)).reshape(n, h, w, c)
+    assert torch.equal(out.cpu(), torch.from_numpy(ref))
+
+
+WINDOW_CASES = [
+    # shape, access_ndim, window, stride, pad_lo, pad_hi, kind
+    ((1, 3, 8, 8), 1, (3, 3, 3), (1, 1, 1), (0, 0, 0), (0, 0, 0), 0),       # the tiny conv configuration
+    ((2, 4, 9, 10), 1, (4, 3, 3), (1, 1, 1), (0, 1, 1), (0, 1, 1), 0),      # 3x3 pad 1, K multiple of 4
+    ((2, 3, 11, 9), 1, (3, 7, 7), (1, 2, 2), (0, 3, 3), (0, 3, 3), 0),      # 7x7 s2 p3, K = 147 (scalar stores)
+    ((2, 8, 6, 6), 1, (8, 1, 1), (1, 2, 2), (0, 0, 0), (0, 0, 0), 0),       # 1x1 stride 2
+    ((2, 3, 9, 8), 2, (3, 2), (2, 1), (0, 0), (0, 0), 0),                   # pooling-style 2D windows
+    ((2, 3, 9, 8), 2, (3, 3), (2, 2), (1, 1), (1, 1), 1),                   # -inf border
+    ((3, 10), 1, (4,), (3,), (1,), (2,), 0),                                # 1D windows, uneven pads
+    ((2, 5, 6, 7), 1, (2, 3, 2), (2, 1, 3), (1, 0, 1), (0, 2, 0), 0),       # windows over channels too
+    ((2, 6, 4), 1, (6, 4), (1, 1), (0, 0), (0, 0), 0),                      # window == whole item
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape,na,wshape,stride,lo,hi,kind", WINDOW_CASES)
+def test_windows(gl, shape, na, wshape, stride, lo, hi, kind, dtype):
+    x = synth.uniform(8, 1, shape, -1.0, 1.0)
+    if dtype == "bf16":
+        x = synth.bf16_round(x)
+    a = gi.access(x, na)
+    for i, (l, h) in enumerate(zip(lo, hi)):
+        if l or h:
+            a = gi.pad(a, na + i, l, h, "neg_inf" if kind else "zero")
+    ref = gi.windows(a, wshape, stride)
+    dev = to_f32_device(x) if dtype == "f32" else to_bf16_device(x)
+    out = gl.gl_access_windows(gl.AccessPattern(dev, na), gl.windows_spec(wshape, stride, lo, hi, kind))
+    assert out.shape == ref.shape
+    _same_bits(out.tensor, ref.data.astype(np.float32))
+    # flatten is metadata: same storage, the im2col matrix view
+    flat = gl.gl_access_flatten(out)
+    assert flat.tensor.data_ptr() == out.tensor.data_ptr()
+    assert flat.shape == gi.flatten(ref).shape
+
+
+def test_im2col_full_size(gl):
+    cfg = synth.MEM_IM2COL
+    x = cfg.inputs(synth.config_seed(4))
+    n, c, h, w = cfg.shape
+    spec = gl.windows_spec((c, 3, 3), (1, 1, 1), (0, 1, 1), (0, 1, 1))
+    out = gl.gl_access_windows(gl.AccessPattern(to_f32_device(x), 1), spec)
+    assert out.shape == ((n, 1, h, w), (c, 3, 3))
+    ref = brute.im2col(x, 3, 3, (1, 1), ((1, 1), (1, 1)))
+    got = gl.gl_access_flatten(out).tensor
+    assert got.shape == ref.shape
+    assert torch.equal(got.cpu(), torch.from_numpy(ref))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape,na,dim,lo,hi,kind", [
+    ((2, 3, 5, 8), 1, 2, 1, 1, 0), ((2, 3, 5, 8), 1, 3, 2, 0, 0), ((2, 3, 5, 7), 2, 3, 1, 3, 1),
+    ((4, 6), 1, 0, 0, 2, 1), ((9,), 0, 0, 3, 3, 0), ((2, 3, 4), 1, 1, 0, 0, 0),
+])
+def test_pad(gl, shape, na, dim, lo, hi, kind, dtype):
+    x = synth.uniform(9, 1, shape, -1.0, 1.0)
+    if dtype == "bf16":
+        x = synth.bf16_round(x)
+    ref = gi.pad(gi.access(x, na), dim, lo, hi, "neg_inf" if kind else "zero")
+    dev = to_f32_device(x) if dtype == "f32" else to_bf16_device(x)
+    out = gl.gl_access_pad(gl.AccessPattern(dev, na), dim, lo, hi, kind)
+    assert out.shape == ref.shape
+    _same_bits(out.tensor, ref.data.astype(np.float32))
+
+
+POOL_CASES = [
+    ((2, 3, 9, 8), 2, (3, 3), (2, 2), (1, 1), (1, 1)),
+    ((2, 3, 9, 8), 2, (2, 3), (1, 2), (0, 0), (0, 0)),
+    ((1, 2, 12, 12), 2, (3, 3), (2, 2), (1, 1), (1, 1)),
+    ((3, 17), 1, (5,), (2,), (2,), (1,)),                   # 1D windows: general kernel
+    ((2, 4, 5, 6), 1, (2, 3, 2), (2, 1, 2), (0, 1, 0), (0, 1, 0)),   # 3D windows: general kernel
+]
+
+
+@pytest.mark.parametrize("shape,na,wshape,stride,lo,hi", POOL_CASES)
+def test_windows_reduce_max(gl, shape, na, wshape, stride, lo, hi):
+    x = synth.uniform(10, 1, shape, -1.0, 1.0) - 2.0          # all negative: a zero border would win
+    a = gi.access(x, na)
+    for i, (l, h) in enumerate(zip(lo, hi)):
+        if l or h:
+            a = gi.pad(a, na + i, l, h, "neg_inf")
+    ref = gi.compute("reduceMax", gi.windows(a, wshape, stride))
+    out = gl.gl_compute_reduce_max(gl.AccessPattern(to_f32_device(x), na),
+                                   gl.windows_spec(wshape, stride, lo, hi, gl.GL_PAD_NEG_INF))
+    assert out.shape == ref.shape
+    _same_bits(out.tensor, ref.data.astype(np.float32))
+
+
+def test_reduce_max_whole_items(gl):
+    x = synth.uniform(11, 1, (7, 5, 33), -1.0, 1.0)
+    ref = gi.compute("reduceMax", gi.access(x, 1))
+    out = gl.gl_compute_reduce_max(gl.AccessPattern(to_f32_device(x), 1), None)
+    _same_bits(out.tensor, ref.data.astype(np.float32))
+
+
+def test_maxpool_full_size(gl):
+    cfg = synth.MEM_MAXPOOL
+    x = cfg.inputs(synth.config_seed(4))
+    spec = gl.windows_spec(cfg.window, (cfg.stride,) * 2, (cfg.pad,) * 2, (cfg.pad,) * 2, gl.GL_PAD_NEG_INF)
+    out = gl.gl_compute_reduce_max(gl.AccessPattern(to_f32_device(x), 2), spec).tensor
+    ref = brute.maxpool(x, cfg.window, (cfg.stride,) * 2, ((cfg.pad,) * 2, (cfg.pad,) * 2))
+    assert torch.equal(out.cpu(), torch.from_numpy(ref))
+
+
+@pytest.mark.parametrize("n", [1, 3, 4, 1000, 4099])
+def test_relu(gl, n):
+    x = synth.uniform(12, 1, (n,), -1.0, 1.0)
+    x[::7] = -0.0
+    ref = gi.compute("relu", gi.access(x, 1)).data.astype(np.float32)
+    dev = to_f32_device(x)
+    out = gl.gl_compute_relu(gl.AccessPattern(dev, 1))
+    _same_bits(out.tensor, ref)
+    gl.gl_compute_relu(gl.AccessPattern(dev, 1), gl.AccessPattern(dev, 1))    # in place
+    _same_bits(dev, ref)
+
+
+def test_output_metadata_is_checked(gl):
+    x = to_f32_device(synth.uniform(13, 1, (4, 6), -1.0, 1.0))
+    bad = gl.AccessPattern(torch.empty((6, 5), device="cuda"), 1)
+    with pytest.raises(gl.GlError) as e:
+        gl.gl_access_transpose(gl.AccessPattern(x, 1), (1, 0), out=bad)
+    assert e.value.code == 4
+    with pytest.raises(gl.GlError) as e:
+        gl.gl_compute_relu(gl.AccessPattern(x.to(torch.bfloat16), 1))
+    assert e.value.code == 2
