@@ -1,0 +1,401 @@
+#!/usr/bin/env python
+"""Throughput of the access-pattern hot path on B200.
+
+A step is one pass of the dense-layer program
+    compute relu (compute dotProd (cartProd A B)),  A, B = ((4096),(4096)) bf16
+through gl_cartesian_dot (relu fused in the epilogue), fp32 result.  One JSON
+line is printed by rank 0.  With --gpus N every rank runs an independent
+replica on its own GPU (the program has no exchange step); the value is the
+work of all ranks over the slowest rank's time.
+
+`--impl reference` times the CPU checker (oracle/) on a bounded sample of the
+same workload instead.  `--detail` (default at one GPU) adds per-workload
+timings of the convolution sweeps and the memory-bound access operators.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "access-pattern conv2d/matmul TFLOP/s (% bf16 peak); windows/pool GB/s (% HBM)"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+L2_BYTES = 126 * 1024 * 1024
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            return json.load(fh), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# --------------------------------------------------------------------------
+# multi-process plumbing (replicas; no data-path collective)
+# --------------------------------------------------------------------------
+
+def dist_env():
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+
+
+def init_dist(backend: str):
+    import torch.distributed as dist
+    rank, _, world = dist_env()
+    if world > 1 and not dist.is_initialized():
+        dist.init_process_group(backend=backend, rank=rank, world_size=world)
+    return rank, world
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+
+
+def max_over_ranks(value: float, device="cpu") -> float:
+    """The slowest rank's time: all-reduce MAX of one scalar (timing only, not on the data path)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(units_per_rank: float, world: int, max_seconds: float) -> float:
+    """Whole-job throughput: units processed by all ranks over the slowest rank's time."""
+    return units_per_rank * world / max_seconds
+
+
+# --------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.QUERY, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+            time.sleep(0.3)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, reasons, smax = [], set(), None
+        try:
+            with open(self.path) as fh:
+                for line in fh:
+                    f = [x.strip() for x in line.split(",")]
+                    if len(f) < 9:
+                        continue
+                    try:
+                        sm.append(float(f[1]))
+                        smax = float(f[2])
+                    except ValueError:
+                        continue
+                    for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                        if val.lower().startswith("active"):
+                            reasons.add(name)
+            os.unlink(self.path)
+        except OSError:
+            pass
+        if sm:
+            busy = [v for v in sm[2:]] or sm      # the first samples precede the timed region
+            out.update(sm_mhz=statistics.median(busy), sm_max_mhz=smax, reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# --------------------------------------------------------------------------
+# reference arm: the CPU checker, as it stands
+# --------------------------------------------------------------------------
+
+def cpu_baseline_dense(target_seconds: float = 12.0):
+    """Times oracle.brute.rowdot on a sample of rows of the 4096^3 workload."""
+    import numpy as np
+    from oracle import brute
+    from paper_2105_09377_b200 import synth
+    case = synth.DENSE_4096
+    a, b = case.inputs(synth.config_seed(1))
+    t0 = time.perf_counter()
+    brute.rowdot(a, b, np.arange(8))
+    probe = max(time.perf_counter() - t0, 1e-4)
+    rows = int(min(case.m, max(8, 8 * target_seconds / probe)))
+    rows -= rows % 8
+    idx = np.arange(rows, dtype=np.int64)
+    t0 = time.perf_counter()
+    brute.rowdot(a, b, idx)
+    dt = time.perf_counter() - t0
+    flops = 2.0 * rows * case.o * case.k
+    return {"value": flops / dt / 1e12, "unit": "TFLOP/s", "cores": brute.num_threads(), "kind": "oracle",
+            "sample": "rows 0..%d of A (of %d) against all %d rows of B, float64 accumulate, %.1f s" % (rows - 1, case.m, case.o, dt),
+            "seconds": dt, "rows": rows}
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return 0
+    import numpy as np
+    from oracle import brute
+    from paper_2105_09377_b200 import synth
+    case = synth.DENSE_4096
+    a, b = case.inputs(synth.config_seed(1))
+    rows_per_step = 32
+    idx = np.arange(rows_per_step, dtype=np.int64)
+    for _ in range(args.warmup):
+        brute.rowdot(a, b, idx)
+    steps = min(args.steps, 400)          # bounded: the whole run stays within a few minutes
+    t0 = time.perf_counter()
+    for s in range(steps):
+        np.maximum(brute.rowdot(a, b, (idx + s * rows_per_step) % case.m), 0.0)
+    dt = time.perf_counter() - t0
+    flops = 2.0 * rows_per_step * case.o * case.k * steps
+    value = flops / dt / 1e12
+    sample = "each step: %d rows of A (of %d) against all rows of B, relu, float64 accumulate" % (rows_per_step, case.m)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": steps, "warmup": args.warmup, "ms_per_step": dt / steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": case.name, "M": case.m, "O": case.o, "K": case.k, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "kind": "oracle", "cores": brute.num_threads(), "sample": sample},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# --------------------------------------------------------------------------
+# GPU arm
+# --------------------------------------------------------------------------
+
+def time_graph(calls, iters: int, device):
+    """Median and best per-call time (seconds) of `calls` (rotating buffer sets), replayed
+    from one CUDA graph so that host launch cost does not pace microsecond kernels."""
+    import torch
+    s = torch.cuda.Stream(device=device)
+    s.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(s):
+        for c in calls:
+            c()
+    torch.cuda.current_stream().wait_stream(s)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for c in calls:
+            c()
+    for _ in range(3):
+        g.replay()
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(iters):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        g.replay()
+        e1.record()
+        e1.synchronize()
+        times.append(e0.elapsed_time(e1) * 1e-3 / len(calls))
+    return statistics.median(times), min(times)
+
+
+def detail_workloads(device, peaks):
+    """Per-workload timings of the other configurations (not the headline value)."""
+    import torch
+    from paper_2105_09377_b200 import run_workload as rw
+    from paper_2105_09377_b200 import synth
+    out = []
+
+    def entry(cfg, layout):
+        nsets = max(2, int((2 * L2_BYTES + cfg.algorithmic_bytes - 1) // cfg.algorithmic_bytes))
+        nsets = min(nsets, 32)
+        calls, flops, nbytes = [], 0.0, 0
+        for _ in range(nsets):
+            c, flops, nbytes = rw.build_call(cfg, layout, device)
+            calls.append(c)
+        med, best = time_graph(calls, 20, device)
+        e = {"workload": cfg.name, "us": med * 1e6, "us_best": best * 1e6, "gbs": nbytes / med / 1e9,
+             "frac_hbm_peak": nbytes / med / 1e9 / peaks["hbm_gbs"], "buffer_sets": nsets}
+        if flops:
+            tf = flops / med / 1e12
+            t_roof = max(flops / (peaks["bf16_tflops"] * 1e12), nbytes / (peaks["hbm_gbs"] * 1e9))
+            e.update(layout=layout, tflops=tf, frac_tensor_peak=tf / peaks["bf16_tflops"], frac_binding_roof=t_roof / med)
+        out.append(e)
+        del calls
+        torch.cuda.empty_cache()
+
+    for cfg in list(synth.CONV_SWEEP_3X3) + list(synth.CONV_STRIDED_1X1):
+        for layout in ("nhwc", "nchw"):
+            entry(cfg, layout)
+    for cfg in (synth.MEM_IM2COL, synth.MEM_TRANSPOSE, synth.MEM_MAXPOOL):
+        entry(cfg, "")
+    return out
+
+
+def run_gpu(args):
+    import numpy as np
+    import torch
+    rank, local_rank, world = dist_env()
+    if world > 1:
+        init_dist("nccl")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    from paper_2105_09377_b200 import binding as gl
+    from paper_2105_09377_b200 import synth
+    peaks, peaks_kind = load_peaks()
+
+    def bf16_host(x):
+        return torch.from_numpy(synth.bf16_bits(x).view(np.int16)).view(torch.bfloat16).reshape(x.shape)
+
+    case = synth.DENSE_4096
+    a_host, b_host = case.inputs(synth.config_seed(1))
+    bytes_per_set = case.algorithmic_bytes
+    nsets = max(2, int((2 * L2_BYTES + bytes_per_set - 1) // bytes_per_set))
+    a0, b0 = bf16_host(a_host).to(device), bf16_host(b_host).to(device)
+    calls = []
+    for i in range(nsets):
+        aa = gl.AccessPattern(a0 if i == 0 else a0.clone(), 1)
+        bb = gl.AccessPattern(b0 if i == 0 else b0.clone(), 1)
+        oo = gl.AccessPattern(torch.empty((case.m, case.o), dtype=torch.float32, device=device), 2)
+        calls.append(gl.prepare_cartesian_dot(aa, None, bb, oo, gl.GL_EPILOGUE_RELU))
+
+    warmup = max(args.warmup, 3)
+    for i in range(warmup):
+        calls[i % nsets]()
+    torch.cuda.synchronize()
+    if gl.gl_poll_device_status() != 0:
+        raise RuntimeError("device status: a bounded wait gave up during warm-up")
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        calls[i % nsets]()
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    seconds = e0.elapsed_time(e1) * 1e-3
+    clocks = sampler.stop() if rank == 0 else None
+    seconds_max = max_over_ranks(seconds, device)
+    if gl.gl_poll_device_status() != 0:
+        raise RuntimeError("device status: a bounded wait gave up during the timed region")
+
+    # end to end through the public call: pinned host operands in, result back to pinned host memory
+    e2e_steps = max(3, min(args.steps, 20))
+    a_pin, b_pin = bf16_host(a_host).pin_memory(), bf16_host(b_host).pin_memory()
+    o_pin = torch.empty((case.m, case.o), dtype=torch.float32).pin_memory()
+    a_dev, b_dev = torch.empty_like(a0), torch.empty_like(b0)
+    o_dev = gl.AccessPattern(torch.empty((case.m, case.o), dtype=torch.float32, device=device), 2)
+    e2e_call = gl.prepare_cartesian_dot(gl.AccessPattern(a_dev, 1), None, gl.AccessPattern(b_dev, 1), o_dev, gl.GL_EPILOGUE_RELU)
+
+    def e2e_step():
+        a_dev.copy_(a_pin, non_blocking=True)
+        b_dev.copy_(b_pin, non_blocking=True)
+        e2e_call()
+        o_pin.copy_(o_dev.tensor, non_blocking=True)
+
+    e2e_step()
+    torch.cuda.synchronize()
+    barrier()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    e2e_seconds = max_over_ranks(e0.elapsed_time(e1) * 1e-3, device)
+
+    if rank != 0:
+        return 0
+
+    value = aggregate_value(case.flops * args.steps, world, seconds_max) / 1e12
+    kernel_s = seconds / args.steps
+    achieved = case.flops / kernel_s / 1e12
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "dense_4096_dram_bytes_per_launch.txt")
+    if os.path.exists(tpath):
+        try:
+            traffic = float(open(tpath).read().split()[0])
+        except (ValueError, IndexError):
+            traffic = None
+    long_region = seconds > 1.0
+    peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) if long_region else peaks["bf16_tflops"]
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": warmup, "ms_per_step": seconds_max / args.steps * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": case.name, "M": case.m, "O": case.o, "K": case.k, "inputs": "N(0,1) seeded, bf16",
+                   "output": "fp32", "epilogue": "relu fused", "parallelism": "replicas x%d" % world,
+                   "l2": "rotating over %d buffer sets (%.0f MB) > L2" % (nsets, nsets * bytes_per_set / 1e6)},
+        "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                     "frac": achieved / peak, "traffic": traffic,
+                     "peak_source": "%s (%s)" % (peaks_kind, "sustained: timed region > 1 s" if long_region else "burst"),
+                     "frac_of_burst": achieved / peaks["bf16_tflops"],
+                     "frac_of_sustained": achieved / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
+                     "frac_of_nominal_2250": achieved / 2250.0, "kernel": "dot_tc (dense)",
+                     "kernel_us": kernel_s * 1e6},
+        "e2e": {"value": aggregate_value(case.flops * e2e_steps, world, e2e_seconds) / 1e12, "unit": "TFLOP/s",
+                "h2d_bytes_per_step": a_pin.numel() * 2 + b_pin.numel() * 2, "d2h_bytes_per_step": o_pin.numel() * 4,
+                "steps": e2e_steps},
+        "gpu_launches": args.steps, "clocks": clocks,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline_dense(args.cpu_seconds)
+    if world == 1 and args.detail:
+        line["detail"] = detail_workloads(device, peaks)
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=4000)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--detail", dest="detail", action="store_true", default=True)
+    ap.add_argument("--no-detail", dest="detail", action="store_false")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_gpu(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -332,3 +332,60 @@ def gl_strerror(code: int) -> str:
 
 def gl_version() -> int:
     return int(LIB.gl_version())
+
+
+class Prepared:
+    """A device call with its argument structures built once, for launch loops
+    where Python marshalling would otherwise outweigh a microsecond-scale kernel.
+    The stream is looked up at call time, so a prepared call can be captured
+    into a CUDA graph."""
+
+    def __init__(self, fn, args, keep):
+        self._fn, self._args, self._keep = fn, args, keep
+
+    def __call__(self, stream=None):
+        rc = self._fn(*self._args, _stream(stream))
+        if rc != GL_OK:
+            raise GlError(rc, self._fn.__name__)
+
+
+def _ws(workspace):
+    if workspace is None:
+        return 0, 0
+    ptr = (workspace.data_ptr() + 1023) // 1024 * 1024
+    return ptr, workspace.numel() * workspace.element_size() - (ptr - workspace.data_ptr())
+
+
+def prepare_cartesian_dot(a0: AccessPattern, w: Optional[GlWindows], a1: AccessPattern, out: AccessPattern,
+                          flags: int = 0, workspace: Optional[torch.Tensor] = None) -> Prepared:
+    s0, s1, so = _struct(a0), _struct(a1), _struct(out)
+    ws_ptr, ws_bytes = _ws(workspace)
+    args = (ctypes.byref(s0), _wptr(w), ctypes.byref(s1), ctypes.byref(so), flags, ws_ptr, ws_bytes)
+    return Prepared(LIB.gl_cartesian_dot, args, (s0, s1, so, w, a0, a1, out, workspace))
+
+
+def prepare_access_windows(a: AccessPattern, w: GlWindows, out: AccessPattern) -> Prepared:
+    sa, so = _struct(a), _struct(out)
+    return Prepared(LIB.gl_access_windows, (ctypes.byref(sa), ctypes.byref(w), ctypes.byref(so)), (sa, so, w, a, out))
+
+
+def prepare_access_transpose(a: AccessPattern, perm, out: AccessPattern) -> Prepared:
+    sa, so = _struct(a), _struct(out)
+    arr = (ctypes.c_int32 * len(perm))(*perm)
+    return Prepared(LIB.gl_access_transpose, (ctypes.byref(sa), arr, ctypes.byref(so)), (sa, so, arr, a, out))
+
+
+def prepare_compute_reduce_max(a: AccessPattern, w: Optional[GlWindows], out: AccessPattern) -> Prepared:
+    sa, so = _struct(a), _struct(out)
+    return Prepared(LIB.gl_compute_reduce_max, (ctypes.byref(sa), _wptr(w), ctypes.byref(so)), (sa, so, w, a, out))
+
+
+def prepare_compute_relu(a: AccessPattern, out: AccessPattern) -> Prepared:
+    sa, so = _struct(a), _struct(out)
+    return Prepared(LIB.gl_compute_relu, (ctypes.byref(sa), ctypes.byref(so)), (sa, so, a, out))
+
+
+def output_like(shape_fn_result, device) -> AccessPattern:
+    """Allocate the output described by a gl_shape_* result (shape, access_ndim, dtype)."""
+    shape, na, dt = shape_fn_result
+    return AccessPattern(torch.empty(shape, dtype=_TORCH[dt], device=device), na)

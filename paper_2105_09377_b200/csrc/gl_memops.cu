@@ -434,10 +434,24 @@ void fill_win_params(const gl_ap* in, const gl_windows* w, const gl_ap& A, WinPa
 }
 
 int device_smem_optin() {
+  static int cached = 0;   // same value on every B200 of a node
+  if (cached) return cached;
   int dev = 0, v = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return 0;
   if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return 0;
+  cached = v;
   return v;
+}
+
+constexpr int kIm2colMaxSmem = 160 * 1024;
+
+// Raises the kernel's dynamic shared-memory limit once (per process) instead of on every call.
+template <typename K>
+bool allow_big_smem(K kern, bool* done) {
+  if (*done) return true;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kIm2colMaxSmem) != cudaSuccess) return false;
+  *done = true;
+  return true;
 }
 
 template <typename T>
@@ -461,13 +475,12 @@ int run_windows(const gl_ap* in, const gl_windows* w, const gl_ap& A, gl_ap* out
     const int64_t wp = p.W + w->pad_lo[2] + w->pad_hi[2];
     const int64_t smem = ((p.K * 4 + 15) / 16) * 16 + p.C * p.Kh * wp * (int64_t)sizeof(T);
     const int64_t blocks = p.N * p.Ho;
-    if (smem <= 160 * 1024 && smem <= device_smem_optin() && blocks <= 0x7FFFFFFF && p.Wo * p.K < (1ll << 30)) {
+    if (smem <= kIm2colMaxSmem && smem <= device_smem_optin() && blocks <= 0x7FFFFFFF && p.Wo * p.K < (1ll << 30)) {
       p.Wp = static_cast<int>(wp);
       const bool vec = p.K % VEC == 0;
       auto kern = vec ? im2col_rows<T, VEC> : im2col_rows<T, 1>;
-      if (smem > 48 * 1024 &&
-          cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
-        return GL_ERR_CUDA;
+      static bool attr_done[2] = {false, false};
+      if (!allow_big_smem(kern, &attr_done[vec ? 1 : 0])) return GL_ERR_CUDA;
       kern<<<static_cast<unsigned>(blocks), kThreads, static_cast<size_t>(smem), st>>>(src, dst, p, fill);
       return launch_status();
     }

@@ -1,0 +1,103 @@
+"""Run one workload of the table in `synth` a few times on cuda:0.
+
+    python -m paper_2105_09377_b200.run_workload --workload conv3x3_56x56x64 --layout nhwc --iters 3
+
+Prints the mean time per call (CUDA events).  Meant for profilers and quick
+checks; the benchmark proper is bench.py.
+"""
+from __future__ import annotations
+
+import argparse
+import functools
+
+import numpy as np
+import torch
+
+from . import binding as gl
+from . import synth
+
+
+def _bf16(x, device):
+    return torch.from_numpy(synth.bf16_bits(x).view(np.int16)).to(device).view(torch.bfloat16).reshape(x.shape)
+
+
+@functools.lru_cache(maxsize=2)
+def _inputs(cfg, seed):
+    """Host inputs of a workload, kept so that several buffer sets can be filled from one draw."""
+    return cfg.inputs(seed)
+
+
+def workloads():
+    table = {c.name: c for c in (synth.CONV_TINY,) + synth.CONV_SWEEP_3X3 + synth.CONV_STRIDED_1X1}
+    table.update({c.name: c for c in (synth.MEM_IM2COL, synth.MEM_TRANSPOSE, synth.MEM_MAXPOOL)})
+    table[synth.DENSE_4096.name] = synth.DENSE_4096
+    return table
+
+
+def build_call(cfg, layout: str, device, batch=None, flags=0):
+    """Returns (prepared call, flops, algorithmic bytes)."""
+    if isinstance(cfg, synth.DenseCase):
+        a, b = _inputs(cfg, synth.config_seed(1))
+        aa, bb = gl.AccessPattern(_bf16(a, device), 1), gl.AccessPattern(_bf16(b, device), 1)
+        out = gl.output_like(gl.gl_shape_cartesian_dot(a.shape, 1, None, b.shape, 1), device)
+        return gl.prepare_cartesian_dot(aa, None, bb, out, flags | gl.GL_EPILOGUE_RELU), cfg.flops, cfg.algorithmic_bytes
+    if isinstance(cfg, synth.ConvCase):
+        if batch:
+            cfg = synth.ConvCase(cfg.name, batch, cfg.c, cfg.h, cfg.w, cfg.o, cfg.kh, cfg.kw, cfg.stride, cfg.pad, cfg.integer)
+        x, wt = _inputs(cfg, synth.config_seed(2))
+        if layout == "nhwc":
+            x, wt = x.transpose(0, 2, 3, 1).copy(), wt.transpose(0, 2, 3, 1).copy()
+            spec = gl.windows_spec((cfg.kh, cfg.kw, cfg.c), (cfg.stride, cfg.stride, 1), (cfg.pad, cfg.pad, 0), (cfg.pad, cfg.pad, 0))
+        else:
+            spec = gl.windows_spec((cfg.c, cfg.kh, cfg.kw), (1, cfg.stride, cfg.stride), (0, cfg.pad, cfg.pad), (0, cfg.pad, cfg.pad))
+        xa, wa = gl.AccessPattern(_bf16(x, device), 1), gl.AccessPattern(_bf16(wt, device), 1)
+        out = gl.output_like(gl.gl_shape_cartesian_dot(x.shape, 1, spec, wt.shape, 1), device)
+        need = gl.gl_cartesian_dot_workspace(xa, spec, wa, flags)
+        ws = torch.empty(need + 1024, dtype=torch.uint8, device=device) if need else None
+        return gl.prepare_cartesian_dot(xa, spec, wa, out, flags, ws), cfg.flops, cfg.algorithmic_bytes
+    if batch:
+        cfg = synth.MemCase(cfg.name, cfg.kind, (batch,) + tuple(cfg.shape[1:]), cfg.window, cfg.stride, cfg.pad, cfg.perm)
+    x = torch.from_numpy(_inputs(cfg, synth.config_seed(4))).to(device)
+    if cfg.kind == "transpose":
+        out = gl.output_like(gl.gl_shape_transpose(cfg.shape, 1, cfg.perm), device)
+        return gl.prepare_access_transpose(gl.AccessPattern(x, 1), cfg.perm, out), 0.0, cfg.algorithmic_bytes
+    if cfg.kind == "im2col":
+        c = cfg.shape[1]
+        spec = gl.windows_spec((c,) + cfg.window, (1, cfg.stride, cfg.stride), (0, cfg.pad, cfg.pad), (0, cfg.pad, cfg.pad))
+        out = gl.output_like(gl.gl_shape_windows(cfg.shape, 1, spec), device)
+        return gl.prepare_access_windows(gl.AccessPattern(x, 1), spec, out), 0.0, cfg.algorithmic_bytes
+    spec = gl.windows_spec(cfg.window, (cfg.stride,) * 2, (cfg.pad,) * 2, (cfg.pad,) * 2, gl.GL_PAD_NEG_INF)
+    out = gl.output_like(gl.gl_shape_reduce_max(cfg.shape, 2, spec), device)
+    return gl.prepare_compute_reduce_max(gl.AccessPattern(x, 2), spec, out), 0.0, cfg.algorithmic_bytes
+
+
+def main():
+    table = workloads()
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", required=True, choices=sorted(table))
+    ap.add_argument("--layout", default="nhwc", choices=["nhwc", "nchw"])
+    ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--batch", type=int, default=0, help="override the leading (batch) extent")
+    ap.add_argument("--general", action="store_true", help="use the general SIMT kernel for dot products")
+    args = ap.parse_args()
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    call, flops, nbytes = build_call(table[args.workload], args.layout, device, args.batch or None,
+                                     gl.GL_DOT_GENERAL_KERNEL if args.general else 0)
+    call()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.iters):
+        call()
+    e1.record()
+    torch.cuda.synchronize()
+    status = gl.gl_poll_device_status()
+    us = e0.elapsed_time(e1) * 1e3 / args.iters
+    print("%s %s: %.2f us/call, %.1f TFLOP/s, %.0f GB/s (algorithmic), status %d"
+          % (args.workload, args.layout, us, flops / us / 1e6, nbytes / us / 1e3, status))
+    return 0 if status == 0 else 1
+
+
+if __name__ == "__main__":
+    raise SystemExit(main())
