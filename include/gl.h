@@ -160,6 +160,32 @@ GL_API int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w_or_null, const 
 GL_API size_t gl_cartesian_dot_workspace(const gl_ap* a0, const gl_windows* w_or_null, const gl_ap* a1,
                                   uint32_t flags);
 
+/* gl_cartesian_dot for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a property of the host program, not of the method.)
+ *
+ * gl_cartesian_dot wants a caller-owned workspace whenever it has to make channels-last
+ * copies of its operands.  Code that runs where no allocator may be called - inside
+ * another framework's operator, in a plug-in that is handed nothing but its input and
+ * output buffers, in a process whose device memory is entirely owned by a pool - cannot
+ * provide one.  This variant takes no workspace: it uses a fixed scratch array of
+ * GL_STATIC_SCRATCH_BYTES (32 MiB) that is part of the library image, so every GPU that
+ * loads the library holds that much memory until the process exits.  It calls no
+ * cudaMalloc, cudaFree or other allocating routine.
+ *
+ *   - Same arguments, results and error codes as gl_cartesian_dot without the workspace
+ *     pair.  If gl_cartesian_dot_workspace() for these arguments exceeds
+ *     GL_STATIC_SCRATCH_BYTES the call returns GL_ERR_WORKSPACE and launches nothing
+ *     (for scale: the (C,H,W) activations of a 32x64x56x56 convolution need 12.3 MiB).
+ *   - The first call on each device looks up the array's device address (that device
+ *     must be current); make that first call before any stream capture begins.
+ *   - All calls share the one array and it keeps whatever the last call left in it.
+ *     Nothing in it has to start at zero: each call overwrites every byte it later
+ *     reads.  Two calls whose kernels can overlap on the GPU (different streams, or
+ *     different host threads without ordering) race on the array; order them. */
+#define GL_STATIC_SCRATCH_BYTES (32u << 20)
+GL_API int gl_cartesian_dot_static(const gl_ap* a0, const gl_windows* w_or_null, const gl_ap* a1, gl_ap* out,
+                                   uint32_t flags, void* stream);
+
 /* compute reduceMax (windows? in) (operator table, Fig. 2c max pooling): the largest
  * value of every item; with w given the windows are formed on the fly and never
  * stored.  GL_F32.  Inputs must be NaN-free. */

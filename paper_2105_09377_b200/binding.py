@@ -51,6 +51,7 @@ EXPORTS = [
     "gl_shape_cartesian_dot", "gl_shape_reduce_max", "gl_access_windows", "gl_access_flatten",
     "gl_access_transpose", "gl_access_pad", "gl_cartesian_dot", "gl_cartesian_dot_workspace",
     "gl_compute_reduce_max", "gl_compute_relu", "gl_poll_device_status", "gl_strerror", "gl_version",
+    "gl_cartesian_dot_static",
 ]
 
 
@@ -75,6 +76,7 @@ def _load() -> ctypes.CDLL:
         "gl_access_transpose": [ap, i32p, ap, vp],
         "gl_access_pad": [ap, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, ctypes.c_int32, ap, vp],
         "gl_cartesian_dot": [ap, win, ap, ap, ctypes.c_uint32, vp, ctypes.c_size_t, vp],
+        "gl_cartesian_dot_static": [ap, win, ap, ap, ctypes.c_uint32, vp],
         "gl_compute_reduce_max": [ap, win, ap, vp],
         "gl_compute_relu": [ap, ap, vp],
         "gl_poll_device_status": [vp],
@@ -298,6 +300,21 @@ def gl_cartesian_dot(a0: AccessPattern, w: Optional[GlWindows], a1: AccessPatter
     so = _struct(out)
     _check(LIB.gl_cartesian_dot(ctypes.byref(s0), _wptr(w), ctypes.byref(s1), ctypes.byref(so), flags, ws_ptr, ws_bytes,
                                 _stream(stream)), "gl_cartesian_dot")
+    return out
+
+
+GL_STATIC_SCRATCH_BYTES = 32 << 20
+
+
+def gl_cartesian_dot_static(a0: AccessPattern, w: Optional[GlWindows], a1: AccessPattern, out: AccessPattern,
+                            flags: int = 0, stream=None) -> AccessPattern:
+    """gl_cartesian_dot without a workspace argument, for callers that may not allocate device
+    memory: the scratch is a fixed 32 MiB array inside the library.  `out` must be supplied (this
+    wrapper allocates nothing either).  Calls that may overlap on the GPU must be ordered by the
+    caller, and the first call on a device should precede any stream capture."""
+    s0, s1, so = _struct(a0), _struct(a1), _struct(out)
+    _check(LIB.gl_cartesian_dot_static(ctypes.byref(s0), _wptr(w), ctypes.byref(s1), ctypes.byref(so), flags,
+                                       _stream(stream)), "gl_cartesian_dot_static")
     return out
 
 

@@ -790,3 +790,63 @@ int gl_poll_device_status(void* stream) {
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------
+// gl_cartesian_dot_static: the same operation for callers that cannot allocate
+// ------------------------------------------------------------------------
+//
+// gl_cartesian_dot needs a caller-supplied workspace when the activations come
+// in the (C,H,W) item layout (or with a channel count that is not a multiple
+// of 8): the channels-last copies live there.  Some hosts of this library have
+// no way to obtain that memory - code running inside a framework's operator
+// where the allocator is off limits, a plug-in that is only handed its input
+// and output buffers, a process that has given all device memory to a pool.
+// For them the scratch is a fixed array inside the library image.  Every GPU
+// that loads the library holds these bytes until the process exits.
+
+// GL_STATIC_SCRATCH_BYTES (gl.h) is what a call may use; 1024 more bytes absorb the alignment.
+static __device__ __align__(256) unsigned char g_static_scratch[GL_STATIC_SCRATCH_BYTES + 1024];
+
+namespace {
+
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void* g_scratch_addr[kMaxDevices] = {nullptr};
+
+// In host code `g_static_scratch` is only a handle for the runtime, not a
+// device address, so the address is asked for once per device (with that
+// device current) and remembered.
+int static_scratch_address(void** ptr) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return GL_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_scratch_mutex);
+  if (!g_scratch_addr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return GL_ERR_CUDA;
+    g_scratch_addr[dev] = p;
+  }
+  *ptr = g_scratch_addr[dev];
+  return GL_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int gl_cartesian_dot_static(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_ap* out, uint32_t flags,
+                            void* stream) {
+  // validate first, so that an over-sized request is told apart from a malformed one
+  DotProblem d;
+  int rc = classify_dot(a0, w, a1, &d);
+  if (rc) return rc;
+  const size_t need = gl_cartesian_dot_workspace(a0, w, a1, flags);
+  if (need > GL_STATIC_SCRATCH_BYTES) return GL_ERR_WORKSPACE;   // beyond the built-in scratch
+  void* base = nullptr;
+  rc = static_scratch_address(&base);
+  if (rc) return rc;
+  // the array is 256-byte aligned; the tensor maps want 1024
+  const uintptr_t aligned = (reinterpret_cast<uintptr_t>(base) + 1023u) & ~static_cast<uintptr_t>(1023u);
+  return gl_cartesian_dot(a0, w, a1, out, flags, reinterpret_cast<void*>(aligned), GL_STATIC_SCRATCH_BYTES, stream);
+}
+
+}  // extern "C"
