@@ -287,40 +287,66 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
 
 constexpr int kBM = 128;
 constexpr int kBK = 64;          // bf16 elements per K block = one 128-byte swizzle row
-constexpr int kTcThreads = 192;  // warp 0 TMA, warp 1 MMA + TMEM, warps 2-5 epilogue
+constexpr int kTcThreads = 224;  // warp 0 TMA (A), warp 1 MMA + TMEM, warps 2-5 epilogue, warp 6 TMA (B)
 
 enum AMode { kDense = 0, kIm2col = 1, kIm2colGranule = 2 };
+
+// Division of a 31-bit number by a fixed divisor as multiply-high + shift: the loops below run
+// in single threads, where an integer division is a ~150-cycle dependent chain.
+// With p = ceil(log2 d) and m = ceil(2^(31+p) / d):  n / d = umulhi(n, m) >> (p - 1)  for n < 2^31.
+struct FastDiv {
+  uint32_t d, mul, shift;
+  __host__ void set(int64_t divisor) {
+    d = static_cast<uint32_t>(divisor);
+    uint32_t p = 0;
+    while ((1ull << p) < d) ++p;
+    if (p == 0) { mul = 0; shift = 0; return; }
+    mul = static_cast<uint32_t>(((1ull << (31 + p)) + d - 1) / d);
+    shift = p - 1;
+  }
+  __device__ __forceinline__ uint32_t div(uint32_t n) const { return d == 1 ? n : (__umulhi(n, mul) >> shift); }
+  __device__ __forceinline__ void divmod(uint32_t n, uint32_t& q, uint32_t& r) const { q = div(n); r = n - q * d; }
+};
 
 struct TcParams {
   int64_t M, O, K;        // K as laid out in B (for conv: Kh*Kw*Cp)
   int tiles_m, tiles_n, kblocks;
   int relu;
+  int tma_store;          // result rows are 16-byte multiples: the epilogue may use TMA stores
   // conv only
   int Cp, Kh, Kw, Sh, Sw, ph, pw, Ho, Wo;
   int cchunks;            // kIm2col: 64-channel chunks per tap; kIm2colGranule: 8-channel granules per tap
+  FastDiv div_tiles_n, div_wo, div_howo;
 };
 
-template <int BN>
+// A stage holds G K-blocks of 64 (G A sub-tiles, then G B sub-tiles) behind one pair of barriers.
+// OCC = blocks per SM the configuration is sized for (2 only for BN <= 128: TMEM has 512 columns).
+template <int BN, int G, int OCC>
 struct TcCfg {
   static constexpr int kStageA = kBM * kBK * 2;
   static constexpr int kStageB = BN * kBK * 2;
-  static constexpr int kStage = kStageA + kStageB;
-  static constexpr int kStages = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
-  static constexpr int kTmemCols = 2 * BN;
-  static constexpr int kSmemBytes = kStages * kStage + 1024 /*alignment slack*/ + 256 /*barriers*/;
+  static constexpr int kStage = G * (kStageA + kStageB);
+  static constexpr int kEpiBufs = OCC == 2 ? 1 : 2;          // 32x32 fp32 staging tiles per epilogue warp
+  static constexpr int kEpiBytes = 4 * kEpiBufs * 4096;
+  static constexpr int kBudget = (OCC == 2 ? 113 * 1024 : 232448) - kEpiBytes - 1024 - 256;
+  static constexpr int kStages = kBudget / kStage > 8 ? 8 : kBudget / kStage;
+  static constexpr int kTmemCols = (2 * BN > 256) ? 512 : (2 * BN > 128 ? 256 : 128);   // power of two
+  static constexpr int kSmemBytes = kStages * kStage + kEpiBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
-template <int BN, int MODE>
-__global__ void __launch_bounds__(kTcThreads, 1)
+template <int BN, int MODE, int G, int OCC>
+__global__ void __launch_bounds__(kTcThreads, OCC)
 dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-       float* __restrict__ out, const TcParams p) {
-  using Cfg = TcCfg<BN>;
+       const __grid_constant__ CUtensorMap map_c, float* __restrict__ out, const TcParams p) {
+  using Cfg = TcCfg<BN, G, OCC>;
+  static_assert(Cfg::kStages >= 2, "ring too shallow");
   extern __shared__ unsigned char smem_raw[];
   // operand tiles need 1024-byte alignment for the 128-byte swizzle
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles = (raw + 1023u) & ~1023u;
   unsigned char* gen_tiles = smem_raw + (tiles - raw);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_tiles + Cfg::kStages * Cfg::kStage);
+  const uint32_t epi_base = tiles + Cfg::kStages * Cfg::kStage;      // 1024-byte aligned staging tiles
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen_tiles + Cfg::kStages * Cfg::kStage + Cfg::kEpiBytes);
   const uint32_t bar_full = smem_u32(bars);                          // [kStages]
   const uint32_t bar_empty = bar_full + 8 * Cfg::kStages;            // [kStages]
   const uint32_t bar_tfull = bar_empty + 8 * Cfg::kStages;           // [2]
@@ -331,7 +357,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < Cfg::kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+    for (int s = 0; s < Cfg::kStages; ++s) { mbar_init(bar_full + 8 * s, 2); mbar_init(bar_empty + 8 * s, 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, 4); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -350,51 +376,66 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
 
   const int num_tiles = p.tiles_m * p.tiles_n;
 
-  if (warp == 0) {
-    // ---------------- TMA producer ----------------
+  if (warp == 0 || warp == 6) {
+    // ---------------- TMA producers: warp 0 stages A, warp 6 stages B ----------------
+    // (issuing one TMA load costs its thread 150-200 cycles; two issuing warps halve that)
+    const bool load_a = warp == 0;
     if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
-      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(load_a ? &map_a : &map_b)) : "memory");
       uint32_t it = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-        const int tm = t / p.tiles_n, tn = t % p.tiles_n;
-        const int m0 = tm * kBM, n0 = tn * BN;
+        uint32_t tm, tn;
+        p.div_tiles_n.divmod(static_cast<uint32_t>(t), tm, tn);
+        const int m0 = static_cast<int>(tm) * kBM, n0 = static_cast<int>(tn) * BN;
         int wbase = 0, hbase = 0, img = 0;
-        if (MODE != kDense) {
-          const int wo = m0 % p.Wo, ho = (m0 / p.Wo) % p.Ho;
-          img = m0 / (p.Wo * p.Ho);
-          wbase = wo * p.Sw - p.pw;
-          hbase = ho * p.Sh - p.ph;
+        if (MODE != kDense && load_a) {
+          uint32_t im, rem, ho, wo;
+          p.div_howo.divmod(static_cast<uint32_t>(m0), im, rem);
+          p.div_wo.divmod(rem, ho, wo);
+          img = static_cast<int>(im);
+          wbase = static_cast<int>(wo) * p.Sw - p.pw;
+          hbase = static_cast<int>(ho) * p.Sh - p.ph;
         }
-        for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+        // filter position of the next K block, advanced without divisions
+        int cc = 0, kw = 0, kh = 0;
+        for (int kb0 = 0; kb0 < p.kblocks; kb0 += G, ++it) {
           const uint32_t s = it % Cfg::kStages, ph = (it / Cfg::kStages) & 1u;
           if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t full = bar_full + 8 * s;
-          const uint32_t sa = tiles + s * Cfg::kStage, sb = sa + Cfg::kStageA;
-          mbar_expect_tx(full, Cfg::kStage);
-          if (MODE == kDense) {
-            tma_load_2d(sa, &map_a, kb * kBK, m0, full);
-            tma_load_2d(sb, &map_b, kb * kBK, n0, full);
-          } else if (MODE == kIm2col) {
-            const int tap = kb / p.cchunks, c0 = (kb % p.cchunks) * kBK;
-            tma_load_im2col(sa, &map_a, c0, wbase, hbase, img, static_cast<uint16_t>(tap % p.Kw),
-                            static_cast<uint16_t>(tap / p.Kw), full);
-            tma_load_2d(sb, &map_b, tap * p.Cp + c0, n0, full);
-          } else {
-            // eight 8-channel granules per K block, each its own (pixels x 16 bytes) box
-            const int taps = p.Kh * p.Kw;
+          const uint32_t stage = tiles + s * Cfg::kStage;
+          const int nsub = min(G, p.kblocks - kb0);
+          mbar_expect_tx(full, nsub * (load_a ? Cfg::kStageA : Cfg::kStageB));
 #pragma unroll 1
-            for (int g = 0; g < 8; ++g) {
-              const int gi = kb * 8 + g;
-              const int tap = gi / p.cchunks;
-              // beyond the last tap: a box that lies outside the channel range reads as zeros
-              const int c0 = tap < taps ? (gi % p.cchunks) * 8 : p.Cp;
-              const int tp = tap < taps ? tap : 0;
-              tma_load_im2col(sa + g * (kBM * 16), &map_a, c0, wbase, hbase, img, static_cast<uint16_t>(tp % p.Kw),
-                              static_cast<uint16_t>(tp / p.Kw), full);
+          for (int j = 0; j < nsub; ++j) {
+            const int kb = kb0 + j;
+            const uint32_t sa = stage + j * Cfg::kStageA, sb = stage + G * Cfg::kStageA + j * Cfg::kStageB;
+            if (MODE == kDense) {
+              if (load_a) tma_load_2d(sa, &map_a, kb * kBK, m0, full);
+              else tma_load_2d(sb, &map_b, kb * kBK, n0, full);
+            } else if (MODE == kIm2col) {
+              if (load_a)
+                tma_load_im2col(sa, &map_a, cc * kBK, wbase, hbase, img, static_cast<uint16_t>(kw),
+                                static_cast<uint16_t>(kh), full);
+              else
+                tma_load_2d(sb, &map_b, (kh * p.Kw + kw) * p.Cp + cc * kBK, n0, full);
+              if (++cc == p.cchunks) { cc = 0; if (++kw == p.Kw) { kw = 0; ++kh; } }
+            } else if (load_a) {
+              // eight 8-channel granules per K block, each its own (pixels x 16 bytes) box
+              const int taps = p.Kh * p.Kw;
+#pragma unroll 1
+              for (int g = 0; g < 8; ++g) {
+                const int gi = kb * 8 + g;
+                const int tap = gi / p.cchunks;
+                // beyond the last tap: a box that lies outside the channel range reads as zeros
+                const int c0 = tap < taps ? (gi % p.cchunks) * 8 : p.Cp;
+                const int tp = tap < taps ? tap : 0;
+                tma_load_im2col(sa + g * (kBM * 16), &map_a, c0, wbase, hbase, img, static_cast<uint16_t>(tp % p.Kw),
+                                static_cast<uint16_t>(tp / p.Kw), full);
+              }
+            } else {
+              tma_load_3d(sb, &map_b, 0, n0, kb * 8, full);
             }
-            tma_load_3d(sb, &map_b, 0, n0, kb * 8, full);
           }
         }
       }
@@ -403,6 +444,9 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc(kBM, BN);
+      const uint64_t desc_a0 = (MODE == kIm2colGranule) ? make_desc(tiles, kBM * 16, 128, 0) : make_desc(tiles, 16, 1024, 2);
+      const uint64_t desc_b0 = (MODE == kIm2colGranule) ? make_desc(tiles + G * Cfg::kStageA, BN * 16, 128, 0)
+                                                        : make_desc(tiles + G * Cfg::kStageA, 16, 1024, 2);
       uint32_t it = 0, tile_it = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_it) {
@@ -410,37 +454,46 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
         if (!mbar_wait(bar_tempty + 8 * acc, aph ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int kb = 0; kb < p.kblocks; ++kb, ++it) {
+        for (int kb0 = 0; kb0 < p.kblocks; kb0 += G, ++it) {
           const uint32_t s = it % Cfg::kStages, ph = (it / Cfg::kStages) & 1u;
           if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sa = tiles + s * Cfg::kStage, sb = sa + Cfg::kStageA;
+          // descriptors differ only in their start-address field (16-byte units): add offsets to a base
+          const uint64_t da0 = desc_a0 + ((s * Cfg::kStage) >> 4);
+          const uint64_t db0 = desc_b0 + ((s * Cfg::kStage) >> 4);
+          const int nsub = min(G, p.kblocks - kb0);
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k) {
-            uint64_t da, db;
-            if (MODE == kIm2colGranule) {
-              da = make_desc(sa + k * 2 * (kBM * 16), kBM * 16, 128, 0);
-              db = make_desc(sb + k * 2 * (BN * 16), BN * 16, 128, 0);
-            } else {
-              da = make_desc(sa + k * 32, 16, 1024, 2);
-              db = make_desc(sb + k * 32, 16, 1024, 2);
+          for (int j = 0; j < G; ++j) {
+            if (j < nsub) {
+#pragma unroll
+              for (int k = 0; k < kBK / 16; ++k) {
+                constexpr int kStepA = (MODE == kIm2colGranule) ? 2 * (kBM * 16) : 32;
+                constexpr int kStepB = (MODE == kIm2colGranule) ? 2 * (BN * 16) : 32;
+                tc_mma_bf16(d_tmem, da0 + ((j * Cfg::kStageA + k * kStepA) >> 4),
+                            db0 + ((j * Cfg::kStageB + k * kStepB) >> 4), idesc, (kb0 | j | k) != 0 ? 1u : 0u);
+              }
             }
-            tc_mma_bf16(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
           }
-          tc_commit(bar_empty + 8 * s);   // frees the stage once these MMAs have read it
+          // one commit per stage (it costs the issuing thread a few hundred cycles): frees the
+          // stage once these MMAs have read it
+          tc_commit(bar_empty + 8 * s);
         }
         if (ok) tc_commit(bar_tfull + 8 * acc);
       }
     }
   } else {
-    // ---------------- epilogue: TMEM -> registers -> global ----------------
+    // ---------------- epilogue: TMEM -> registers -> (shared memory -> TMA store | global) ----------------
     const int q = warp & 3;   // TMEM lane quarter this warp may read
-    uint32_t tile_it = 0;
+    uint32_t tile_it = 0, chunk_it = 0;
     bool ok = true;
     const bool vec_ok = (p.O & 3) == 0;
+    const uint32_t stage_buf = epi_base + q * (Cfg::kEpiBufs * 4096);   // this warp's 32 rows x 128 bytes tiles
+    if (p.tma_store && lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_c)) : "memory");
     for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_it) {
       const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
-      const int tm = t / p.tiles_n, tn = t % p.tiles_n;
+      uint32_t tmu, tnu;
+      p.div_tiles_n.divmod(static_cast<uint32_t>(t), tmu, tnu);
+      const int tm = static_cast<int>(tmu), tn = static_cast<int>(tnu);
       if (!mbar_wait(bar_tfull + 8 * acc, aph, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const int64_t m = static_cast<int64_t>(tm) * kBM + q * 32 + lane;
@@ -455,7 +508,32 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
 #pragma unroll
           for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(fmaxf(__uint_as_float(r[i]), 0.f));
         }
-        if (m < p.M) {
+        if (p.tma_store) {
+          // 32x32 fp32 block: each lane parks its row in shared memory (16-byte pieces XOR-swizzled by
+          // row, the 128-byte swizzle of the tensor map), then one lane hands the block to the TMA unit,
+          // which writes whole 128-byte rows and clips at the matrix edge.
+          const uint32_t buf = stage_buf + (Cfg::kEpiBufs == 2 ? (chunk_it & 1u) * 4096 : 0u);
+          if (lane == 0) {   // the store that last used this buffer has read it
+            if (Cfg::kEpiBufs == 2) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            else asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          }
+          __syncwarp();
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(buf + lane * 128 + ((j ^ (lane & 7)) << 4)),
+                         "r"(r[4 * j]), "r"(r[4 * j + 1]), "r"(r[4 * j + 2]), "r"(r[4 * j + 3])
+                         : "memory");
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) {
+            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
+                             reinterpret_cast<uint64_t>(&map_c)),
+                         "r"(static_cast<int>(n0)), "r"(tm * kBM + q * 32), "r"(buf)
+                         : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          }
+          ++chunk_it;
+        } else if (m < p.M) {
           if (vec_ok && n0 + 32 <= p.O) {
 #pragma unroll
             for (int i = 0; i < 32; i += 4)
@@ -471,6 +549,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
     }
+    if (p.tma_store && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   // teardown: a block that gave up lets its copies in flight land before it leaves
@@ -574,19 +653,40 @@ bool encode_im2col(CUtensorMap* m, const void* base, const DotProblem& d, int64_
                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int MODE>
-int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, const TcParams& p, cudaStream_t st) {
-  using Cfg = TcCfg<BN>;
+// fp32 result [M, O]: 32x32 boxes, 128-byte swizzle (what the epilogue stages).
+bool encode_result(CUtensorMap* m, float* base, int64_t M, int64_t O) {
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(O), static_cast<cuuint64_t>(M)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(O) * 4};
+  const cuuint32_t box[2] = {32, 32};
+  const cuuint32_t estr[2] = {1, 1};
+  return driver_api().tiled(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN, int MODE, int G, int OCC>
+int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams p, cudaStream_t st) {
+  using Cfg = TcCfg<BN, G, OCC>;
   static bool attr_set = false;   // benign race: the attribute call is idempotent
   if (!attr_set) {
-    if (cudaFuncSetAttribute(dot_tc<BN, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) !=
+    if (cudaFuncSetAttribute(dot_tc<BN, MODE, G, OCC>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) !=
         cudaSuccess)
       return GL_ERR_CUDA;
     attr_set = true;
   }
+  p.div_tiles_n.set(p.tiles_n);
+  p.div_wo.set(p.Wo > 0 ? p.Wo : 1);
+  p.div_howo.set(p.Wo > 0 ? static_cast<int64_t>(p.Wo) * p.Ho : 1);
+  CUtensorMap mc;
+  p.tma_store = (p.O % 4 == 0) ? 1 : 0;
+  if (p.tma_store) {
+    if (!encode_result(&mc, out, p.M, p.O)) return GL_ERR_CUDA;
+  } else {
+    mc = ma;   // unused by the kernel; any valid map
+  }
   const int tiles = p.tiles_m * p.tiles_n;
-  const int grid = tiles < num_sms() ? tiles : num_sms();
-  dot_tc<BN, MODE><<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(ma, mb, out, p);
+  const int grid = tiles < OCC * num_sms() ? tiles : OCC * num_sms();
+  dot_tc<BN, MODE, G, OCC><<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(ma, mb, mc, out, p);
   return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;
 }
 
@@ -594,20 +694,24 @@ template <int MODE>
 int launch_tc_bn(int bn, const CUtensorMap& ma, const CUtensorMap& mb, float* out, const TcParams& p,
                  cudaStream_t st) {
   switch (bn) {
-    case 256: return launch_tc<256, MODE>(ma, mb, out, p, st);
-    case 128: return launch_tc<128, MODE>(ma, mb, out, p, st);
-    default: return launch_tc<64, MODE>(ma, mb, out, p, st);
+    case 256: return launch_tc<256, MODE, 1, 1>(ma, mb, out, p, st);
+    // narrower tiles are bound by the MMA-issuing thread (about 50 cycles per MMA, 250 per commit):
+    // 128 wide: two K blocks per stage halve the commits; 64 wide: two blocks per SM interleave
+    // their issue threads (measured on the 3x3 and 1x1 convolution shapes)
+    case 128: return launch_tc<128, MODE, 2, 1>(ma, mb, out, p, st);
+    default:
+      if (MODE == kIm2colGranule) return launch_tc<64, MODE, 1, 1>(ma, mb, out, p, st);
+      return launch_tc<64, MODE, 1, 2>(ma, mb, out, p, st);
   }
 }
 
-// Column-tile width: the widest tile that still leaves every SM a tile.
+// Column-tile width: 256 when that still leaves every SM a tile (wide tiles halve the operand
+// traffic per flop), else the narrowest width that covers O in one or few tiles.
 int pick_bn(int64_t M, int64_t O) {
   const int64_t tiles_m = (M + kBM - 1) / kBM;
   const int sms = num_sms();
-  for (int bn : {256, 128}) {
-    if (O > bn / 2 && tiles_m * ((O + bn - 1) / bn) >= sms) return bn;
-  }
-  return 64;
+  if (O > 128 && tiles_m * ((O + 255) / 256) >= sms) return 256;
+  return O > 64 ? 128 : 64;
 }
 
 struct ConvPlan {

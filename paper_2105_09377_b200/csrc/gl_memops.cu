@@ -7,6 +7,8 @@
 // would otherwise scatter.
 #include <cuda_runtime.h>
 
+#include <algorithm>
+#include <cmath>
 #include <cstring>
 
 #include "gl_internal.h"
@@ -317,11 +319,15 @@ __global__ void __launch_bounds__(kThreads) window_max_generic(const float* __re
 // Convolution-style windows over ((N),(C,H,W)) items with window (C,Kh,Kw) and
 // strides (1,Sh,Sw): the im2col matrix of Section 5.3, rows (n,h',w'), columns
 // (c,kh,kw).  One block owns one (n,h'): it stages the Kh input rows of every
-// channel in shared memory (zero or -inf border included), then streams the
+// channel in shared memory (border cells hold the fill value), then streams the
 // Wo x K output slab, which is contiguous in memory, with 128-bit stores.
+// Indexing is by warp (one staged row, then one output row per warp pass), so
+// the inner loops carry no divisions; the staged row pitch is chosen on the host
+// to spread the (c,kh,kw) gather over the shared-memory banks.
 struct Im2colParams {
   int64_t N, C, H, W, Kh, Kw, Sh, Sw, ph_lo, pw_lo, Ho, Wo, K;
   int Wp;       // staged row length = W + pw_lo + pw_hi
+  int pitch;    // staged row pitch in elements (>= Wp)
 };
 
 template <typename T, int VEC>
@@ -329,36 +335,94 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
                                                         const Im2colParams p, T fill) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   int* lut = reinterpret_cast<int*>(smem_raw);                     // K entries: staged offset of column k at w'=0
-  T* stage = reinterpret_cast<T*>(smem_raw + ((p.K * 4 + 15) / 16) * 16);   // [C][Kh][Wp]
+  T* stage = reinterpret_cast<T*>(smem_raw + ((p.K * 4 + 15) / 16) * 16);   // [C*Kh][pitch]
   const int64_t n = blockIdx.x / p.Ho, ho = blockIdx.x % p.Ho;
-  const int rows = static_cast<int>(p.C * p.Kh);
-  for (int k = threadIdx.x; k < p.K; k += blockDim.x) {
-    const int kw = k % static_cast<int>(p.Kw), ckh = k / static_cast<int>(p.Kw);
-    lut[k] = ckh * p.Wp + kw;
-  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+  const int rows = static_cast<int>(p.C * p.Kh), Kw = static_cast<int>(p.Kw), Kh = static_cast<int>(p.Kh);
+  const int K = static_cast<int>(p.K), W = static_cast<int>(p.W), pw = static_cast<int>(p.pw_lo);
+  for (int k = threadIdx.x; k < K; k += blockDim.x) lut[k] = (k / Kw) * p.pitch + k % Kw;
   const int64_t h0 = ho * p.Sh - p.ph_lo;
-  for (int e = threadIdx.x; e < rows * p.Wp; e += blockDim.x) {
-    const int x = e % p.Wp, r = e / p.Wp;
-    const int kh = r % static_cast<int>(p.Kh), c = r / static_cast<int>(p.Kh);
-    const int64_t h = h0 + kh, w = x - p.pw_lo;
-    stage[e] = (h >= 0 && h < p.H && w >= 0 && w < p.W) ? in[((n * p.C + c) * p.H + h) * p.W + w] : fill;
-  }
-  __syncthreads();
-  T* dst = out + (n * p.Ho + ho) * p.Wo * p.K;
-  const int total = static_cast<int>(p.Wo * p.K);
-  union Chunk { uint4 v; T e[VEC]; };
-  for (int e = threadIdx.x * VEC; e < total; e += blockDim.x * VEC) {
-    const int wo = e / static_cast<int>(p.K), k = e - wo * static_cast<int>(p.K);
-    const int shift = wo * static_cast<int>(p.Sw);
-    if (VEC == 1) {
-      dst[e] = stage[lut[k] + shift];
-    } else {
-      Chunk ch;
+  // staging: four rows per warp pass so that several global loads are in flight per thread
+  for (int r0 = warp * 4; r0 < rows; r0 += nwarps * 4) {
+    for (int x = lane; x < p.Wp; x += 32) {
+      const int w = x - pw;
+      const bool col_ok = w >= 0 && w < W;
+      T v[4];
 #pragma unroll
-      for (int i = 0; i < VEC; ++i) ch.e[i] = stage[lut[k + i] + shift];
-      *reinterpret_cast<uint4*>(dst + e) = ch.v;
+      for (int i = 0; i < 4; ++i) {
+        const int r = r0 + i;
+        const int c = r / Kh, kh = r - c * Kh;
+        const int64_t h = h0 + kh;
+        v[i] = (r < rows && col_ok && h >= 0 && h < p.H) ? in[((n * p.C + c) * p.H + h) * p.W + w] : fill;
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (r0 + i < rows) stage[(r0 + i) * p.pitch + x] = v[i];
     }
   }
+  __syncthreads();
+  T* slab = out + (n * p.Ho + ho) * p.Wo * p.K;
+  const int Wo = static_cast<int>(p.Wo), Sw = static_cast<int>(p.Sw);
+  union Chunk { uint4 v; T e[VEC]; };
+  constexpr int kLutPasses = 5;
+  int lutreg[kLutPasses][VEC];
+  if (VEC > 1 && K <= kLutPasses * 32 * VEC) {
+#pragma unroll
+    for (int t = 0; t < kLutPasses; ++t)
+#pragma unroll
+      for (int i = 0; i < VEC; ++i) {
+        const int k = (t * 32 + lane) * VEC + i;
+        lutreg[t][i] = k < K ? lut[k] : 0;
+      }
+  }
+  for (int wo = warp; wo < Wo; wo += nwarps) {
+    const T* base = stage + wo * Sw;
+    T* orow = slab + static_cast<int64_t>(wo) * K;
+    if (VEC == 1) {
+      for (int k = lane; k < K; k += 32) orow[k] = base[lut[k]];
+    } else if (K <= kLutPasses * 32 * VEC) {
+      // the gather offsets of this lane do not depend on the output row: keep them in registers
+#pragma unroll
+      for (int t = 0; t < kLutPasses; ++t) {
+        const int k = (t * 32 + lane) * VEC;
+        if (k < K) {
+          Chunk ch;
+#pragma unroll
+          for (int i = 0; i < VEC; ++i) ch.e[i] = base[lutreg[t][i]];
+          *reinterpret_cast<uint4*>(orow + k) = ch.v;
+        }
+      }
+    } else {
+      for (int k = lane * VEC; k < K; k += 32 * VEC) {
+        Chunk ch;
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) ch.e[i] = base[lut[k + i]];
+        *reinterpret_cast<uint4*>(orow + k) = ch.v;
+      }
+    }
+  }
+}
+
+// Row pitch (>= Wp, < Wp + 32) with the fewest shared-memory bank conflicts for the
+// gather "lane reads staged[(k/Kw)*pitch + k%Kw], k = VEC*lane + i" (4-byte banks).
+int best_im2col_pitch(int Wp, int Kw, int K, int vec, int elem_bytes) {
+  int best = Wp, best_cost = 1 << 30;
+  for (int pitch = Wp; pitch < Wp + 32; ++pitch) {
+    int cost = 0;
+    for (int pass = 0; pass * 32 * vec < K && pass < 8; ++pass)
+      for (int i = 0; i < vec; ++i) {
+        int hits[32] = {0}, worst = 0;
+        for (int lane = 0; lane < 32; ++lane) {
+          const int k = pass * 32 * vec + lane * vec + i;
+          if (k >= K) break;
+          const int bank = (((k / Kw) * pitch + k % Kw) * elem_bytes / 4) & 31;
+          worst = std::max(worst, ++hits[bank]);
+        }
+        cost += worst;
+      }
+    if (cost < best_cost) { best_cost = cost; best = pitch; }
+  }
+  return best;
 }
 
 // 2D windows + reduceMax over ((..),(H,W)) items (Fig. 2c): one thread per output.
@@ -380,6 +444,107 @@ __global__ void __launch_bounds__(kThreads) window_max_2d(const float* __restric
       }
     }
     out[c] = best;
+  }
+}
+
+// 2D windows + reduceMax, tiled: one block owns TH output rows of one plane.  It
+// stages the (TH-1)*Sh+Kh input rows it needs (border cells hold the fill value)
+// with 128-bit loads, then every thread reduces whole windows out of shared
+// memory.  Each input cell is read from HBM once per block.
+struct PoolTile {
+  int H, W, Kh, Kw, Sh, Sw, ph, pw, Ho, Wo;
+  int TH;        // output rows per block
+  int tiles;     // row tiles per plane
+  int Wp;        // staged row length = pw + W + right border
+  int vec;       // rows are 16-byte multiples: float4 loads
+};
+
+__global__ void __launch_bounds__(kThreads) window_max_2d_tiled(const float* __restrict__ in, float* __restrict__ out,
+                                                                 const PoolTile p, float fill) {
+  extern __shared__ __align__(16) float pool_stage[];
+  const int64_t plane = blockIdx.x / p.tiles;
+  const int tile = blockIdx.x % p.tiles;
+  const int y0 = tile * p.TH;
+  const int th = min(p.TH, p.Ho - y0);
+  const int rows = (th - 1) * p.Sh + p.Kh;
+  const int h0 = y0 * p.Sh - p.ph;
+  const float* src = in + plane * p.H * p.W;
+  // left and right border columns, then the rows themselves
+  const int right = p.Wp - p.pw - p.W;
+  for (int e = threadIdx.x; e < rows * (p.pw + right); e += blockDim.x) {
+    const int r = e / (p.pw + right), j = e % (p.pw + right);
+    pool_stage[r * p.Wp + (j < p.pw ? j : p.W + j)] = fill;
+  }
+  if (p.vec) {
+    const int w4 = p.W >> 2;
+    for (int e = threadIdx.x; e < rows * w4; e += blockDim.x) {
+      const int r = e / w4, x = (e - r * w4) << 2;
+      const int h = h0 + r;
+      float4 v = make_float4(fill, fill, fill, fill);
+      if (h >= 0 && h < p.H) v = *reinterpret_cast<const float4*>(src + (int64_t)h * p.W + x);
+      float* d = pool_stage + r * p.Wp + p.pw + x;
+      d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+    }
+  } else {
+    for (int e = threadIdx.x; e < rows * p.W; e += blockDim.x) {
+      const int r = e / p.W, x = e - r * p.W;
+      const int h = h0 + r;
+      pool_stage[r * p.Wp + p.pw + x] = (h >= 0 && h < p.H) ? src[(int64_t)h * p.W + x] : fill;
+    }
+  }
+  __syncthreads();
+  float* dst = out + (plane * p.Ho + y0) * p.Wo;
+  for (int e = threadIdx.x; e < th * p.Wo; e += blockDim.x) {
+    const int y = e / p.Wo, x = e - y * p.Wo;
+    const float* win = pool_stage + (y * p.Sh) * p.Wp + x * p.Sw;
+    float best = -INFINITY;
+    for (int dy = 0; dy < p.Kh; ++dy)
+      for (int dx = 0; dx < p.Kw; ++dx) best = fmaxf(best, win[dy * p.Wp + dx]);
+    dst[e] = best;
+  }
+}
+
+// Fig. 2c with a 3x3 window, stride 2 and one border cell on the low side (the pooling layer of
+// ResNet-style networks), rows that are multiples of four floats: no staging at all.  A thread
+// owns four input columns (two outputs) and walks R output rows downwards; each input row is read
+// once with one 128-bit load plus the neighbour's last column, its two horizontal maxima are kept
+// in registers, and the odd rows are shared by two consecutive output rows.
+struct Pool3s2 {
+  int H, W, Ho, Wo, R, strips, w4;
+  int64_t units;   // planes * strips
+};
+
+__global__ void __launch_bounds__(256) window_max_3x3s2(const float* __restrict__ in, float* __restrict__ out,
+                                                         const Pool3s2 p, float fill) {
+  const int64_t u = blockIdx.x * (int64_t)blockDim.y + threadIdx.y;
+  if (u >= p.units) return;
+  const int64_t plane = u / p.strips;
+  const int strip = static_cast<int>(u - plane * p.strips);
+  const float* src = in + plane * p.H * p.W;
+  float* dst = out + plane * p.Ho * p.Wo;
+  const int y0 = strip * p.R, y1 = min(p.Ho, y0 + p.R);
+  for (int j = threadIdx.x; j < p.w4; j += blockDim.x) {
+    const int x = 4 * j;
+    auto hmax = [&](int h, float& m0, float& m1) {
+      if (h < 0 || h >= p.H) { m0 = m1 = fill; return; }
+      const float* row = src + (int64_t)h * p.W + x;
+      const float4 v = *reinterpret_cast<const float4*>(row);
+      const float left = j > 0 ? row[-1] : fill;
+      m0 = fmaxf(fmaxf(left, v.x), v.y);
+      m1 = fmaxf(fmaxf(v.y, v.z), v.w);
+    };
+    float c0, c1;
+    hmax(2 * y0 - 1, c0, c1);
+#pragma unroll 2
+    for (int y = y0; y < y1; ++y) {
+      float a0, a1, b0, b1;
+      hmax(2 * y, a0, a1);
+      hmax(2 * y + 1, b0, b1);
+      const float o0 = fmaxf(fmaxf(c0, a0), b0), o1 = fmaxf(fmaxf(c1, a1), b1);
+      if (2 * j + 1 < p.Wo) *reinterpret_cast<float2*>(dst + (int64_t)y * p.Wo + 2 * j) = make_float2(o0, o1);
+      else if (2 * j < p.Wo) dst[(int64_t)y * p.Wo + 2 * j] = o0;
+      c0 = b0; c1 = b1;
+    }
   }
 }
 
@@ -473,11 +638,16 @@ int run_windows(const gl_ap* in, const gl_windows* w, const gl_ap& A, gl_ap* out
     p.Ho = A.shape[na + 1]; p.Wo = A.shape[na + 2];
     p.K = p.C * p.Kh * p.Kw;
     const int64_t wp = p.W + w->pad_lo[2] + w->pad_hi[2];
-    const int64_t smem = ((p.K * 4 + 15) / 16) * 16 + p.C * p.Kh * wp * (int64_t)sizeof(T);
+    const bool vec = p.K % VEC == 0;
+    const int pitch = wp < (1 << 20) && p.K < (1 << 24)
+                          ? best_im2col_pitch(static_cast<int>(wp), static_cast<int>(p.Kw), static_cast<int>(p.K),
+                                              vec ? VEC : 1, static_cast<int>(sizeof(T)))
+                          : static_cast<int>(wp);
+    const int64_t smem = ((p.K * 4 + 15) / 16) * 16 + p.C * p.Kh * pitch * (int64_t)sizeof(T);
     const int64_t blocks = p.N * p.Ho;
     if (smem <= kIm2colMaxSmem && smem <= device_smem_optin() && blocks <= 0x7FFFFFFF && p.Wo * p.K < (1ll << 30)) {
       p.Wp = static_cast<int>(wp);
-      const bool vec = p.K % VEC == 0;
+      p.pitch = pitch;
       auto kern = vec ? im2col_rows<T, VEC> : im2col_rows<T, 1>;
       static bool attr_done[2] = {false, false};
       if (!allow_big_smem(kern, &attr_done[vec ? 1 : 0])) return GL_ERR_CUDA;
@@ -587,6 +757,49 @@ int gl_compute_reduce_max(const gl_ap* in, const gl_windows* w, gl_ap* out, void
   const float fill = w->pad_kind == GL_PAD_NEG_INF ? -INFINITY : 0.0f;
   const int64_t nwin = numel(want);
   const int na = in->access_ndim;
+  if (w->n == 2 && w->wshape[0] == 3 && w->wshape[1] == 3 && w->stride[0] == 2 && w->stride[1] == 2 &&
+      w->pad_lo[0] == 1 && w->pad_lo[1] == 1 && in->shape[na + 1] % 4 == 0 && in->shape[na] < (1 << 20) &&
+      in->shape[na + 1] < (1 << 20) && A.shape[na + 1] % 2 == 0) {
+    Pool3s2 t;
+    t.H = (int)in->shape[na]; t.W = (int)in->shape[na + 1];
+    t.Ho = (int)A.shape[na]; t.Wo = (int)A.shape[na + 1];
+    t.R = 7;
+    t.strips = (t.Ho + t.R - 1) / t.R;
+    t.w4 = t.W / 4;
+    t.units = prod(in->shape, 0, na) * t.strips;
+    const int64_t blocks = (t.units + 7) / 8;
+    if (blocks <= 0x7FFFFFFF) {
+      window_max_3x3s2<<<static_cast<unsigned>(blocks), dim3(32, 8), 0, st>>>(src, dst, t, fill);
+      return launch_status();
+    }
+  }
+  if (w->n == 2 && in->shape[na] < (1 << 20) && in->shape[na + 1] < (1 << 20) && w->wshape[0] < 1024 &&
+      w->wshape[1] < 1024 && w->stride[0] < 1024 && w->stride[1] < 1024) {
+    PoolTile t;
+    t.H = (int)in->shape[na]; t.W = (int)in->shape[na + 1];
+    t.Kh = (int)w->wshape[0]; t.Kw = (int)w->wshape[1];
+    t.Sh = (int)w->stride[0]; t.Sw = (int)w->stride[1];
+    t.ph = (int)w->pad_lo[0]; t.pw = (int)w->pad_lo[1];
+    t.Ho = (int)A.shape[na]; t.Wo = (int)A.shape[na + 1];
+    // staged columns: left border, the row, and whatever the last window reaches beyond it
+    t.Wp = std::max(t.pw + t.W, (t.Wo - 1) * t.Sw + t.Kw);
+    t.vec = (t.W % 4 == 0) ? 1 : 0;
+    const int budget = 24 * 1024 / 4;   // floats of shared memory per block
+    const int max_rows = budget / t.Wp;
+    const int64_t planes = prod(in->shape, 0, na);
+    if (max_rows >= t.Kh) {
+      t.TH = std::min(t.Ho, (max_rows - t.Kh) / t.Sh + 1);
+      t.tiles = (t.Ho + t.TH - 1) / t.TH;
+      t.TH = (t.Ho + t.tiles - 1) / t.tiles;   // even out the tiles
+      const int rows = (t.TH - 1) * t.Sh + t.Kh;
+      const int64_t blocks = planes * t.tiles;
+      if (blocks <= 0x7FFFFFFF) {
+        window_max_2d_tiled<<<static_cast<unsigned>(blocks), kThreads, static_cast<size_t>(rows) * t.Wp * 4, st>>>(
+            src, dst, t, fill);
+        return launch_status();
+      }
+    }
+  }
   if (w->n == 2 && in->shape[na] < (1 << 30) && in->shape[na + 1] < (1 << 30)) {
     window_max_2d<<<grid_for(nwin, kThreads), kThreads, 0, st>>>(
         src, dst, prod(in->shape, 0, na), (int)in->shape[na], (int)in->shape[na + 1], (int)w->wshape[0],

@@ -78,6 +78,7 @@ def main():
     ap.add_argument("--layout", default="nhwc", choices=["nhwc", "nchw"])
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--batch", type=int, default=0, help="override the leading (batch) extent")
+    ap.add_argument("--graph", action="store_true", help="time one CUDA graph holding all iterations")
     ap.add_argument("--general", action="store_true", help="use the general SIMT kernel for dot products")
     args = ap.parse_args()
     device = torch.device("cuda", 0)
@@ -87,10 +88,26 @@ def main():
     call()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(args.iters):
-        call()
-    e1.record()
+    if args.graph:
+        # replay the calls from one CUDA graph: host launch cost no longer paces short kernels
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            call()
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            for _ in range(args.iters):
+                call()
+        graph.replay()
+        torch.cuda.synchronize()
+        e0.record()
+        graph.replay()
+        e1.record()
+    else:
+        e0.record()
+        for _ in range(args.iters):
+            call()
+        e1.record()
     torch.cuda.synchronize()
     status = gl.gl_poll_device_status()
     us = e0.elapsed_time(e1) * 1e3 / args.iters
