@@ -850,10 +850,25 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
       weights_to_channels_last<<<static_cast<unsigned>(std::min<int64_t>((d.O * T * pl.Cp + 255) / 256, 1 << 20)), 256, 0,
                                  st>>>(pb, ws, d.O * T, d.C, 1, pl.Cp);
     } else {
-      if (d.N > 65535 || (d.C + 31) / 32 > 65535) return GL_ERR_UNSUPPORTED;
-      const dim3 grid(static_cast<unsigned>((HW + 31) / 32), static_cast<unsigned>((pl.Cp + 31) / 32),
-                      static_cast<unsigned>(d.N));
-      nchw_to_nhwc_pad<<<grid, 256, 0, st>>>(pa, xs, d.C, HW, pl.Cp);
+      if (pl.Cp == d.C) {
+        // no channel padding: (N,C,HW) -> (N,HW,C) is the library's own tiled transpose
+        gl_ap src, dstp;
+        std::memset(&src, 0, sizeof(src));
+        src.data = const_cast<uint16_t*>(pa);
+        src.dtype = GL_BF16; src.ndim = 3; src.access_ndim = 1;
+        src.shape[0] = d.N; src.shape[1] = d.C; src.shape[2] = HW;
+        dstp = src;
+        dstp.data = xs;
+        dstp.shape[1] = HW; dstp.shape[2] = d.C;
+        const int32_t perm[3] = {0, 2, 1};
+        rc = gl_access_transpose(&src, perm, &dstp, stream);
+        if (rc) return rc;
+      } else {
+        if (d.N > 65535 || (d.C + 31) / 32 > 65535) return GL_ERR_UNSUPPORTED;
+        const dim3 grid(static_cast<unsigned>((HW + 31) / 32), static_cast<unsigned>((pl.Cp + 31) / 32),
+                        static_cast<unsigned>(d.N));
+        nchw_to_nhwc_pad<<<grid, 256, 0, st>>>(pa, xs, d.C, HW, pl.Cp);
+      }
       weights_to_channels_last<<<static_cast<unsigned>(std::min<int64_t>((d.O * T * pl.Cp + 255) / 256, 1 << 20)), 256, 0,
                                  st>>>(pb, ws, d.O, d.C, T, pl.Cp);
     }

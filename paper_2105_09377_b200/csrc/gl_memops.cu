@@ -343,21 +343,59 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
   for (int k = threadIdx.x; k < K; k += blockDim.x) lut[k] = (k / Kw) * p.pitch + k % Kw;
   const int64_t h0 = ho * p.Sh - p.ph_lo;
   // staging: four rows per warp pass so that several global loads are in flight per thread
-  for (int r0 = warp * 4; r0 < rows; r0 += nwarps * 4) {
-    for (int x = lane; x < p.Wp; x += 32) {
-      const int w = x - pw;
-      const bool col_ok = w >= 0 && w < W;
-      T v[4];
+  constexpr int LV = 16 / sizeof(T);   // elements per 128-bit load
+  if (p.W % LV == 0) {
+    // rows are 16-byte multiples: border cells first, then eight rows per warp pass with one
+    // 128-bit load per lane and row, all requested before any is stored
+    const int border = p.Wp - W;
+    for (int e = threadIdx.x; e < rows * border; e += blockDim.x) {
+      const int r = e / border, j = e - r * border;
+      stage[r * p.pitch + (j < pw ? j : W + j)] = fill;
+    }
+    const int wv = W / LV;
+    union Vec { uint4 v; T e[LV]; };
+    for (int r0 = warp * 8; r0 < rows; r0 += nwarps * 8) {
+      for (int l = lane; l < wv; l += 32) {
+        Vec v[8];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int r = r0 + i;
-        const int c = r / Kh, kh = r - c * Kh;
-        const int64_t h = h0 + kh;
-        v[i] = (r < rows && col_ok && h >= 0 && h < p.H) ? in[((n * p.C + c) * p.H + h) * p.W + w] : fill;
+        for (int i = 0; i < 8; ++i) {
+          const int r = r0 + i;
+          const int c = r / Kh, kh = r - c * Kh;
+          const int64_t h = h0 + kh;
+          if (r < rows && h >= 0 && h < p.H) {
+            v[i].v = *reinterpret_cast<const uint4*>(in + ((n * p.C + c) * p.H + h) * p.W + l * LV);
+          } else {
+#pragma unroll
+            for (int e = 0; e < LV; ++e) v[i].e[e] = fill;
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          if (r0 + i < rows) {
+            T* d = stage + (r0 + i) * p.pitch + pw + l * LV;
+#pragma unroll
+            for (int e = 0; e < LV; ++e) d[e] = v[i].e[e];
+          }
+        }
       }
+    }
+  } else {
+    for (int r0 = warp * 4; r0 < rows; r0 += nwarps * 4) {
+      for (int x = lane; x < p.Wp; x += 32) {
+        const int w = x - pw;
+        const bool col_ok = w >= 0 && w < W;
+        T v[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
-        if (r0 + i < rows) stage[(r0 + i) * p.pitch + x] = v[i];
+        for (int i = 0; i < 4; ++i) {
+          const int r = r0 + i;
+          const int c = r / Kh, kh = r - c * Kh;
+          const int64_t h = h0 + kh;
+          v[i] = (r < rows && col_ok && h >= 0 && h < p.H) ? in[((n * p.C + c) * p.H + h) * p.W + w] : fill;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (r0 + i < rows) stage[(r0 + i) * p.pitch + x] = v[i];
+      }
     }
   }
   __syncthreads();
@@ -514,6 +552,7 @@ struct Pool3s2 {
   int64_t units;   // planes * strips
 };
 
+template <int R>
 __global__ void __launch_bounds__(256) window_max_3x3s2(const float* __restrict__ in, float* __restrict__ out,
                                                          const Pool3s2 p, float fill) {
   const int64_t u = blockIdx.x * (int64_t)blockDim.y + threadIdx.y;
@@ -522,28 +561,36 @@ __global__ void __launch_bounds__(256) window_max_3x3s2(const float* __restrict_
   const int strip = static_cast<int>(u - plane * p.strips);
   const float* src = in + plane * p.H * p.W;
   float* dst = out + plane * p.Ho * p.Wo;
-  const int y0 = strip * p.R, y1 = min(p.Ho, y0 + p.R);
+  const int y0 = strip * R;
   for (int j = threadIdx.x; j < p.w4; j += blockDim.x) {
-    const int x = 4 * j;
-    auto hmax = [&](int h, float& m0, float& m1) {
-      if (h < 0 || h >= p.H) { m0 = m1 = fill; return; }
-      const float* row = src + (int64_t)h * p.W + x;
-      const float4 v = *reinterpret_cast<const float4*>(row);
-      const float left = j > 0 ? row[-1] : fill;
-      m0 = fmaxf(fmaxf(left, v.x), v.y);
-      m1 = fmaxf(fmaxf(v.y, v.z), v.w);
-    };
-    float c0, c1;
-    hmax(2 * y0 - 1, c0, c1);
-#pragma unroll 2
-    for (int y = y0; y < y1; ++y) {
-      float a0, a1, b0, b1;
-      hmax(2 * y, a0, a1);
-      hmax(2 * y + 1, b0, b1);
-      const float o0 = fmaxf(fmaxf(c0, a0), b0), o1 = fmaxf(fmaxf(c1, a1), b1);
-      if (2 * j + 1 < p.Wo) *reinterpret_cast<float2*>(dst + (int64_t)y * p.Wo + 2 * j) = make_float2(o0, o1);
-      else if (2 * j < p.Wo) dst[(int64_t)y * p.Wo + 2 * j] = o0;
-      c0 = b0; c1 = b1;
+    // all 2R+1 input rows of the strip are requested before the first maximum is taken
+    float4 v[2 * R + 1];
+    float left[2 * R + 1];
+#pragma unroll
+    for (int i = 0; i < 2 * R + 1; ++i) {
+      const int h = 2 * y0 - 1 + i;
+      if (h >= 0 && h < p.H) {
+        const float* row = src + (int64_t)h * p.W + 4 * j;
+        v[i] = *reinterpret_cast<const float4*>(row);
+        left[i] = j > 0 ? row[-1] : fill;
+      } else {
+        v[i] = make_float4(fill, fill, fill, fill);
+        left[i] = fill;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+      const int y = y0 + i;
+      if (y < p.Ho) {
+        float o0 = -INFINITY, o1 = -INFINITY;
+#pragma unroll
+        for (int d = 0; d < 3; ++d) {
+          const float4 w = v[2 * i + d];
+          o0 = fmaxf(o0, fmaxf(fmaxf(left[2 * i + d], w.x), w.y));
+          o1 = fmaxf(o1, fmaxf(fmaxf(w.y, w.z), w.w));
+        }
+        *reinterpret_cast<float2*>(dst + (int64_t)y * p.Wo + 2 * j) = make_float2(o0, o1);
+      }
     }
   }
 }
@@ -763,13 +810,14 @@ int gl_compute_reduce_max(const gl_ap* in, const gl_windows* w, gl_ap* out, void
     Pool3s2 t;
     t.H = (int)in->shape[na]; t.W = (int)in->shape[na + 1];
     t.Ho = (int)A.shape[na]; t.Wo = (int)A.shape[na + 1];
-    t.R = 7;
+    constexpr int kRows = 2;   // short strips: more threads in flight beat the shared odd rows (measured)
+    t.R = kRows;
     t.strips = (t.Ho + t.R - 1) / t.R;
     t.w4 = t.W / 4;
     t.units = prod(in->shape, 0, na) * t.strips;
     const int64_t blocks = (t.units + 7) / 8;
     if (blocks <= 0x7FFFFFFF) {
-      window_max_3x3s2<<<static_cast<unsigned>(blocks), dim3(32, 8), 0, st>>>(src, dst, t, fill);
+      window_max_3x3s2<kRows><<<static_cast<unsigned>(blocks), dim3(32, 8), 0, st>>>(src, dst, t, fill);
       return launch_status();
     }
   }

@@ -116,8 +116,12 @@ class ConvCase:
 
     @property
     def algorithmic_bytes(self):
-        """bf16 activations and weights read once, fp32 result written once."""
-        return 2 * self.n * self.c * self.h * self.w + 2 * self.o * self.kd + 4 * self.m * self.o
+        """bf16 activations (only the rows and columns some window touches) and weights read
+        once, fp32 result written once."""
+        def touched(extent, out, k):
+            return min(extent, out * k if k < self.stride else (out - 1) * self.stride + k)
+        cells = touched(self.h, self.ho, self.kh) * touched(self.w, self.wo, self.kw)
+        return 2 * self.n * self.c * cells + 2 * self.o * self.kd + 4 * self.m * self.o
 
     def inputs(self, seed: int):
         """(activations NCHW, weights OCKhKw) as float32 arrays of bf16 values."""
