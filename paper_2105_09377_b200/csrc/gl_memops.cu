@@ -335,7 +335,7 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
                                                         const Im2colParams p, T fill) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   int* lut = reinterpret_cast<int*>(smem_raw);                     // K entries: staged offset of column k at w'=0
-  T* stage = reinterpret_cast<T*>(smem_raw + ((p.K * 4 + 15) / 16) * 16);   // [C*Kh][pitch]
+  T* stage = reinterpret_cast<T*>(smem_raw + (((p.K + p.C * p.Kh) * 4 + 15) / 16) * 16);   // [C*Kh][pitch]
   const int64_t n = blockIdx.x / p.Ho, ho = blockIdx.x % p.Ho;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
   const int rows = static_cast<int>(p.C * p.Kh), Kw = static_cast<int>(p.Kw), Kh = static_cast<int>(p.Kh);
@@ -345,37 +345,48 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
   // staging: four rows per warp pass so that several global loads are in flight per thread
   constexpr int LV = 16 / sizeof(T);   // elements per 128-bit load
   if (p.W % LV == 0) {
-    // rows are 16-byte multiples: border cells first, then eight rows per warp pass with one
-    // 128-bit load per lane and row, all requested before any is stored
+    // rows are 16-byte multiples.  rowoff[r] = offset of staged row r inside this image, or -1
+    // for a row of border cells; then every thread takes 128-bit pieces of the flattened
+    // (row, piece) space, four loads in flight each.
+    int* rowoff = lut + K;   // the host reserves rows more ints behind the gather table
+    for (int r = threadIdx.x; r < rows; r += blockDim.x) {
+      const int c = r / Kh, kh = r - c * Kh;
+      const int64_t h = h0 + kh;
+      rowoff[r] = (h >= 0 && h < p.H) ? static_cast<int>((c * p.H + h) * p.W) : -1;
+    }
     const int border = p.Wp - W;
     for (int e = threadIdx.x; e < rows * border; e += blockDim.x) {
       const int r = e / border, j = e - r * border;
       stage[r * p.pitch + (j < pw ? j : W + j)] = fill;
     }
-    const int wv = W / LV;
+    __syncthreads();
+    const T* image = in + n * p.C * p.H * p.W;
+    const int wv = W / LV, slots = rows * wv;
     union Vec { uint4 v; T e[LV]; };
-    for (int r0 = warp * 8; r0 < rows; r0 += nwarps * 8) {
-      for (int l = lane; l < wv; l += 32) {
-        Vec v[8];
+    for (int s0 = threadIdx.x; s0 < slots; s0 += 4 * blockDim.x) {
+      Vec v[4];
+      int at[4];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int r = r0 + i;
-          const int c = r / Kh, kh = r - c * Kh;
-          const int64_t h = h0 + kh;
-          if (r < rows && h >= 0 && h < p.H) {
-            v[i].v = *reinterpret_cast<const uint4*>(in + ((n * p.C + c) * p.H + h) * p.W + l * LV);
+      for (int i = 0; i < 4; ++i) {
+        const int sl = s0 + i * blockDim.x;
+        at[i] = -1;
+        if (sl < slots) {
+          const int r = sl / wv, l = sl - r * wv;
+          at[i] = r * p.pitch + pw + l * LV;
+          const int off = rowoff[r];
+          if (off >= 0) {
+            v[i].v = *reinterpret_cast<const uint4*>(image + off + l * LV);
           } else {
 #pragma unroll
             for (int e = 0; e < LV; ++e) v[i].e[e] = fill;
           }
         }
+      }
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          if (r0 + i < rows) {
-            T* d = stage + (r0 + i) * p.pitch + pw + l * LV;
+      for (int i = 0; i < 4; ++i) {
+        if (at[i] >= 0) {
 #pragma unroll
-            for (int e = 0; e < LV; ++e) d[e] = v[i].e[e];
-          }
+          for (int e = 0; e < LV; ++e) stage[at[i] + e] = v[i].e[e];
         }
       }
     }
@@ -690,9 +701,10 @@ int run_windows(const gl_ap* in, const gl_windows* w, const gl_ap& A, gl_ap* out
                           ? best_im2col_pitch(static_cast<int>(wp), static_cast<int>(p.Kw), static_cast<int>(p.K),
                                               vec ? VEC : 1, static_cast<int>(sizeof(T)))
                           : static_cast<int>(wp);
-    const int64_t smem = ((p.K * 4 + 15) / 16) * 16 + p.C * p.Kh * pitch * (int64_t)sizeof(T);
+    const int64_t smem = (((p.K + p.C * p.Kh) * 4 + 15) / 16) * 16 + p.C * p.Kh * pitch * (int64_t)sizeof(T);
     const int64_t blocks = p.N * p.Ho;
-    if (smem <= kIm2colMaxSmem && smem <= device_smem_optin() && blocks <= 0x7FFFFFFF && p.Wo * p.K < (1ll << 30)) {
+    if (smem <= kIm2colMaxSmem && smem <= device_smem_optin() && blocks <= 0x7FFFFFFF && p.Wo * p.K < (1ll << 30) &&
+        p.C * p.H * p.W < (1ll << 31)) {
       p.Wp = static_cast<int>(wp);
       p.pitch = pitch;
       auto kern = vec ? im2col_rows<T, VEC> : im2col_rows<T, 1>;
