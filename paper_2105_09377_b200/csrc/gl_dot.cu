@@ -148,6 +148,48 @@ __global__ void __launch_bounds__(256) weights_to_channels_last(const uint16_t* 
   }
 }
 
+// Few input channels (Kw*Cp <= 64): "row window" layout.  The activations are copied to
+// (N, Hp, Wpa, Cp) with the border cells written out as zeros.  In that copy the Kw*Cp values
+// that one filter row meets at output column w' are contiguous and start Sw*Cp elements after
+// those of w'-1, so a tensor map whose second dimension has that (overlapping) stride delivers,
+// per filter row, a ready K-major tile of 64 values per output column.  The weights go to
+// (O, Kh, 64) with zeros in the unused tail of every 64.
+__global__ void __launch_bounds__(256) rowwin_pack_x(const uint16_t* __restrict__ in, uint16_t* __restrict__ out,
+                                                     int channels_last, int64_t N, int64_t C, int64_t H, int64_t W,
+                                                     int64_t Hp, int64_t Wpa, int Cp, int64_t ph, int64_t pw) {
+  const int64_t pixels = N * Hp * Wpa;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < pixels; e += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t wp = e % Wpa, hp = (e / Wpa) % Hp, n = e / (Wpa * Hp);
+    const int64_t h = hp - ph, w = wp - pw;
+    const bool inside = h >= 0 && h < H && w >= 0 && w < W;
+    for (int c0 = 0; c0 < Cp; c0 += 8) {
+      union { uint4 v; uint16_t e[8]; } px;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int c = c0 + i;
+        uint16_t val = 0;
+        if (inside && c < C) val = channels_last ? in[((n * H + h) * W + w) * C + c] : in[((n * C + c) * H + h) * W + w];
+        px.e[i] = val;
+      }
+      *reinterpret_cast<uint4*>(out + e * Cp + c0) = px.v;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) rowwin_pack_w(const uint16_t* __restrict__ in, uint16_t* __restrict__ out,
+                                                     int channels_last, int64_t O, int64_t C, int64_t Kh, int64_t Kw,
+                                                     int Cp) {
+  const int64_t total = O * Kh * 64;
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+    const int j = static_cast<int>(e % 64);
+    const int64_t kh = (e / 64) % Kh, o = e / (64 * Kh);
+    const int kw = j / Cp, c = j % Cp;
+    uint16_t val = 0;
+    if (kw < Kw && c < C) val = channels_last ? in[((o * Kh + kh) * Kw + kw) * C + c] : in[((o * C + c) * Kh + kh) * Kw + kw];
+    out[e] = val;
+  }
+}
+
 // ------------------------------------------------------------------------
 // tcgen05 / TMA building blocks (inline PTX)
 // ------------------------------------------------------------------------
@@ -289,7 +331,7 @@ constexpr int kBM = 128;
 constexpr int kBK = 64;          // bf16 elements per K block = one 128-byte swizzle row
 constexpr int kTcThreads = 224;  // warp 0 TMA (A), warp 1 MMA + TMEM, warps 2-5 epilogue, warp 6 TMA (B)
 
-enum AMode { kDense = 0, kIm2col = 1, kIm2colGranule = 2 };
+enum AMode { kDense = 0, kIm2col = 1, kIm2colGranule = 2, kRowWin = 3 };
 
 // Division of a 31-bit number by a fixed divisor as multiply-high + shift: the loops below run
 // in single threads, where an integer division is a ~150-cycle dependent chain.
@@ -317,6 +359,9 @@ struct TcParams {
   int Cp, Kh, Kw, Sh, Sw, ph, pw, Ho, Wo;
   int cchunks;            // kIm2col: 64-channel chunks per tap; kIm2colGranule: 8-channel granules per tap
   FastDiv div_tiles_n, div_wo, div_howo;
+  // kRowWin only: one tile = (up to) 128 outputs of one output row
+  int Hp, segs;           // padded input rows per image; 128-wide segments per output row
+  FastDiv div_segs, div_ho;
 };
 
 // A stage holds G K-blocks of 64 (G A sub-tiles, then G B sub-tiles) behind one pair of barriers.
@@ -389,7 +434,15 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
         p.div_tiles_n.divmod(static_cast<uint32_t>(t), tm, tn);
         const int m0 = static_cast<int>(tm) * kBM, n0 = static_cast<int>(tn) * BN;
         int wbase = 0, hbase = 0, img = 0;
-        if (MODE != kDense && load_a) {
+        if (MODE == kRowWin) {
+          if (load_a) {   // tile -> (output row, segment) -> first padded input row
+            uint32_t row, seg, im, ho;
+            p.div_segs.divmod(tm, row, seg);
+            p.div_ho.divmod(row, im, ho);
+            wbase = static_cast<int>(seg) * kBM;
+            hbase = static_cast<int>(im) * p.Hp + static_cast<int>(ho) * p.Sh;
+          }
+        } else if (MODE != kDense && load_a) {
           uint32_t im, rem, ho, wo;
           p.div_howo.divmod(static_cast<uint32_t>(m0), im, rem);
           p.div_wo.divmod(rem, ho, wo);
@@ -412,6 +465,10 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
             const uint32_t sa = stage + j * Cfg::kStageA, sb = stage + G * Cfg::kStageA + j * Cfg::kStageB;
             if (MODE == kDense) {
               if (load_a) tma_load_2d(sa, &map_a, kb * kBK, m0, full);
+              else tma_load_2d(sb, &map_b, kb * kBK, n0, full);
+            } else if (MODE == kRowWin) {
+              // K block kb = filter row kb: 128 output columns x 64 values of padded input row hbase + kb
+              if (load_a) tma_load_3d(sa, &map_a, 0, wbase, hbase + kb, full);
               else tma_load_2d(sb, &map_b, kb * kBK, n0, full);
             } else if (MODE == kIm2col) {
               if (load_a)
@@ -496,7 +553,15 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
       const int tm = static_cast<int>(tmu), tn = static_cast<int>(tnu);
       if (!mbar_wait(bar_tfull + 8 * acc, aph, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      const int64_t m = static_cast<int64_t>(tm) * kBM + q * 32 + lane;
+      int64_t m = static_cast<int64_t>(tm) * kBM + q * 32 + lane;
+      bool m_ok = m < p.M;
+      uint32_t orow = 0, oseg = 0;
+      if (MODE == kRowWin) {
+        p.div_segs.divmod(tmu, orow, oseg);
+        const int wloc = static_cast<int>(oseg) * kBM + q * 32 + lane;
+        m = static_cast<int64_t>(orow) * p.Wo + wloc;
+        m_ok = wloc < p.Wo;
+      }
       float* row = out + m * p.O;
 #pragma unroll 1
       for (int c = 0; c < BN; c += 32) {
@@ -526,14 +591,21 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           __syncwarp();
           if (lane == 0) {
-            asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
-                             reinterpret_cast<uint64_t>(&map_c)),
-                         "r"(static_cast<int>(n0)), "r"(tm * kBM + q * 32), "r"(buf)
-                         : "memory");
+            if (MODE == kRowWin)   // result viewed as (N*Ho, Wo, O): columns past Wo are clipped
+              asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(
+                               reinterpret_cast<uint64_t>(&map_c)),
+                           "r"(static_cast<int>(n0)), "r"(static_cast<int>(oseg) * kBM + q * 32),
+                           "r"(static_cast<int>(orow)), "r"(buf)
+                           : "memory");
+            else
+              asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
+                               reinterpret_cast<uint64_t>(&map_c)),
+                           "r"(static_cast<int>(n0)), "r"(tm * kBM + q * 32), "r"(buf)
+                           : "memory");
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
           }
           ++chunk_it;
-        } else if (m < p.M) {
+        } else if (m_ok) {
           if (vec_ok && n0 + 32 <= p.O) {
 #pragma unroll
             for (int i = 0; i < 32; i += 4)
@@ -664,6 +736,29 @@ bool encode_result(CUtensorMap* m, float* base, int64_t M, int64_t O) {
                             CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// fp32 result of a row-window convolution viewed as (N*Ho, Wo, O): 32x32 boxes inside one output row.
+bool encode_result_rows(CUtensorMap* m, float* base, int64_t rows, int64_t Wo, int64_t O) {
+  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(O), static_cast<cuuint64_t>(Wo), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(O) * 4, static_cast<cuuint64_t>(Wo * O) * 4};
+  const cuuint32_t box[3] = {32, 32, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return driver_api().tiled(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Row-window activations (N*Hp, Wpa, Cp): dimension 1 walks output columns with a stride of
+// Sw*Cp elements, shorter than the 64 elements of dimension 0 (the windows overlap).
+bool encode_rowwin(CUtensorMap* m, const void* base, int64_t rows, int64_t Wo, int64_t Wpa, int64_t Cp, int64_t Sw) {
+  const cuuint64_t dims[3] = {64, static_cast<cuuint64_t>(Wo), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(Sw * Cp) * 2, static_cast<cuuint64_t>(Wpa * Cp) * 2};
+  const cuuint32_t box[3] = {64, kBM, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return driver_api().tiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int BN, int MODE, int G, int OCC>
 int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams p, cudaStream_t st) {
   using Cfg = TcCfg<BN, G, OCC>;
@@ -679,8 +774,13 @@ int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams
   p.div_howo.set(p.Wo > 0 ? static_cast<int64_t>(p.Wo) * p.Ho : 1);
   CUtensorMap mc;
   p.tma_store = (p.O % 4 == 0) ? 1 : 0;
+  if (MODE == kRowWin) {
+    p.div_segs.set(p.segs);
+    p.div_ho.set(p.Ho);
+  }
   if (p.tma_store) {
-    if (!encode_result(&mc, out, p.M, p.O)) return GL_ERR_CUDA;
+    const bool ok = MODE == kRowWin ? encode_result_rows(&mc, out, p.M / p.Wo, p.Wo, p.O) : encode_result(&mc, out, p.M, p.O);
+    if (!ok) return GL_ERR_CUDA;
   } else {
     mc = ma;   // unused by the kernel; any valid map
   }
@@ -719,6 +819,8 @@ struct ConvPlan {
   bool prepass = false;  // needs channels-last copies in the workspace
   int64_t Cp = 0;
   size_t x_bytes = 0, w_bytes = 0;
+  bool rowwin = false;   // few channels: row-window layout (always through the workspace)
+  int64_t Hp = 0, Wpa = 0;
 };
 
 ConvPlan plan_conv(const DotProblem& d) {
@@ -730,6 +832,17 @@ ConvPlan plan_conv(const DotProblem& d) {
                     d.Kh * d.Kw * pl.Cp < (1ll << 31);
   pl.tc = fits;
   pl.prepass = !d.channels_last || pl.Cp != d.C;
+  if (fits && pl.Cp < kBK && d.Kw * pl.Cp <= kBK && d.Wo < (1ll << 24) && d.N * (d.H + d.ph_lo + d.ph_hi) < (1ll << 31)) {
+    pl.rowwin = true;
+    pl.prepass = true;
+    pl.Hp = d.H + d.ph_lo + d.ph_hi;
+    // wide enough for the 64 values behind the last output column; a multiple of Sw (tensor-map stride rule)
+    pl.Wpa = std::max(d.W + d.pw_lo + d.pw_hi, (d.Wo - 1) * d.Sw + kBK / pl.Cp);
+    pl.Wpa = (pl.Wpa + d.Sw - 1) / d.Sw * d.Sw;
+    pl.x_bytes = round_up(static_cast<size_t>(d.N * pl.Hp * pl.Wpa * pl.Cp) * 2, 1024);
+    pl.w_bytes = round_up(static_cast<size_t>(d.O * d.Kh * kBK) * 2, 1024);
+    return pl;
+  }
   if (pl.prepass) {
     pl.x_bytes = round_up(static_cast<size_t>(d.N * d.H * d.W * pl.Cp) * 2, 1024);
     pl.w_bytes = round_up(static_cast<size_t>(d.O * d.Kh * d.Kw * pl.Cp) * 2, 1024);
@@ -842,6 +955,27 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u)) return GL_ERR_WORKSPACE;
     uint16_t* xs = static_cast<uint16_t*>(workspace);
     uint16_t* ws = reinterpret_cast<uint16_t*>(static_cast<unsigned char*>(workspace) + pl.x_bytes);
+    if (pl.rowwin) {
+      const int64_t pixels = d.N * pl.Hp * pl.Wpa;
+      rowwin_pack_x<<<static_cast<unsigned>(std::min<int64_t>((pixels + 255) / 256, 1 << 20)), 256, 0, st>>>(
+          pa, xs, d.channels_last ? 1 : 0, d.N, d.C, d.H, d.W, pl.Hp, pl.Wpa, static_cast<int>(pl.Cp), d.ph_lo, d.pw_lo);
+      rowwin_pack_w<<<static_cast<unsigned>(std::min<int64_t>((d.O * d.Kh * 64 + 255) / 256, 1 << 20)), 256, 0, st>>>(
+          pb, ws, d.channels_last ? 1 : 0, d.O, d.C, d.Kh, d.Kw, static_cast<int>(pl.Cp));
+      if (cudaGetLastError() != cudaSuccess) return GL_ERR_CUDA;
+      p.K = d.Kh * kBK;
+      p.kblocks = static_cast<int>(d.Kh);
+      p.Cp = static_cast<int>(pl.Cp);
+      p.Kh = static_cast<int>(d.Kh); p.Kw = static_cast<int>(d.Kw);
+      p.Sh = static_cast<int>(d.Sh); p.Sw = static_cast<int>(d.Sw);
+      p.Ho = static_cast<int>(d.Ho); p.Wo = static_cast<int>(d.Wo);
+      p.Hp = static_cast<int>(pl.Hp);
+      p.segs = static_cast<int>((d.Wo + kBM - 1) / kBM);
+      p.tiles_m = static_cast<int>(d.N * d.Ho * p.segs);
+      if (encode_rowwin(&ma, xs, d.N * pl.Hp, d.Wo, pl.Wpa, pl.Cp, d.Sw) &&
+          encode_kmajor_sw128(&mb, ws, d.O, p.K, bn))
+        return launch_tc_bn<kRowWin>(bn, ma, mb, dst, p, st);
+      return GL_ERR_CUDA;
+    }
     const int64_t HW = d.H * d.W, T = d.Kh * d.Kw;
     if (d.channels_last) {
       // (N,H,W,C) with C not a multiple of 8: re-pitch the channel dim (a (N*HW, C) -> (N*HW, Cp) copy)
