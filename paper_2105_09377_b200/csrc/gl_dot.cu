@@ -148,6 +148,26 @@ __global__ void __launch_bounds__(256) weights_to_channels_last(const uint16_t* 
   }
 }
 
+// Same permutation for (C,Kh,Kw) filters, staged: a block reads 64 channels x T taps of one
+// filter as one contiguous run, and writes T runs of 64 channels.
+__global__ void __launch_bounds__(256) weights_to_channels_last_staged(const uint16_t* __restrict__ in,
+                                                                       uint16_t* __restrict__ out, int C, int T,
+                                                                       int Cp) {
+  extern __shared__ uint16_t wstage[];   // [64][T]
+  const int64_t o = blockIdx.y;
+  const int c0 = blockIdx.x * 64;
+  const int nc = min(64, C - c0);        // channels with data (may be <= 0 in the padded tail)
+  const uint16_t* src = in + (o * C + c0) * T;
+  for (int e = threadIdx.x; e < nc * T; e += blockDim.x) wstage[e] = src[e];
+  __syncthreads();
+  const int ncp = min(64, Cp - c0);
+  uint16_t* dst = out + o * T * Cp + c0;
+  for (int e = threadIdx.x; e < T * 64; e += blockDim.x) {
+    const int t = e >> 6, c = e & 63;
+    if (c < ncp) dst[static_cast<int64_t>(t) * Cp + c] = c < nc ? wstage[c * T + t] : (uint16_t)0;
+  }
+}
+
 // Few input channels (Kw*Cp <= 64): "row window" layout.  The activations are copied to
 // (N, Hp, Wpa, Cp) with the border cells written out as zeros.  In that copy the Kw*Cp values
 // that one filter row meets at output column w' are contiguous and start Sw*Cp elements after
@@ -155,23 +175,29 @@ __global__ void __launch_bounds__(256) weights_to_channels_last(const uint16_t* 
 // per filter row, a ready K-major tile of 64 values per output column.  The weights go to
 // (O, Kh, 64) with zeros in the unused tail of every 64.
 __global__ void __launch_bounds__(256) rowwin_pack_x(const uint16_t* __restrict__ in, uint16_t* __restrict__ out,
-                                                     int channels_last, int64_t N, int64_t C, int64_t H, int64_t W,
-                                                     int64_t Hp, int64_t Wpa, int Cp, int64_t ph, int64_t pw) {
-  const int64_t pixels = N * Hp * Wpa;
-  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < pixels; e += (int64_t)gridDim.x * blockDim.x) {
-    const int64_t wp = e % Wpa, hp = (e / Wpa) % Hp, n = e / (Wpa * Hp);
-    const int64_t h = hp - ph, w = wp - pw;
-    const bool inside = h >= 0 && h < H && w >= 0 && w < W;
+                                                     int channels_last, int C, int H, int W, int Hp, int Wpa, int Cp,
+                                                     int ph, int pw) {
+  // one block per padded row (n, hp); threads walk the row's pixels
+  const int64_t rowid = blockIdx.x;
+  const int hp = static_cast<int>(rowid % Hp);
+  const int64_t n = rowid / Hp;
+  const int h = hp - ph;
+  const bool row_ok = h >= 0 && h < H;
+  uint16_t* orow = out + rowid * Wpa * Cp;
+  for (int wp = threadIdx.x; wp < Wpa; wp += blockDim.x) {
+    const int w = wp - pw;
+    const bool inside = row_ok && w >= 0 && w < W;
     for (int c0 = 0; c0 < Cp; c0 += 8) {
       union { uint4 v; uint16_t e[8]; } px;
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const int c = c0 + i;
         uint16_t val = 0;
-        if (inside && c < C) val = channels_last ? in[((n * H + h) * W + w) * C + c] : in[((n * C + c) * H + h) * W + w];
+        if (inside && c < C)
+          val = channels_last ? in[((n * H + h) * W + w) * C + c] : in[((n * C + c) * H + h) * static_cast<int64_t>(W) + w];
         px.e[i] = val;
       }
-      *reinterpret_cast<uint4*>(out + e * Cp + c0) = px.v;
+      *reinterpret_cast<uint4*>(orow + static_cast<int64_t>(wp) * Cp + c0) = px.v;
     }
   }
 }
@@ -956,9 +982,10 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     uint16_t* xs = static_cast<uint16_t*>(workspace);
     uint16_t* ws = reinterpret_cast<uint16_t*>(static_cast<unsigned char*>(workspace) + pl.x_bytes);
     if (pl.rowwin) {
-      const int64_t pixels = d.N * pl.Hp * pl.Wpa;
-      rowwin_pack_x<<<static_cast<unsigned>(std::min<int64_t>((pixels + 255) / 256, 1 << 20)), 256, 0, st>>>(
-          pa, xs, d.channels_last ? 1 : 0, d.N, d.C, d.H, d.W, pl.Hp, pl.Wpa, static_cast<int>(pl.Cp), d.ph_lo, d.pw_lo);
+      rowwin_pack_x<<<static_cast<unsigned>(d.N * pl.Hp), 256, 0, st>>>(
+          pa, xs, d.channels_last ? 1 : 0, static_cast<int>(d.C), static_cast<int>(d.H), static_cast<int>(d.W),
+          static_cast<int>(pl.Hp), static_cast<int>(pl.Wpa), static_cast<int>(pl.Cp), static_cast<int>(d.ph_lo),
+          static_cast<int>(d.pw_lo));
       rowwin_pack_w<<<static_cast<unsigned>(std::min<int64_t>((d.O * d.Kh * 64 + 255) / 256, 1 << 20)), 256, 0, st>>>(
           pb, ws, d.channels_last ? 1 : 0, d.O, d.C, d.Kh, d.Kw, static_cast<int>(pl.Cp));
       if (cudaGetLastError() != cudaSuccess) return GL_ERR_CUDA;
@@ -1003,8 +1030,14 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
                         static_cast<unsigned>(d.N));
         nchw_to_nhwc_pad<<<grid, 256, 0, st>>>(pa, xs, d.C, HW, pl.Cp);
       }
-      weights_to_channels_last<<<static_cast<unsigned>(std::min<int64_t>((d.O * T * pl.Cp + 255) / 256, 1 << 20)), 256, 0,
-                                 st>>>(pb, ws, d.O, d.C, T, pl.Cp);
+      if (T <= 256 && d.O <= 65535 && d.C < (1ll << 30)) {
+        const dim3 grid(static_cast<unsigned>((pl.Cp + 63) / 64), static_cast<unsigned>(d.O));
+        weights_to_channels_last_staged<<<grid, 256, static_cast<size_t>(64 * T * 2), st>>>(
+            pb, ws, static_cast<int>(d.C), static_cast<int>(T), static_cast<int>(pl.Cp));
+      } else {
+        weights_to_channels_last<<<static_cast<unsigned>(std::min<int64_t>((d.O * T * pl.Cp + 255) / 256, 1 << 20)), 256,
+                                   0, st>>>(pb, ws, d.O, d.C, T, pl.Cp);
+      }
     }
     if (cudaGetLastError() != cudaSuccess) return GL_ERR_CUDA;
     x = xs;
