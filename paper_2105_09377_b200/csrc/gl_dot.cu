@@ -385,6 +385,11 @@ struct TcParams {
   int Cp, Kh, Kw, Sh, Sw, ph, pw, Ho, Wo;
   int cchunks;            // kIm2col: 64-channel chunks per tap; kIm2colGranule: 8-channel granules per tap
   FastDiv div_tiles_n, div_wo, div_howo;
+  // K split (Section 5.4: a split of the contracted dimension turns dotProd into reduceSum over
+  // partial dotProds): unit u = tile u / ksplit, K blocks [s*kper, (s+1)*kper), s = u % ksplit.
+  // With ksplit > 1 the kernel writes partial [s][M][O] planes and a second kernel adds them up.
+  int ksplit, kper;
+  FastDiv div_ksplit;
   // kRowWin only: one tile = (up to) 128 outputs of one output row
   int Hp, segs;           // padded input rows per image; 128-wide segments per output row
   FastDiv div_segs, div_ho;
@@ -445,7 +450,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int num_tiles = p.tiles_m * p.tiles_n;
+  const int num_tiles = p.tiles_m * p.tiles_n * p.ksplit;   // work units
 
   if (warp == 0 || warp == 6) {
     // ---------------- TMA producers: warp 0 stages A, warp 6 stages B ----------------
@@ -455,9 +460,11 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
       asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(load_a ? &map_a : &map_b)) : "memory");
       uint32_t it = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-        uint32_t tm, tn;
-        p.div_tiles_n.divmod(static_cast<uint32_t>(t), tm, tn);
+      for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x) {
+        uint32_t t, ks, tm, tn;
+        p.div_ksplit.divmod(static_cast<uint32_t>(u), t, ks);
+        p.div_tiles_n.divmod(t, tm, tn);
+        const int kb_begin = static_cast<int>(ks) * p.kper, kb_end = min(p.kblocks, kb_begin + p.kper);
         const int m0 = static_cast<int>(tm) * kBM, n0 = static_cast<int>(tn) * BN;
         int wbase = 0, hbase = 0, img = 0;
         if (MODE == kRowWin) {
@@ -478,12 +485,18 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
         }
         // filter position of the next K block, advanced without divisions
         int cc = 0, kw = 0, kh = 0;
-        for (int kb0 = 0; kb0 < p.kblocks; kb0 += G, ++it) {
+        if (MODE == kIm2col && kb_begin > 0) {
+          const int tap = kb_begin / p.cchunks;
+          cc = kb_begin - tap * p.cchunks;
+          kh = tap / p.Kw;
+          kw = tap - kh * p.Kw;
+        }
+        for (int kb0 = kb_begin; kb0 < kb_end; kb0 += G, ++it) {
           const uint32_t s = it % Cfg::kStages, ph = (it / Cfg::kStages) & 1u;
           if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t full = bar_full + 8 * s;
           const uint32_t stage = tiles + s * Cfg::kStage;
-          const int nsub = min(G, p.kblocks - kb0);
+          const int nsub = min(G, kb_end - kb0);
           mbar_expect_tx(full, nsub * (load_a ? Cfg::kStageA : Cfg::kStageB));
 #pragma unroll 1
           for (int j = 0; j < nsub; ++j) {
@@ -532,19 +545,22 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
                                                         : make_desc(tiles + G * Cfg::kStageA, 16, 1024, 2);
       uint32_t it = 0, tile_it = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_it) {
+      for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x, ++tile_it) {
         const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
+        uint32_t t, ks;
+        p.div_ksplit.divmod(static_cast<uint32_t>(u), t, ks);
+        const int kb_begin = static_cast<int>(ks) * p.kper, kb_end = min(p.kblocks, kb_begin + p.kper);
         if (!mbar_wait(bar_tempty + 8 * acc, aph ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int kb0 = 0; kb0 < p.kblocks; kb0 += G, ++it) {
+        for (int kb0 = kb_begin; kb0 < kb_end; kb0 += G, ++it) {
           const uint32_t s = it % Cfg::kStages, ph = (it / Cfg::kStages) & 1u;
           if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
           // descriptors differ only in their start-address field (16-byte units): add offsets to a base
           const uint64_t da0 = desc_a0 + ((s * Cfg::kStage) >> 4);
           const uint64_t db0 = desc_b0 + ((s * Cfg::kStage) >> 4);
-          const int nsub = min(G, p.kblocks - kb0);
+          const int nsub = min(G, kb_end - kb0);
 #pragma unroll
           for (int j = 0; j < G; ++j) {
             if (j < nsub) {
@@ -553,7 +569,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
                 constexpr int kStepA = (MODE == kIm2colGranule) ? 2 * (kBM * 16) : 32;
                 constexpr int kStepB = (MODE == kIm2colGranule) ? 2 * (BN * 16) : 32;
                 tc_mma_bf16(d_tmem, da0 + ((j * Cfg::kStageA + k * kStepA) >> 4),
-                            db0 + ((j * Cfg::kStageB + k * kStepB) >> 4), idesc, (kb0 | j | k) != 0 ? 1u : 0u);
+                            db0 + ((j * Cfg::kStageB + k * kStepB) >> 4), idesc, ((kb0 - kb_begin) | j | k) != 0 ? 1u : 0u);
               }
             }
           }
@@ -572,10 +588,11 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
     const bool vec_ok = (p.O & 3) == 0;
     const uint32_t stage_buf = epi_base + q * (Cfg::kEpiBufs * 4096);   // this warp's 32 rows x 128 bytes tiles
     if (p.tma_store && lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_c)) : "memory");
-    for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_it) {
+    for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x, ++tile_it) {
       const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
-      uint32_t tmu, tnu;
-      p.div_tiles_n.divmod(static_cast<uint32_t>(t), tmu, tnu);
+      uint32_t t, ks, tmu, tnu;
+      p.div_ksplit.divmod(static_cast<uint32_t>(u), t, ks);
+      p.div_tiles_n.divmod(t, tmu, tnu);
       const int tm = static_cast<int>(tmu), tn = static_cast<int>(tnu);
       if (!mbar_wait(bar_tfull + 8 * acc, aph, abort_flag)) { ok = false; break; }
       tc_fence_after();
@@ -588,7 +605,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
         m = static_cast<int64_t>(orow) * p.Wo + wloc;
         m_ok = wloc < p.Wo;
       }
-      float* row = out + m * p.O;
+      float* row = out + (static_cast<int64_t>(ks) * p.M + m) * p.O;   // partial plane ks (0 without a K split)
 #pragma unroll 1
       for (int c = 0; c < BN; c += 32) {
         const int64_t n0 = static_cast<int64_t>(tn) * BN + c;
@@ -623,10 +640,10 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
                            "r"(static_cast<int>(n0)), "r"(static_cast<int>(oseg) * kBM + q * 32),
                            "r"(static_cast<int>(orow)), "r"(buf)
                            : "memory");
-            else
-              asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
+            else   // (planes, M, O): plane = K-split index, 0 without a split
+              asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(
                                reinterpret_cast<uint64_t>(&map_c)),
-                           "r"(static_cast<int>(n0)), "r"(tm * kBM + q * 32), "r"(buf)
+                           "r"(static_cast<int>(n0)), "r"(tm * kBM + q * 32), "r"(static_cast<int>(ks)), "r"(buf)
                            : "memory");
             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
           }
@@ -751,13 +768,13 @@ bool encode_im2col(CUtensorMap* m, const void* base, const DotProblem& d, int64_
                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// fp32 result [M, O]: 32x32 boxes, 128-byte swizzle (what the epilogue stages).
-bool encode_result(CUtensorMap* m, float* base, int64_t M, int64_t O) {
-  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(O), static_cast<cuuint64_t>(M)};
-  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(O) * 4};
-  const cuuint32_t box[2] = {32, 32};
-  const cuuint32_t estr[2] = {1, 1};
-  return driver_api().tiled(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr,
+// fp32 result planes [planes, M, O]: 32x32 boxes, 128-byte swizzle (what the epilogue stages).
+bool encode_result(CUtensorMap* m, float* base, int64_t M, int64_t O, int64_t planes) {
+  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(O), static_cast<cuuint64_t>(M), static_cast<cuuint64_t>(planes)};
+  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(O) * 4, static_cast<cuuint64_t>(M * O) * 4};
+  const cuuint32_t box[3] = {32, 32, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return driver_api().tiled(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr,
                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                             CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -795,6 +812,8 @@ int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams
       return GL_ERR_CUDA;
     attr_set = true;
   }
+  if (p.ksplit < 1) { p.ksplit = 1; p.kper = p.kblocks; }
+  p.div_ksplit.set(p.ksplit);
   p.div_tiles_n.set(p.tiles_n);
   p.div_wo.set(p.Wo > 0 ? p.Wo : 1);
   p.div_howo.set(p.Wo > 0 ? static_cast<int64_t>(p.Wo) * p.Ho : 1);
@@ -805,12 +824,12 @@ int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams
     p.div_ho.set(p.Ho);
   }
   if (p.tma_store) {
-    const bool ok = MODE == kRowWin ? encode_result_rows(&mc, out, p.M / p.Wo, p.Wo, p.O) : encode_result(&mc, out, p.M, p.O);
+    const bool ok = MODE == kRowWin ? encode_result_rows(&mc, out, p.M / p.Wo, p.Wo, p.O) : encode_result(&mc, out, p.M, p.O, p.ksplit);
     if (!ok) return GL_ERR_CUDA;
   } else {
     mc = ma;   // unused by the kernel; any valid map
   }
-  const int tiles = p.tiles_m * p.tiles_n;
+  const int tiles = p.tiles_m * p.tiles_n * p.ksplit;
   const int grid = tiles < OCC * num_sms() ? tiles : OCC * num_sms();
   dot_tc<BN, MODE, G, OCC><<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(ma, mb, mc, out, p);
   return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;
@@ -838,6 +857,45 @@ int pick_bn(int64_t M, int64_t O) {
   const int sms = num_sms();
   if (O > 128 && tiles_m * ((O + 255) / 256) >= sms) return 256;
   return O > 64 ? 128 : 64;
+}
+
+// compute reduceSum over the K-split partial planes (Section 5.4, last blocking rewrite), planes
+// added in index order so that the result does not depend on scheduling; relu applied last.
+__global__ void __launch_bounds__(256) splitk_reduce(const float* __restrict__ part, float* __restrict__ out,
+                                                     int64_t n, int planes, int relu) {
+  const int64_t n4 = n >> 2;
+  const float4* p4 = reinterpret_cast<const float4*>(part);
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+    float4 acc = p4[i];
+    for (int s = 1; s < planes; ++s) {
+      const float4 v = p4[(s * n >> 2) + i];
+      acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+    }
+    if (relu) { acc.x = fmaxf(acc.x, 0.f); acc.y = fmaxf(acc.y, 0.f); acc.z = fmaxf(acc.z, 0.f); acc.w = fmaxf(acc.w, 0.f); }
+    reinterpret_cast<float4*>(out)[i] = acc;
+  }
+}
+
+// Tile width and K split for a [M,O] result with `kblocks` K blocks.  A problem with fewer tiles
+// than a quarter of the SMs is split along K so that every SM gets a unit of at least four K blocks.
+struct TilePlan { int bn = 64; int ksplit = 1; int kper = 0; size_t partial_bytes = 0; };
+
+TilePlan plan_tiles(int64_t M, int64_t O, int64_t kblocks, bool may_split) {
+  TilePlan tp;
+  tp.bn = pick_bn(M, O);
+  tp.kper = static_cast<int>(kblocks);
+  if (!may_split || (M * O) % 4 != 0 || O % 4 != 0) return tp;
+  const int wide = O > 128 ? 256 : (O > 64 ? 128 : 64);
+  const int64_t tiles = ((M + kBM - 1) / kBM) * ((O + wide - 1) / wide);
+  const int sms = num_sms();
+  if (4 * tiles > sms) return tp;   // measured: a 2-3 way split costs more in the second pass than it gains
+  int split = static_cast<int>(std::min<int64_t>(sms / tiles, kblocks / 4));
+  if (split < 2) return tp;
+  tp.bn = wide;
+  tp.kper = static_cast<int>((kblocks + split - 1) / split);
+  tp.ksplit = static_cast<int>((kblocks + tp.kper - 1) / tp.kper);
+  tp.partial_bytes = round_up(static_cast<size_t>(tp.ksplit) * M * O * 4, 1024);
+  return tp;
 }
 
 struct ConvPlan {
@@ -915,9 +973,17 @@ extern "C" {
 size_t gl_cartesian_dot_workspace(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, uint32_t flags) {
   DotProblem d;
   if (classify_dot(a0, w, a1, &d) != GL_OK) return 0;
-  if ((flags & GL_DOT_GENERAL_KERNEL) || !d.conv) return 0;
+  if (flags & GL_DOT_GENERAL_KERNEL) return 0;
+  if (!d.conv) {
+    if (!dense_tc_ok(d)) return 0;
+    return plan_tiles(d.M, d.O, (d.K + kBK - 1) / kBK, true).partial_bytes;
+  }
   const ConvPlan pl = plan_conv(d);
-  return pl.tc && pl.prepass ? pl.x_bytes + pl.w_bytes : 0;
+  if (!pl.tc) return 0;
+  size_t need = pl.prepass ? pl.x_bytes + pl.w_bytes : 0;
+  if (!pl.rowwin && pl.Cp >= kBK)
+    need += plan_tiles(d.M, d.O, d.Kh * d.Kw * ((pl.Cp + kBK - 1) / kBK), true).partial_bytes;
+  return need;
 }
 
 int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_ap* out, uint32_t flags,
@@ -962,7 +1028,30 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
   TcParams p;
   std::memset(&p, 0, sizeof(p));
   p.M = d.M; p.O = d.O; p.relu = relu;
-  const int bn = pick_bn(d.M, d.O);
+  // tile width and K split; a K split needs room for its partial planes behind the layout copies
+  const size_t pre_bytes = (d.conv && pl.prepass) ? pl.x_bytes + pl.w_bytes : 0;
+  const bool split_mode = !d.conv || (!pl.rowwin && pl.Cp >= kBK);
+  const int64_t kblocks_all = !d.conv ? (d.K + kBK - 1) / kBK : d.Kh * d.Kw * ((pl.Cp + kBK - 1) / kBK);
+  TilePlan tp = plan_tiles(d.M, d.O, kblocks_all, split_mode);
+  if (tp.ksplit > 1 && (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023u) ||
+                        workspace_bytes < pre_bytes + tp.partial_bytes))
+    tp = plan_tiles(d.M, d.O, kblocks_all, false);
+  const int bn = tp.bn;
+  p.ksplit = tp.ksplit;
+  p.kper = tp.kper;
+  float* const final_dst = dst;
+  if (tp.ksplit > 1) {
+    dst = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + pre_bytes);
+    p.relu = 0;
+  }
+  // the launch of the partial-sum kernel when the contraction was split
+  auto finish = [&](int rc_launch) -> int {
+    if (rc_launch != GL_OK || tp.ksplit == 1) return rc_launch;
+    const int64_t n = d.M * d.O;
+    splitk_reduce<<<static_cast<unsigned>(std::min<int64_t>((n / 4 + 255) / 256, 148 * 8)), 256, 0, st>>>(
+        dst, final_dst, n, tp.ksplit, relu);
+    return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+  };
   p.tiles_m = static_cast<int>((d.M + kBM - 1) / kBM);
   p.tiles_n = static_cast<int>((d.O + bn - 1) / bn);
   CUtensorMap ma, mb;
@@ -971,7 +1060,7 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     p.K = d.K;
     p.kblocks = static_cast<int>((d.K + kBK - 1) / kBK);
     if (!encode_kmajor_sw128(&ma, pa, d.M, d.K, kBM) || !encode_kmajor_sw128(&mb, pb, d.O, d.K, bn)) return GL_ERR_CUDA;
-    return launch_tc_bn<kDense>(bn, ma, mb, dst, p, st);
+    return finish(launch_tc_bn<kDense>(bn, ma, mb, dst, p, st));
   }
 
   const uint16_t* x = pa;
@@ -1054,7 +1143,7 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     p.cchunks = static_cast<int>((Cp + kBK - 1) / kBK);
     p.kblocks = static_cast<int>(taps) * p.cchunks;
     if (!encode_im2col(&ma, x, d, Cp, kBK, true) || !encode_kmajor_sw128(&mb, wt, d.O, p.K, bn)) return GL_ERR_CUDA;
-    return launch_tc_bn<kIm2col>(bn, ma, mb, dst, p, st);
+    return finish(launch_tc_bn<kIm2col>(bn, ma, mb, dst, p, st));
   }
   p.cchunks = static_cast<int>(Cp / 8);
   p.kblocks = static_cast<int>((taps * p.cchunks + 7) / 8);
