@@ -86,6 +86,8 @@ typedef struct {
 
 /* Flags of gl_cartesian_dot */
 #define GL_EPILOGUE_RELU 0x2u       /* apply compute relu to every result before it is stored  */
+#define GL_OUT_NCHW 0x4u             /* conv2d only: store transpose(squeeze(...)) of Fig. 2a, i.e.
+                                        ((N, O, H', W'),()); see gl_shape_cartesian_dot_nchw      */
 #define GL_DOT_GENERAL_KERNEL 0x100u /* skip the tensor-core path: run the general kernel, which
                                         takes any shape and sums each window in index order      */
 
@@ -117,6 +119,13 @@ GL_API int gl_shape_pad(const gl_ap* in, int32_t dim, int64_t lo, int64_t hi, gl
  * dotProd, Fig. 2a/2b): with A = windows(a0) (or a0 itself when w is NULL) of shape
  * ((m..),(k..)) and a1 of shape ((o..),(k..)), the result is ((m.., o..),()), GL_F32. */
 GL_API int gl_shape_cartesian_dot(const gl_ap* a0, const gl_windows* w_or_null, const gl_ap* a1, gl_ap* out);
+
+/* The whole conv2d of Fig. 2a: transpose (squeeze (compute dotProd (cartProd (windows a0) a1)) 1)
+ * (0 3 1 2).  a0 must be ((n..),(C,H,W)) with window (C,Kh,Kw), or ((n..),(H,W,C)) with window
+ * (Kh,Kw,C); the result is ((n.., o.., H', W'),()), GL_F32: the window-position dims move behind
+ * the filter dims and the size-1 channel position is squeezed away.  This is the shape
+ * gl_cartesian_dot expects for `out` when GL_OUT_NCHW is set. */
+GL_API int gl_shape_cartesian_dot_nchw(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_ap* out);
 
 /* compute reduceMax (windows? in) (operator table; Fig. 2c): ((access dims of A),()). */
 GL_API int gl_shape_reduce_max(const gl_ap* in, const gl_windows* w_or_null, gl_ap* out);

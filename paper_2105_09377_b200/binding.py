@@ -18,6 +18,7 @@ GL_BF16, GL_F32 = 1, 2
 GL_PAD_ZERO, GL_PAD_NEG_INF = 0, 1
 GL_EPILOGUE_RELU = 0x2
 GL_DOT_GENERAL_KERNEL = 0x100
+GL_OUT_NCHW = 0x4
 GL_OK = 0
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -51,7 +52,7 @@ EXPORTS = [
     "gl_shape_cartesian_dot", "gl_shape_reduce_max", "gl_access_windows", "gl_access_flatten",
     "gl_access_transpose", "gl_access_pad", "gl_cartesian_dot", "gl_cartesian_dot_workspace",
     "gl_compute_reduce_max", "gl_compute_relu", "gl_poll_device_status", "gl_strerror", "gl_version",
-    "gl_cartesian_dot_static",
+    "gl_cartesian_dot_static", "gl_shape_cartesian_dot_nchw",
 ]
 
 
@@ -70,6 +71,7 @@ def _load() -> ctypes.CDLL:
         "gl_shape_transpose": [ap, i32p, ap],
         "gl_shape_pad": [ap, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, ap],
         "gl_shape_cartesian_dot": [ap, win, ap, ap],
+        "gl_shape_cartesian_dot_nchw": [ap, win, ap, ap],
         "gl_shape_reduce_max": [ap, win, ap],
         "gl_access_windows": [ap, win, ap, vp],
         "gl_access_flatten": [ap, ap],
@@ -225,6 +227,14 @@ def gl_shape_cartesian_dot(shape0, access0, w: Optional[GlWindows], shape1, acce
     return _shape_result(out)
 
 
+def gl_shape_cartesian_dot_nchw(shape0, access0, w: GlWindows, shape1, access1):
+    out = GlAp()
+    _check(LIB.gl_shape_cartesian_dot_nchw(ctypes.byref(_meta(shape0, access0, GL_BF16)), ctypes.byref(w),
+                                           ctypes.byref(_meta(shape1, access1, GL_BF16)), ctypes.byref(out)),
+           "gl_shape_cartesian_dot_nchw")
+    return _shape_result(out)
+
+
 def gl_shape_reduce_max(shape, access_ndim, w: Optional[GlWindows]):
     out = GlAp()
     _check(LIB.gl_shape_reduce_max(ctypes.byref(_meta(shape, access_ndim, GL_F32)), _wptr(w), ctypes.byref(out)),
@@ -286,8 +296,12 @@ def gl_cartesian_dot(a0: AccessPattern, w: Optional[GlWindows], a1: AccessPatter
     s0, s1 = _struct(a0), _struct(a1)
     if out is None:
         m = GlAp()
-        _check(LIB.gl_shape_cartesian_dot(ctypes.byref(s0), _wptr(w), ctypes.byref(s1), ctypes.byref(m)),
-               "gl_shape_cartesian_dot")
+        if flags & GL_OUT_NCHW:
+            _check(LIB.gl_shape_cartesian_dot_nchw(ctypes.byref(s0), _wptr(w), ctypes.byref(s1), ctypes.byref(m)),
+                   "gl_shape_cartesian_dot_nchw")
+        else:
+            _check(LIB.gl_shape_cartesian_dot(ctypes.byref(s0), _wptr(w), ctypes.byref(s1), ctypes.byref(m)),
+                   "gl_shape_cartesian_dot")
         out = _alloc(m, a0.tensor.device)
     if workspace is None:
         need = int(LIB.gl_cartesian_dot_workspace(ctypes.byref(s0), _wptr(w), ctypes.byref(s1), flags))

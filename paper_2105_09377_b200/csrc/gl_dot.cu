@@ -43,6 +43,9 @@ struct GenA {            // how to fetch A[m,k]
   int64_t in_size[GL_MAX_DIMS], in_stride[GL_MAX_DIMS], out_ext[GL_MAX_DIMS];
   int64_t w[GL_MAX_DIMS], s[GL_MAX_DIMS], pad_lo[GL_MAX_DIMS];
   int64_t item;
+  // result layout: [M,O], or (image, O, H'W') when the squeeze + transpose of Fig. 2a is fused
+  int out_nchw;
+  int64_t HoWo;
 };
 
 __device__ __forceinline__ float bf16_to_f32(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }
@@ -107,7 +110,8 @@ __global__ void __launch_bounds__(256) dot_general(const uint16_t* __restrict__ 
       if (m < g.M && o < g.O) {
         float v = acc[i][j];
         if (relu) v = v > 0.f ? v : 0.f;
-        out[m * g.O + o] = v;
+        if (g.out_nchw) out[((m / g.HoWo) * g.O + o) * g.HoWo + m % g.HoWo] = v;
+        else out[m * g.O + o] = v;
       }
     }
 }
@@ -380,6 +384,7 @@ struct TcParams {
   int64_t M, O, K;        // K as laid out in B (for conv: Kh*Kw*Cp)
   int tiles_m, tiles_n, kblocks;
   int relu;
+  int out_nchw;           // store (image, O, H'W') instead of [M,O]: squeeze + transpose (0 3 1 2) of Fig. 2a
   int tma_store;          // result rows are 16-byte multiples: the epilogue may use TMA stores
   // conv only
   int Cp, Kh, Kw, Sh, Sw, ph, pw, Ho, Wo;
@@ -606,6 +611,12 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
         m_ok = wloc < p.Wo;
       }
       float* row = out + (static_cast<int64_t>(ks) * p.M + m) * p.O;   // partial plane ks (0 without a K split)
+      float* col = out;      // out_nchw: &out[image][0][pixel]; channel o then lies o*H'W' further
+      if (p.out_nchw && m_ok) {
+        uint32_t img_o, pix_o;
+        p.div_howo.divmod(static_cast<uint32_t>(m), img_o, pix_o);
+        col = out + static_cast<int64_t>(img_o) * p.O * p.div_howo.d + pix_o;
+      }
 #pragma unroll 1
       for (int c = 0; c < BN; c += 32) {
         const int64_t n0 = static_cast<int64_t>(tn) * BN + c;
@@ -616,7 +627,15 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
 #pragma unroll
           for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(fmaxf(__uint_as_float(r[i]), 0.f));
         }
-        if (p.tma_store) {
+        if (p.out_nchw) {
+          // lanes hold consecutive pixels: for every channel the warp writes one contiguous run
+          if (m_ok) {
+            const int64_t plane = p.div_howo.d;
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (n0 + i < p.O) col[(n0 + i) * plane] = __uint_as_float(r[i]);
+          }
+        } else if (p.tma_store) {
           // 32x32 fp32 block: each lane parks its row in shared memory (16-byte pieces XOR-swizzled by
           // row, the 128-byte swizzle of the tensor map), then one lane hands the block to the TMA unit,
           // which writes whole 128-byte rows and clips at the matrix edge.
@@ -818,7 +837,7 @@ int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams
   p.div_wo.set(p.Wo > 0 ? p.Wo : 1);
   p.div_howo.set(p.Wo > 0 ? static_cast<int64_t>(p.Wo) * p.Ho : 1);
   CUtensorMap mc;
-  p.tma_store = (p.O % 4 == 0) ? 1 : 0;
+  p.tma_store = (p.O % 4 == 0 && !p.out_nchw) ? 1 : 0;
   if (MODE == kRowWin) {
     p.div_segs.set(p.segs);
     p.div_ho.set(p.Ho);
@@ -941,6 +960,7 @@ bool dense_tc_ok(const DotProblem& d) {
 void fill_general(const gl_ap* a0, const gl_windows* w, const DotProblem& d, GenA* g) {
   std::memset(g, 0, sizeof(*g));
   g->M = d.M; g->K = d.K; g->O = d.O;
+  g->HoWo = d.conv ? d.Ho * d.Wo : 1;
   if (!w) { g->mode = 0; return; }
   if (d.conv) {
     g->mode = 1;
@@ -981,7 +1001,7 @@ size_t gl_cartesian_dot_workspace(const gl_ap* a0, const gl_windows* w, const gl
   const ConvPlan pl = plan_conv(d);
   if (!pl.tc) return 0;
   size_t need = pl.prepass ? pl.x_bytes + pl.w_bytes : 0;
-  if (!pl.rowwin && pl.Cp >= kBK)
+  if (!pl.rowwin && pl.Cp >= kBK && !(flags & GL_OUT_NCHW))
     need += plan_tiles(d.M, d.O, d.Kh * d.Kw * ((pl.Cp + kBK - 1) / kBK), true).partial_bytes;
   return need;
 }
@@ -994,12 +1014,13 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
   if (rc) return rc;
   if (!out) return GL_ERR_NULL;
   if (a0->dtype != GL_BF16 || a1->dtype != GL_BF16) return GL_ERR_DTYPE;
-  if (flags & ~(GL_EPILOGUE_RELU | GL_DOT_GENERAL_KERNEL)) return GL_ERR_UNSUPPORTED;
+  if (flags & ~(GL_EPILOGUE_RELU | GL_DOT_GENERAL_KERNEL | GL_OUT_NCHW)) return GL_ERR_UNSUPPORTED;
+  const int out_nchw = (flags & GL_OUT_NCHW) ? 1 : 0;
   DotProblem d;
   rc = classify_dot(a0, w, a1, &d);
   if (rc) return rc;
   gl_ap want = *out;
-  rc = gl_shape_cartesian_dot(a0, w, a1, &want);
+  rc = out_nchw ? gl_shape_cartesian_dot_nchw(a0, w, a1, &want) : gl_shape_cartesian_dot(a0, w, a1, &want);
   if (rc) return rc;
   rc = check_same_meta(want, out);
   if (rc) return rc;
@@ -1018,6 +1039,7 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
   if (!use_tc) {
     GenA g;
     fill_general(a0, w, d, &g);
+    g.out_nchw = out_nchw;
     const int64_t gx = (d.O + 63) / 64, gy = (d.M + 63) / 64;
     if (gy > 65535 || gx > 0x7FFFFFFF) return GL_ERR_UNSUPPORTED;
     dot_general<<<dim3(static_cast<unsigned>(gx), static_cast<unsigned>(gy)), 256, 0, st>>>(pa, pb, dst, g, relu);
@@ -1028,9 +1050,10 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
   TcParams p;
   std::memset(&p, 0, sizeof(p));
   p.M = d.M; p.O = d.O; p.relu = relu;
+  p.out_nchw = out_nchw;
   // tile width and K split; a K split needs room for its partial planes behind the layout copies
   const size_t pre_bytes = (d.conv && pl.prepass) ? pl.x_bytes + pl.w_bytes : 0;
-  const bool split_mode = !d.conv || (!pl.rowwin && pl.Cp >= kBK);
+  const bool split_mode = (!d.conv || (!pl.rowwin && pl.Cp >= kBK)) && !out_nchw;
   const int64_t kblocks_all = !d.conv ? (d.K + kBK - 1) / kBK : d.Kh * d.Kw * ((pl.Cp + kBK - 1) / kBK);
   TilePlan tp = plan_tiles(d.M, d.O, kblocks_all, split_mode);
   if (tp.ksplit > 1 && (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023u) ||

@@ -209,6 +209,27 @@ int gl_shape_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1
   return GL_OK;
 }
 
+int gl_shape_cartesian_dot_nchw(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_ap* out) {
+  if (!out) return GL_ERR_NULL;
+  if (!w) return GL_ERR_SHAPE;
+  DotProblem d;
+  int rc = classify_dot(a0, w, a1, &d);
+  if (rc) return rc;
+  if (!d.conv) return GL_ERR_UNSUPPORTED;   // only the conv2d item layouts have an H' and a W'
+  if (a0->access_ndim + a1->access_ndim + 2 > GL_MAX_DIMS) return GL_ERR_NDIM;
+  gl_ap r;
+  std::memset(&r, 0, sizeof(r));
+  r.dtype = GL_F32;
+  for (int i = 0; i < a0->access_ndim; ++i) r.shape[r.ndim++] = a0->shape[i];
+  for (int i = 0; i < a1->access_ndim; ++i) r.shape[r.ndim++] = a1->shape[i];
+  r.shape[r.ndim++] = d.Ho;
+  r.shape[r.ndim++] = d.Wo;
+  r.access_ndim = r.ndim;
+  r.data = out->data;
+  *out = r;
+  return GL_OK;
+}
+
 int gl_shape_reduce_max(const gl_ap* in, const gl_windows* w, gl_ap* out) {
   if (!out) return GL_ERR_NULL;
   int rc = check_meta(in);

@@ -65,6 +65,12 @@ def test_shape_rules_against_interpreter(gl):
     shp, na, _ = gl.gl_shape_reduce_max((n, c, h, w), 2, gl.windows_spec((kh, kw), (sh, sw)))
     assert (shp[:na], shp[na:]) == pool.shape
     assert gl.gl_shape_reduce_max((4, 5, 6), 1, None)[:2] == ((4,), 1)
+    # Fig. 2a in full: transpose(squeeze(dotProd ...)) -> ((N,O,H',W'),())
+    full = gi.transpose(gi.squeeze(dot, 1), (0, 3, 1, 2))
+    shp, na, dt = gl.gl_shape_cartesian_dot_nchw((n, c, h, w), 1, spec, (o, c, kh, kw), 1)
+    assert (shp[:na], shp[na:]) == full.shape and dt == gl.GL_F32
+    cl = gl.windows_spec((kh, kw, c), (sh, sw, 1))
+    assert gl.gl_shape_cartesian_dot_nchw((n, h, w, c), 1, cl, (o, kh, kw, c), 1)[0] == full.data.shape
     # access, flatten edge cases, pad
     assert gl.gl_shape_access((2, 3, 4), 1, 3)[:2] == ((2, 3, 4), 3)
     assert gl.gl_shape_flatten((2, 3, 4), 3)[:2] == ((24,), 1)

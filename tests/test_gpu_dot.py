@@ -132,6 +132,45 @@ def test_conv_gaussian_within_tolerance(gl, case):
     assert rel_err(got, ref) <= REL_TOL
 
 
+@pytest.mark.parametrize("layout", ["nchw", "nhwc"])
+@pytest.mark.parametrize("case", [CONV_SMALL[0], CONV_SMALL[2], CONV_SMALL[3], CONV_SMALL[5], CONV_SMALL[7]])
+def test_conv_fused_squeeze_transpose_is_fig2a(gl, case, layout):
+    # GL_OUT_NCHW: the whole program of Fig. 2a in one call, result ((N,O,H',W'),())
+    n, c, h, w, o, kh, kw, sh, sw, ph, pw = case
+    x = synth.uniform_int(25, 1, (n, c, h, w), -3, 3)
+    wt = synth.uniform_int(25, 2, (o, c, kh, kw), -3, 3)
+    ref = brute.conv2d(x, wt, (sh, sw), ((ph, ph), (pw, pw)))                 # (N,O,H',W')
+    if layout == "nhwc":
+        xa = gl.AccessPattern(to_bf16_device(np.ascontiguousarray(x.transpose(0, 2, 3, 1))), 1)
+        wa = gl.AccessPattern(to_bf16_device(np.ascontiguousarray(wt.transpose(0, 2, 3, 1))), 1)
+        spec = gl.windows_spec((kh, kw, c), (sh, sw, 1), (ph, pw, 0), (ph, pw, 0))
+    else:
+        xa, wa = gl.AccessPattern(to_bf16_device(x), 1), gl.AccessPattern(to_bf16_device(wt), 1)
+        spec = gl.windows_spec((c, kh, kw), (1, sh, sw), (0, ph, pw), (0, ph, pw))
+    for flags in (gl.GL_OUT_NCHW, gl.GL_OUT_NCHW | gl.GL_DOT_GENERAL_KERNEL, gl.GL_OUT_NCHW | gl.GL_EPILOGUE_RELU):
+        out = gl.gl_cartesian_dot(xa, spec, wa, flags=flags)
+        _ok(gl)
+        assert out.shape == ((n, o) + ref.shape[2:], ())
+        want = np.maximum(ref, 0.0) if flags & gl.GL_EPILOGUE_RELU else ref
+        assert np.array_equal(out.tensor.cpu().numpy().astype(np.float64), want)
+    # the same thing in two steps: [M,O] result, then the library's transpose (0 3 1 2)
+    two = gl.gl_cartesian_dot(xa, spec, wa)
+    t = two.tensor.squeeze(3 if layout == "nhwc" else 1).contiguous()
+    nchw = gl.gl_access_transpose(gl.AccessPattern(t, 4), (0, 3, 1, 2))
+    assert np.array_equal(nchw.tensor.cpu().numpy().astype(np.float64), ref)
+    # the interpreter's full program on a small case
+    if n * o * ref.shape[2] * ref.shape[3] * c * kh * kw <= 600000:
+        full = gi.conv2d_program(x, wt, (sh, sw), ((ph, ph), (pw, pw)))
+        assert full.shape == ((n, o) + ref.shape[2:], ()) and np.array_equal(full.data, ref)
+
+
+def test_out_nchw_needs_a_conv(gl):
+    a = gl.AccessPattern(to_bf16_device(synth.uniform_int(26, 1, (8, 16), -3, 3)), 1)
+    out = gl.AccessPattern(torch.empty((8, 8), device="cuda"), 2)
+    with pytest.raises(gl.GlError):
+        gl.gl_cartesian_dot(a, None, a, out=out, flags=gl.GL_OUT_NCHW)
+
+
 def test_windows_over_other_dims_uses_general_kernel(gl):
     # windows that also slide over the channel dim: not a conv2d, still a valid program
     x = synth.uniform_int(24, 1, (2, 5, 6, 7), -3, 3)
