@@ -953,6 +953,13 @@ ConvPlan plan_conv(const DotProblem& d) {
   return pl;
 }
 
+// A 1x1, stride-1, unpadded window over channels-last items is no window at all: the activations
+// already are the [N*H*W, C] matrix (the special case "1x1 conv == matmul").
+bool conv_is_plain_matrix(const DotProblem& d, uint32_t flags) {
+  return d.conv && d.channels_last && d.Kh == 1 && d.Kw == 1 && d.Sh == 1 && d.Sw == 1 && d.ph_lo == 0 &&
+         d.ph_hi == 0 && d.pw_lo == 0 && d.pw_hi == 0 && d.C % 8 == 0 && !(flags & GL_OUT_NCHW);
+}
+
 bool dense_tc_ok(const DotProblem& d) {
   return !d.conv && !d.general && d.K % 8 == 0 && d.M < (1ll << 31) && d.O < (1ll << 31) && d.K < (1ll << 31);
 }
@@ -994,6 +1001,7 @@ size_t gl_cartesian_dot_workspace(const gl_ap* a0, const gl_windows* w, const gl
   DotProblem d;
   if (classify_dot(a0, w, a1, &d) != GL_OK) return 0;
   if (flags & GL_DOT_GENERAL_KERNEL) return 0;
+  if (conv_is_plain_matrix(d, flags)) d.conv = false;
   if (!d.conv) {
     if (!dense_tc_ok(d)) return 0;
     return plan_tiles(d.M, d.O, (d.K + kBK - 1) / kBK, true).partial_bytes;
@@ -1033,6 +1041,7 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
   const uint16_t* pb = static_cast<const uint16_t*>(a1->data);
 
   const bool force_general = (flags & GL_DOT_GENERAL_KERNEL) != 0;
+  if (!force_general && conv_is_plain_matrix(d, flags)) d.conv = false;
   ConvPlan pl;
   if (d.conv) pl = plan_conv(d);
   const bool use_tc = !force_general && ((d.conv && pl.tc) || dense_tc_ok(d));

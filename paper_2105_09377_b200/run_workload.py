@@ -45,6 +45,21 @@ def build_call(cfg, layout: str, device, batch=None, flags=0):
         if batch:
             cfg = synth.ConvCase(cfg.name, batch, cfg.c, cfg.h, cfg.w, cfg.o, cfg.kh, cfg.kw, cfg.stride, cfg.pad, cfg.integer)
         x, wt = _inputs(cfg, synth.config_seed(2))
+        if layout == "rewritten":
+            # Section 5.3: flatten(windows(act)) materialised as the im2col matrix, flatten(weights), plain matmul
+            spec = gl.windows_spec((cfg.c, cfg.kh, cfg.kw), (1, cfg.stride, cfg.stride), (0, cfg.pad, cfg.pad), (0, cfg.pad, cfg.pad))
+            xa, wa = gl.AccessPattern(_bf16(x, device), 1), gl.AccessPattern(_bf16(wt, device), 1)
+            cols = gl.output_like(gl.gl_shape_windows(x.shape, 1, spec, gl.GL_BF16), device)
+            flat, wflat = gl.gl_access_flatten(cols), gl.gl_access_flatten(wa)
+            out = gl.output_like(gl.gl_shape_cartesian_dot(tuple(flat.tensor.shape), 1, None, tuple(wflat.tensor.shape), 1), device)
+            need = gl.gl_cartesian_dot_workspace(flat, None, wflat, flags)
+            ws = torch.empty(need + 1024, dtype=torch.uint8, device=device) if need else None
+            steps = (gl.prepare_access_windows(xa, spec, cols), gl.prepare_cartesian_dot(flat, None, wflat, out, flags, ws))
+
+            def both(stream=None):
+                for step in steps:
+                    step(stream)
+            return both, cfg.flops, cfg.algorithmic_bytes
         if layout == "nhwc":
             x, wt = x.transpose(0, 2, 3, 1).copy(), wt.transpose(0, 2, 3, 1).copy()
             spec = gl.windows_spec((cfg.kh, cfg.kw, cfg.c), (cfg.stride, cfg.stride, 1), (cfg.pad, cfg.pad, 0), (cfg.pad, cfg.pad, 0))
@@ -75,7 +90,7 @@ def main():
     table = workloads()
     ap = argparse.ArgumentParser()
     ap.add_argument("--workload", required=True, choices=sorted(table))
-    ap.add_argument("--layout", default="nhwc", choices=["nhwc", "nchw"])
+    ap.add_argument("--layout", default="nhwc", choices=["nhwc", "nchw", "rewritten"])
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--batch", type=int, default=0, help="override the leading (batch) extent")
     ap.add_argument("--graph", action="store_true", help="time one CUDA graph holding all iterations")
