@@ -164,6 +164,45 @@ def test_conv_fused_squeeze_transpose_is_fig2a(gl, case, layout):
         assert full.shape == ((n, o) + ref.shape[2:], ()) and np.array_equal(full.data, ref)
 
 
+def _random_conv_cases(count, seed):
+    rng = np.random.default_rng(seed)
+    cases = []
+    while len(cases) < count:
+        c = int(rng.choice([1, 3, 4, 8, 12, 16, 24, 32, 40, 64, 72, 128, 136]))
+        kh, kw = int(rng.integers(1, 5)), int(rng.integers(1, 5))
+        sh, sw = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+        ph, pw = int(rng.integers(0, kh)), int(rng.integers(0, kw))
+        h, w = int(rng.integers(kh, 20)), int(rng.integers(kw, 20))
+        n, o = int(rng.integers(1, 5)), int(rng.choice([1, 3, 8, 20, 64, 70, 130, 260]))
+        if n * c * h * w * o * kh * kw > 6e7:
+            continue
+        cases.append((n, c, h, w, o, kh, kw, sh, sw, ph, pw))
+    return cases
+
+
+@pytest.mark.parametrize("case", _random_conv_cases(40, 2105), ids=lambda c: "x".join(map(str, c)))
+def test_conv_random_shapes_bit_exact(gl, case):
+    # seeded shape fuzzing across all tensor-core modes (dense shortcut, im2col, row-window, granule, K split)
+    n, c, h, w, o, kh, kw, sh, sw, ph, pw = case
+    x = synth.uniform_int(sum(case), 1, (n, c, h, w), -3, 3)
+    wt = synth.uniform_int(sum(case), 2, (o, c, kh, kw), -3, 3)
+    ref = _conv_ref(x, wt, (sh, sw), (ph, pw))
+    for cl in (False, True):
+        got = _conv_gpu(gl, x, wt, (sh, sw), (ph, pw), channels_last=cl)
+        assert got.shape == ref.shape
+        assert np.array_equal(got.astype(np.float64), ref), "layout channels_last=%s" % cl
+
+
+@pytest.mark.parametrize("m,o,k", [(int(a), int(b), int(c) * 8) for a, b, c in
+                                   np.random.default_rng(99).integers(1, 400, (16, 3))])
+def test_dense_random_shapes_bit_exact(gl, m, o, k):
+    a = synth.uniform_int(m + o, 1, (m, k), -3, 3)
+    b = synth.uniform_int(m + o, 2, (o, k), -3, 3)
+    out = gl.gl_cartesian_dot(gl.AccessPattern(to_bf16_device(a), 1), None, gl.AccessPattern(to_bf16_device(b), 1))
+    _ok(gl)
+    assert np.array_equal(out.tensor.cpu().numpy().astype(np.float64), brute.rowdot(a, b))
+
+
 def test_out_nchw_needs_a_conv(gl):
     a = gl.AccessPattern(to_bf16_device(synth.uniform_int(26, 1, (8, 16), -3, 3)), 1)
     out = gl.AccessPattern(torch.empty((8, 8), device="cuda"), 2)
