@@ -115,6 +115,27 @@ GL_API int gl_shape_transpose(const gl_ap* in, const int32_t* perm, gl_ap* out);
 /* `pad` (not in the paper): dimension `dim` grows by lo + hi. */
 GL_API int gl_shape_pad(const gl_ap* in, int32_t dim, int64_t lo, int64_t hi, gl_ap* out);
 
+/* `slice` (transformer table): dimension `dim` keeps [lo, hi). */
+GL_API int gl_shape_slice(const gl_ap* in, int32_t dim, int64_t lo, int64_t hi, gl_ap* out);
+
+/* `concat` (used by the blocking rewrites of Section 5.4, Fig. 7): join a and b along `dim`; all
+ * other extents, the split position and the dtype must agree. */
+GL_API int gl_shape_concat(const gl_ap* a, const gl_ap* b, int32_t dim, gl_ap* out);
+
+/* `pair` (transformer table): two patterns of one shape -> ((a..),(2, c..)). */
+GL_API int gl_shape_pair(const gl_ap* a, const gl_ap* b, gl_ap* out);
+
+/* `squeeze` (transformer table): drop dimension `dim`, which must have extent 1.  Metadata only:
+ * the data of the result is the data of the input. */
+GL_API int gl_shape_squeeze(const gl_ap* in, int32_t dim, gl_ap* out);
+
+/* `reshape` (transformer table): new shape `shape[0..ndim)` split at `access_ndim`; the element
+ * counts of the access side and of the compute side must both be kept.  Metadata only. */
+GL_API int gl_shape_reshape(const gl_ap* in, const int64_t* shape, int32_t ndim, int32_t access_ndim, gl_ap* out);
+
+/* compute reduceSum (operator table): ((access dims),()). */
+GL_API int gl_shape_reduce_sum(const gl_ap* in, gl_ap* out);
+
 /* compute dotProd (cartProd (windows? a0) a1)  (Section 4.2 cartProd, Section 4.3
  * dotProd, Fig. 2a/2b): with A = windows(a0) (or a0 itself when w is NULL) of shape
  * ((m..),(k..)) and a1 of shape ((o..),(k..)), the result is ((m.., o..),()), GL_F32. */
@@ -149,6 +170,15 @@ GL_API int gl_access_transpose(const gl_ap* in, const int32_t* perm, gl_ap* out,
 /* Materialised `pad` of one dimension with 0 or -inf (not in the paper). */
 GL_API int gl_access_pad(const gl_ap* in, int32_t dim, int64_t lo, int64_t hi, int32_t pad_kind,
                   gl_ap* out, void* stream);
+
+/* `slice`, `concat`, `pair` with data movement (transformer table; Fig. 7).  GL_F32 or GL_BF16. */
+GL_API int gl_access_slice(const gl_ap* in, int32_t dim, int64_t lo, int64_t hi, gl_ap* out, void* stream);
+GL_API int gl_access_concat(const gl_ap* a, const gl_ap* b, int32_t dim, gl_ap* out, void* stream);
+GL_API int gl_access_pair(const gl_ap* a, const gl_ap* b, gl_ap* out, void* stream);
+
+/* compute reduceSum (operator table): the sum of every item, GL_F32, added in a fixed order (a
+ * strided partial sum per lane of one warp, then a butterfly), so results repeat bit for bit. */
+GL_API int gl_compute_reduce_sum(const gl_ap* in, gl_ap* out, void* stream);
 
 /* out = compute dotProd (cartProd (windows? a0) a1), optionally followed by compute
  * relu (Fig. 2a for conv2d with w given, Fig. 2b / Fig. 6 for matrix products with

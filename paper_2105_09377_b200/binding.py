@@ -53,6 +53,8 @@ EXPORTS = [
     "gl_access_transpose", "gl_access_pad", "gl_cartesian_dot", "gl_cartesian_dot_workspace",
     "gl_compute_reduce_max", "gl_compute_relu", "gl_poll_device_status", "gl_strerror", "gl_version",
     "gl_cartesian_dot_static", "gl_shape_cartesian_dot_nchw",
+    "gl_shape_slice", "gl_shape_concat", "gl_shape_pair", "gl_shape_squeeze", "gl_shape_reshape",
+    "gl_shape_reduce_sum", "gl_access_slice", "gl_access_concat", "gl_access_pair", "gl_compute_reduce_sum",
 ]
 
 
@@ -73,6 +75,16 @@ def _load() -> ctypes.CDLL:
         "gl_shape_cartesian_dot": [ap, win, ap, ap],
         "gl_shape_cartesian_dot_nchw": [ap, win, ap, ap],
         "gl_shape_reduce_max": [ap, win, ap],
+        "gl_shape_slice": [ap, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, ap],
+        "gl_shape_concat": [ap, ap, ctypes.c_int32, ap],
+        "gl_shape_pair": [ap, ap, ap],
+        "gl_shape_squeeze": [ap, ctypes.c_int32, ap],
+        "gl_shape_reshape": [ap, ctypes.POINTER(ctypes.c_int64), ctypes.c_int32, ctypes.c_int32, ap],
+        "gl_shape_reduce_sum": [ap, ap],
+        "gl_access_slice": [ap, ctypes.c_int32, ctypes.c_int64, ctypes.c_int64, ap, vp],
+        "gl_access_concat": [ap, ap, ctypes.c_int32, ap, vp],
+        "gl_access_pair": [ap, ap, ap, vp],
+        "gl_compute_reduce_sum": [ap, ap, vp],
         "gl_access_windows": [ap, win, ap, vp],
         "gl_access_flatten": [ap, ap],
         "gl_access_transpose": [ap, i32p, ap, vp],
@@ -341,6 +353,70 @@ def gl_compute_reduce_max(a: AccessPattern, w: Optional[GlWindows], out: Optiona
         out = _alloc(m, a.tensor.device)
     so = _struct(out)
     _check(LIB.gl_compute_reduce_max(ctypes.byref(sa), _wptr(w), ctypes.byref(so), _stream(stream)), "gl_compute_reduce_max")
+    return out
+
+
+def gl_access_slice(a: AccessPattern, dim: int, lo: int, hi: int, out: Optional[AccessPattern] = None,
+                    stream=None) -> AccessPattern:
+    sa = _struct(a)
+    if out is None:
+        m = GlAp()
+        _check(LIB.gl_shape_slice(ctypes.byref(sa), dim, lo, hi, ctypes.byref(m)), "gl_shape_slice")
+        out = _alloc(m, a.tensor.device)
+    so = _struct(out)
+    _check(LIB.gl_access_slice(ctypes.byref(sa), dim, lo, hi, ctypes.byref(so), _stream(stream)), "gl_access_slice")
+    return out
+
+
+def gl_access_concat(a: AccessPattern, b: AccessPattern, dim: int, out: Optional[AccessPattern] = None,
+                     stream=None) -> AccessPattern:
+    sa, sb = _struct(a), _struct(b)
+    if out is None:
+        m = GlAp()
+        _check(LIB.gl_shape_concat(ctypes.byref(sa), ctypes.byref(sb), dim, ctypes.byref(m)), "gl_shape_concat")
+        out = _alloc(m, a.tensor.device)
+    so = _struct(out)
+    _check(LIB.gl_access_concat(ctypes.byref(sa), ctypes.byref(sb), dim, ctypes.byref(so), _stream(stream)),
+           "gl_access_concat")
+    return out
+
+
+def gl_access_pair(a: AccessPattern, b: AccessPattern, out: Optional[AccessPattern] = None, stream=None) -> AccessPattern:
+    sa, sb = _struct(a), _struct(b)
+    if out is None:
+        m = GlAp()
+        _check(LIB.gl_shape_pair(ctypes.byref(sa), ctypes.byref(sb), ctypes.byref(m)), "gl_shape_pair")
+        out = _alloc(m, a.tensor.device)
+    so = _struct(out)
+    _check(LIB.gl_access_pair(ctypes.byref(sa), ctypes.byref(sb), ctypes.byref(so), _stream(stream)), "gl_access_pair")
+    return out
+
+
+def gl_access_squeeze(a: AccessPattern, dim: int) -> AccessPattern:
+    """`squeeze` is metadata: the result views the same storage."""
+    m = GlAp()
+    _check(LIB.gl_shape_squeeze(ctypes.byref(_struct(a)), dim, ctypes.byref(m)), "gl_shape_squeeze")
+    return AccessPattern(a.tensor.view(tuple(m.shape[i] for i in range(m.ndim))), m.access_ndim)
+
+
+def gl_access_reshape(a: AccessPattern, access_shape, compute_shape) -> AccessPattern:
+    """`reshape` is metadata: the result views the same storage."""
+    shape = tuple(access_shape) + tuple(compute_shape)
+    arr = (ctypes.c_int64 * max(1, len(shape)))(*shape)
+    m = GlAp()
+    _check(LIB.gl_shape_reshape(ctypes.byref(_struct(a)), arr, len(shape), len(access_shape), ctypes.byref(m)),
+           "gl_shape_reshape")
+    return AccessPattern(a.tensor.view(shape), len(access_shape))
+
+
+def gl_compute_reduce_sum(a: AccessPattern, out: Optional[AccessPattern] = None, stream=None) -> AccessPattern:
+    sa = _struct(a)
+    if out is None:
+        m = GlAp()
+        _check(LIB.gl_shape_reduce_sum(ctypes.byref(sa), ctypes.byref(m)), "gl_shape_reduce_sum")
+        out = _alloc(m, a.tensor.device)
+    so = _struct(out)
+    _check(LIB.gl_compute_reduce_sum(ctypes.byref(sa), ctypes.byref(so), _stream(stream)), "gl_compute_reduce_sum")
     return out
 
 

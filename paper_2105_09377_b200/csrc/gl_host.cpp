@@ -191,6 +191,91 @@ int gl_shape_pad(const gl_ap* in, int32_t dim, int64_t lo, int64_t hi, gl_ap* ou
   return GL_OK;
 }
 
+int gl_shape_slice(const gl_ap* in, int32_t dim, int64_t lo, int64_t hi, gl_ap* out) {
+  int rc = check_meta(in);
+  if (rc) return rc;
+  if (!out) return GL_ERR_NULL;
+  if (dim < 0 || dim >= in->ndim) return GL_ERR_NDIM;
+  if (lo < 0 || hi <= lo || hi > in->shape[dim]) return GL_ERR_SHAPE;
+  copy_meta(in, out);
+  out->shape[dim] = hi - lo;
+  return GL_OK;
+}
+
+int gl_shape_concat(const gl_ap* a, const gl_ap* b, int32_t dim, gl_ap* out) {
+  int rc = check_meta(a);
+  if (rc) return rc;
+  rc = check_meta(b);
+  if (rc) return rc;
+  if (!out) return GL_ERR_NULL;
+  if (a->dtype != b->dtype) return GL_ERR_DTYPE;
+  if (dim < 0 || dim >= a->ndim) return GL_ERR_NDIM;
+  if (a->ndim != b->ndim || a->access_ndim != b->access_ndim) return GL_ERR_SHAPE;
+  for (int i = 0; i < a->ndim; ++i)
+    if (i != dim && a->shape[i] != b->shape[i]) return GL_ERR_SHAPE;
+  copy_meta(a, out);
+  out->shape[dim] = a->shape[dim] + b->shape[dim];
+  return GL_OK;
+}
+
+int gl_shape_pair(const gl_ap* a, const gl_ap* b, gl_ap* out) {
+  int rc = check_meta(a);
+  if (rc) return rc;
+  rc = check_meta(b);
+  if (rc) return rc;
+  if (!out) return GL_ERR_NULL;
+  if (a->dtype != b->dtype) return GL_ERR_DTYPE;
+  if (a->ndim + 1 > GL_MAX_DIMS) return GL_ERR_NDIM;
+  if (a->ndim != b->ndim || a->access_ndim != b->access_ndim) return GL_ERR_SHAPE;
+  for (int i = 0; i < a->ndim; ++i)
+    if (a->shape[i] != b->shape[i]) return GL_ERR_SHAPE;
+  gl_ap r = *a;
+  r.ndim = a->ndim + 1;
+  r.shape[a->access_ndim] = 2;   // the 2 is the first compute dimension
+  for (int i = a->access_ndim; i < a->ndim; ++i) r.shape[i + 1] = a->shape[i];
+  r.data = out->data;
+  *out = r;
+  return GL_OK;
+}
+
+int gl_shape_squeeze(const gl_ap* in, int32_t dim, gl_ap* out) {
+  int rc = check_meta(in);
+  if (rc) return rc;
+  if (!out) return GL_ERR_NULL;
+  if (dim < 0 || dim >= in->ndim) return GL_ERR_NDIM;
+  if (in->shape[dim] != 1) return GL_ERR_SHAPE;
+  gl_ap r = *in;
+  for (int i = dim; i + 1 < in->ndim; ++i) r.shape[i] = in->shape[i + 1];
+  r.shape[in->ndim - 1] = 0;
+  r.ndim = in->ndim - 1;
+  if (dim < in->access_ndim) r.access_ndim = in->access_ndim - 1;
+  r.data = out->data;
+  *out = r;
+  return GL_OK;
+}
+
+int gl_shape_reshape(const gl_ap* in, const int64_t* shape, int32_t ndim, int32_t access_ndim, gl_ap* out) {
+  int rc = check_meta(in);
+  if (rc) return rc;
+  if (!out || (!shape && ndim > 0)) return GL_ERR_NULL;
+  if (ndim < 0 || ndim > GL_MAX_DIMS || access_ndim < 0 || access_ndim > ndim) return GL_ERR_NDIM;
+  for (int i = 0; i < ndim; ++i)
+    if (shape[i] < 1) return GL_ERR_SHAPE;
+  if (prod(shape, 0, access_ndim) != prod(in->shape, 0, in->access_ndim)) return GL_ERR_SHAPE;
+  if (prod(shape, access_ndim, ndim) != prod(in->shape, in->access_ndim, in->ndim)) return GL_ERR_SHAPE;
+  gl_ap r;
+  std::memset(&r, 0, sizeof(r));
+  r.dtype = in->dtype;
+  r.ndim = ndim;
+  r.access_ndim = access_ndim;
+  for (int i = 0; i < ndim; ++i) r.shape[i] = shape[i];
+  r.data = out->data;
+  *out = r;
+  return GL_OK;
+}
+
+int gl_shape_reduce_sum(const gl_ap* in, gl_ap* out) { return gl_shape_reduce_max(in, nullptr, out); }
+
 int gl_shape_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_ap* out) {
   if (!out) return GL_ERR_NULL;
   DotProblem d;

@@ -636,6 +636,57 @@ __global__ void relu_tail(const float* __restrict__ in, float* __restrict__ out,
   if (i < n) out[i] = in[i] > 0.f ? in[i] : 0.f;
 }
 
+// slice / concat / pair: dst[u, dst_off + d, i] = src[u, src_off + d, i] for d < count, the tensors seen
+// as (outer, dim, inner).
+template <typename V>
+__global__ void __launch_bounds__(kThreads) copy_dim_block(const V* __restrict__ src, V* __restrict__ dst,
+                                                           int64_t outer, int64_t d_src, int64_t src_off,
+                                                           int64_t d_dst, int64_t dst_off, int64_t count,
+                                                           int64_t inner) {
+  const int64_t total = outer * count * inner;
+  for (int64_t c = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; c < total; c += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t i = c % inner;
+    const int64_t d = (c / inner) % count;
+    const int64_t u = c / (inner * count);
+    dst[(u * d_dst + dst_off + d) * inner + i] = src[(u * d_src + src_off + d) * inner + i];
+  }
+}
+
+// reduceSum of whole items: one warp per item, lane l adds cells l, l+32, ... in order, then a
+// fixed butterfly: the order of additions does not depend on the launch.
+__global__ void __launch_bounds__(kThreads) item_sum(const float* __restrict__ in, float* __restrict__ out,
+                                                      int64_t items, int64_t item) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+  for (int64_t a = blockIdx.x * (int64_t)(blockDim.x >> 5) + (threadIdx.x >> 5); a < items; a += warps) {
+    float acc = 0.f;
+    for (int64_t i = lane; i < item; i += 32) acc += in[a * item + i];
+#pragma unroll
+    for (int s = 16; s > 0; s >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, s);
+    if (lane == 0) out[a] = acc;
+  }
+}
+
+int run_copy_dim(const void* src, void* dst, int dtype, int64_t outer, int64_t d_src, int64_t src_off, int64_t d_dst,
+                 int64_t dst_off, int64_t count, int64_t inner, cudaStream_t st) {
+  const size_t es = dtype_size(dtype);
+  const int vec = static_cast<int>(16 / es);
+  const int64_t total = outer * count * inner;
+  if (total == 0) return GL_OK;
+  if (inner % vec == 0) {   // every row piece starts on a 16-byte boundary (bases are 16-byte aligned)
+    const int64_t iv = inner / vec;
+    copy_dim_block<uint4><<<grid_for(outer * count * iv, kThreads), kThreads, 0, st>>>(
+        static_cast<const uint4*>(src), static_cast<uint4*>(dst), outer, d_src, src_off, d_dst, dst_off, count, iv);
+  } else if (dtype == GL_F32) {
+    copy_dim_block<uint32_t><<<grid_for(total, kThreads), kThreads, 0, st>>>(
+        static_cast<const uint32_t*>(src), static_cast<uint32_t*>(dst), outer, d_src, src_off, d_dst, dst_off, count, inner);
+  } else {
+    copy_dim_block<uint16_t><<<grid_for(total, kThreads), kThreads, 0, st>>>(
+        static_cast<const uint16_t*>(src), static_cast<uint16_t*>(dst), outer, d_src, src_off, d_dst, dst_off, count, inner);
+  }
+  return launch_status();
+}
+
 void fill_win_params(const gl_ap* in, const gl_windows* w, const gl_ap& A, WinParams* p) {
   std::memset(p, 0, sizeof(*p));
   const int na = in->access_ndim;
@@ -870,6 +921,80 @@ int gl_compute_reduce_max(const gl_ap* in, const gl_windows* w, gl_ap* out, void
   WinParams p;
   fill_win_params(in, w, A, &p);
   window_max_generic<<<grid_for(nwin, kThreads), kThreads, 0, st>>>(src, dst, p, nwin, fill);
+  return launch_status();
+}
+
+int gl_access_slice(const gl_ap* in, int32_t dim, int64_t lo, int64_t hi, gl_ap* out, void* stream) {
+  int rc = check_data(in);
+  if (rc) return rc;
+  if (!out) return GL_ERR_NULL;
+  gl_ap want = *in;
+  rc = gl_shape_slice(in, dim, lo, hi, &want);
+  if (rc) return rc;
+  rc = check_same_meta(want, out);
+  if (rc) return rc;
+  rc = check_data(out);
+  if (rc) return rc;
+  return run_copy_dim(in->data, out->data, in->dtype, prod(in->shape, 0, dim), in->shape[dim], lo, hi - lo, 0, hi - lo,
+                      prod(in->shape, dim + 1, in->ndim), static_cast<cudaStream_t>(stream));
+}
+
+int gl_access_concat(const gl_ap* a, const gl_ap* b, int32_t dim, gl_ap* out, void* stream) {
+  int rc = check_data(a);
+  if (rc) return rc;
+  rc = check_data(b);
+  if (rc) return rc;
+  if (!out) return GL_ERR_NULL;
+  gl_ap want = *a;
+  rc = gl_shape_concat(a, b, dim, &want);
+  if (rc) return rc;
+  rc = check_same_meta(want, out);
+  if (rc) return rc;
+  rc = check_data(out);
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t outer = prod(a->shape, 0, dim), inner = prod(a->shape, dim + 1, a->ndim);
+  const int64_t da = a->shape[dim], db = b->shape[dim];
+  rc = run_copy_dim(a->data, out->data, a->dtype, outer, da, 0, da + db, 0, da, inner, st);
+  if (rc) return rc;
+  return run_copy_dim(b->data, out->data, a->dtype, outer, db, 0, da + db, da, db, inner, st);
+}
+
+int gl_access_pair(const gl_ap* a, const gl_ap* b, gl_ap* out, void* stream) {
+  int rc = check_data(a);
+  if (rc) return rc;
+  rc = check_data(b);
+  if (rc) return rc;
+  if (!out) return GL_ERR_NULL;
+  gl_ap want = *a;
+  rc = gl_shape_pair(a, b, &want);
+  if (rc) return rc;
+  rc = check_same_meta(want, out);
+  if (rc) return rc;
+  rc = check_data(out);
+  if (rc) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int64_t outer = prod(a->shape, 0, a->access_ndim), inner = prod(a->shape, a->access_ndim, a->ndim);
+  rc = run_copy_dim(a->data, out->data, a->dtype, outer, 1, 0, 2, 0, 1, inner, st);
+  if (rc) return rc;
+  return run_copy_dim(b->data, out->data, a->dtype, outer, 1, 0, 2, 1, 1, inner, st);
+}
+
+int gl_compute_reduce_sum(const gl_ap* in, gl_ap* out, void* stream) {
+  int rc = check_data(in);
+  if (rc) return rc;
+  if (!out) return GL_ERR_NULL;
+  if (in->dtype != GL_F32) return GL_ERR_DTYPE;
+  gl_ap want = *in;
+  rc = gl_shape_reduce_sum(in, &want);
+  if (rc) return rc;
+  rc = check_same_meta(want, out);
+  if (rc) return rc;
+  rc = check_data(out);
+  if (rc) return rc;
+  const int64_t items = prod(in->shape, 0, in->access_ndim), item = prod(in->shape, in->access_ndim, in->ndim);
+  item_sum<<<grid_for(items, kThreads / 32), kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
+      static_cast<const float*>(in->data), static_cast<float*>(out->data), items, item);
   return launch_status();
 }
 

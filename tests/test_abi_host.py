@@ -121,3 +121,46 @@ def test_argument_errors(gl):
     rc = gl.LIB.gl_compute_relu(ctypes.byref(a), ctypes.byref(a), None)
     assert rc == 6                                              # GL_ERR_ALIGN
     assert gl.LIB.gl_cartesian_dot_workspace(ctypes.byref(a), None, ctypes.byref(out), 0) == 0
+
+
+def test_blocking_transformer_shapes(gl, golden_dir):
+    """slice / transpose / cartProd / dotProd / pair / reduceSum / concat: the library's shape rules
+    reproduce the annotations of the blocked 32x32 matMul (Fig. 8) and agree with the interpreter."""
+    import ctypes as ct
+
+    def shape_of(fn, *args):
+        out = gl.GlAp()
+        rc = fn(*args, ct.byref(out))
+        assert rc == 0, rc
+        shp = tuple(out.shape[i] for i in range(out.ndim))
+        return (shp[:out.access_ndim], shp[out.access_ndim:])
+
+    m = gl._meta
+    act = m((32, 32), 1, gl.GL_BF16)
+    s1 = gl.GlAp()
+    assert gl.LIB.gl_shape_slice(ct.byref(act), 0, 0, 16, ct.byref(s1)) == 0
+    assert shape_of(gl.LIB.gl_shape_slice, ct.byref(s1), 1, 0, 16) == ((16,), (16,))
+    dot = m((16, 16), 2, gl.GL_F32)
+    assert shape_of(gl.LIB.gl_shape_pair, ct.byref(dot), ct.byref(dot)) == ((16, 16), (2,))
+    pr = m((16, 16, 2), 2, gl.GL_F32)
+    assert shape_of(gl.LIB.gl_shape_reduce_sum, ct.byref(pr)) == ((16, 16), ())
+    assert shape_of(gl.LIB.gl_shape_concat, ct.byref(dot), ct.byref(dot), 1) == ((16, 32), ())
+    row = m((16, 32), 2, gl.GL_F32)
+    assert shape_of(gl.LIB.gl_shape_concat, ct.byref(row), ct.byref(row), 0) == ((32, 32), ())
+    # against the interpreter on lopsided shapes
+    a = gi.access(np.zeros((2, 3, 4, 5)), 2)
+    am = m((2, 3, 4, 5), 2, gl.GL_F32)
+    assert shape_of(gl.LIB.gl_shape_slice, ct.byref(am), 2, 1, 3) == gi.slice_(a, 2, 1, 3).shape
+    assert shape_of(gl.LIB.gl_shape_pair, ct.byref(am), ct.byref(am)) == gi.pair(a, a).shape
+    b = m((2, 3, 6, 5), 2, gl.GL_F32)
+    assert shape_of(gl.LIB.gl_shape_concat, ct.byref(am), ct.byref(b), 2) == gi.concat(a, gi.access(np.zeros((2, 3, 6, 5)), 2), 2).shape
+    assert shape_of(gl.LIB.gl_shape_squeeze, ct.byref(m((2, 1, 3), 2, gl.GL_F32)), 1) == gi.squeeze(gi.access(np.zeros((2, 1, 3)), 2), 1).shape
+    assert shape_of(gl.LIB.gl_shape_squeeze, ct.byref(m((2, 3, 1), 2, gl.GL_F32)), 2) == ((2, 3), ())
+    arr = (ct.c_int64 * 3)(6, 2, 10)
+    assert shape_of(gl.LIB.gl_shape_reshape, ct.byref(am), arr, 3, 1) == gi.reshape(a, (6,), (2, 10)).shape
+    out = gl.GlAp()
+    bad = (ct.c_int64 * 2)(3, 40)
+    assert gl.LIB.gl_shape_reshape(ct.byref(am), bad, 2, 1, ct.byref(out)) == 4
+    assert gl.LIB.gl_shape_slice(ct.byref(am), 2, 3, 3, ct.byref(out)) == 4          # empty range
+    assert gl.LIB.gl_shape_concat(ct.byref(am), ct.byref(m((2, 4, 4, 5), 2, gl.GL_F32)), 2, ct.byref(out)) == 4
+    assert gl.LIB.gl_shape_squeeze(ct.byref(am), 0, ct.byref(out)) == 4
