@@ -463,7 +463,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
     const bool load_a = warp == 0;
     if (lane == 0) {
       asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(load_a ? &map_a : &map_b)) : "memory");
-      uint32_t it = 0;
+      uint32_t s = 0, ph = 0;   // ring slot and its phase, advanced by hand (no division in this thread)
       bool ok = true;
       for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x) {
         uint32_t t, ks, tm, tn;
@@ -496,8 +496,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
           kh = tap / p.Kw;
           kw = tap - kh * p.Kw;
         }
-        for (int kb0 = kb_begin; kb0 < kb_end; kb0 += G, ++it) {
-          const uint32_t s = it % Cfg::kStages, ph = (it / Cfg::kStages) & 1u;
+        for (int kb0 = kb_begin; kb0 < kb_end; kb0 += G) {
           if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
           const uint32_t full = bar_full + 8 * s;
           const uint32_t stage = tiles + s * Cfg::kStage;
@@ -538,6 +537,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
               tma_load_3d(sb, &map_b, 0, n0, kb * 8, full);
             }
           }
+          if (++s == Cfg::kStages) { s = 0; ph ^= 1u; }
         }
       }
     }
@@ -548,7 +548,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
       const uint64_t desc_a0 = (MODE == kIm2colGranule) ? make_desc(tiles, kBM * 16, 128, 0) : make_desc(tiles, 16, 1024, 2);
       const uint64_t desc_b0 = (MODE == kIm2colGranule) ? make_desc(tiles + G * Cfg::kStageA, BN * 16, 128, 0)
                                                         : make_desc(tiles + G * Cfg::kStageA, 16, 1024, 2);
-      uint32_t it = 0, tile_it = 0;
+      uint32_t s = 0, ph = 0, tile_it = 0;
       bool ok = true;
       for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x, ++tile_it) {
         const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
@@ -558,8 +558,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
         if (!mbar_wait(bar_tempty + 8 * acc, aph ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
-        for (int kb0 = kb_begin; kb0 < kb_end; kb0 += G, ++it) {
-          const uint32_t s = it % Cfg::kStages, ph = (it / Cfg::kStages) & 1u;
+        for (int kb0 = kb_begin; kb0 < kb_end; kb0 += G) {
           if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
           // descriptors differ only in their start-address field (16-byte units): add offsets to a base
@@ -581,6 +580,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
           // one commit per stage (it costs the issuing thread a few hundred cycles): frees the
           // stage once these MMAs have read it
           tc_commit(bar_empty + 8 * s);
+          if (++s == Cfg::kStages) { s = 0; ph ^= 1u; }
         }
         if (ok) tc_commit(bar_tfull + 8 * acc);
       }
