@@ -1,0 +1,41 @@
+"""Operators composed into one program on the device: the conv2d of Fig. 2a (squeeze and transpose
+fused, relu in the epilogue) followed by the max pooling of Fig. 2c, against the same chain run by
+the CPU checker.  Integer inputs: every intermediate is exact, so the comparison is bit for bit."""
+import numpy as np
+import pytest
+
+from oracle import brute
+from oracle import interp as gi
+from paper_2105_09377_b200 import synth
+from tests.gpu_util import to_bf16_device
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gl():
+    from paper_2105_09377_b200 import binding
+    return binding
+
+
+@pytest.mark.parametrize("n,c,h,w,o", [(2, 3, 23, 21, 8), (1, 16, 18, 18, 24), (2, 64, 12, 12, 64)])
+def test_conv_relu_maxpool_chain(gl, n, c, h, w, o):
+    x = synth.uniform_int(61, 1, (n, c, h, w), -3, 3)
+    wt = synth.uniform_int(61, 2, (o, c, 3, 3), -3, 3)
+    # device: conv 3x3 pad 1 -> relu -> (N,O,H,W) -> max pool 3x3 stride 2 pad 1
+    spec = gl.windows_spec((c, 3, 3), (1, 1, 1), (0, 1, 1), (0, 1, 1))
+    act = gl.gl_cartesian_dot(gl.AccessPattern(to_bf16_device(x), 1), spec, gl.AccessPattern(to_bf16_device(wt), 1),
+                              flags=gl.GL_OUT_NCHW | gl.GL_EPILOGUE_RELU)
+    assert act.shape == ((n, o, h, w), ())
+    pooled = gl.gl_compute_reduce_max(gl.AccessPattern(act.tensor, 2),
+                                      gl.windows_spec((3, 3), (2, 2), (1, 1), (1, 1), gl.GL_PAD_NEG_INF))
+    assert gl.gl_poll_device_status() == 0
+    # checker: the same chain from the brute-force equations
+    conv = np.maximum(brute.conv2d(x, wt, (1, 1), ((1, 1), (1, 1))), 0.0)
+    ref = brute.maxpool(conv.astype(np.float32), (3, 3), (2, 2), ((1, 1), (1, 1)))
+    assert pooled.tensor.shape == ref.shape
+    assert np.array_equal(pooled.tensor.cpu().numpy(), ref)
+    if n * c * h * w * o < 40000:          # and from the interpreter's programs on the smallest case
+        prog = gi.maxpool_program(gi.compute("relu", gi.conv2d_program(x, wt, (1, 1), ((1, 1), (1, 1)))).data,
+                                  (3, 3), (2, 2), ((1, 1), (1, 1)))
+        assert np.array_equal(prog.data, ref.astype(np.float64))
