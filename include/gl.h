@@ -239,6 +239,12 @@ GL_API int gl_compute_relu(const gl_ap* in, gl_ap* out, void* stream);
  * (that kernel's output is then undefined), GL_ERR_CUDA on a runtime error. */
 GL_API int gl_poll_device_status(void* stream);
 
+/* Failure-path self-test that faults nothing: launches one block that waits, for at most
+ * `limit_ms` (1..1000), on a barrier nothing ever arrives at, using the same bounded wait as the
+ * tensor-core pipeline.  The kernel returns normally; the next gl_poll_device_status() on that
+ * stream must report GL_ERR_TIMEOUT (and clear it). */
+GL_API int gl_selftest_bounded_wait(uint32_t limit_ms, void* stream);
+
 GL_API const char* gl_strerror(int code);
 GL_API int gl_version(void);
 

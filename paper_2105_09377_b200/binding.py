@@ -55,6 +55,7 @@ EXPORTS = [
     "gl_cartesian_dot_static", "gl_shape_cartesian_dot_nchw",
     "gl_shape_slice", "gl_shape_concat", "gl_shape_pair", "gl_shape_squeeze", "gl_shape_reshape",
     "gl_shape_reduce_sum", "gl_access_slice", "gl_access_concat", "gl_access_pair", "gl_compute_reduce_sum",
+    "gl_selftest_bounded_wait",
 ]
 
 
@@ -94,6 +95,7 @@ def _load() -> ctypes.CDLL:
         "gl_compute_reduce_max": [ap, win, ap, vp],
         "gl_compute_relu": [ap, ap, vp],
         "gl_poll_device_status": [vp],
+        "gl_selftest_bounded_wait": [ctypes.c_uint32, vp],
     }
     for name, args in sig.items():
         fn = getattr(lib, name)
@@ -431,6 +433,10 @@ def gl_compute_relu(a: AccessPattern, out: Optional[AccessPattern] = None, strea
 
 def gl_poll_device_status(stream=None) -> int:
     return int(LIB.gl_poll_device_status(_stream(stream)))
+
+
+def gl_selftest_bounded_wait(limit_ms: int, stream=None) -> None:
+    _check(LIB.gl_selftest_bounded_wait(limit_ms, _stream(stream)), "gl_selftest_bounded_wait")
 
 
 def gl_strerror(code: int) -> str:

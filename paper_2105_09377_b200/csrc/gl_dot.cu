@@ -258,14 +258,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait.  Returns false when the block is giving up: either this wait
 // ran out of time (it then raises the block's abort flag and the device status
 // word) or another role of the block already did.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_timer();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++spins & 0xFFu) == 0) {
       if (*abort_flag) return false;
-      if (global_timer() - t0 > kWaitLimitNs) {
+      if (global_timer() - t0 > limit_ns) {
         *abort_flag = 1;
         atomicOr(&g_status, 1u);
         return false;
@@ -700,6 +701,21 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
                  "r"(static_cast<uint32_t>(Cfg::kTmemCols))
                  : "memory");
   }
+}
+
+// One block waits on a barrier that nothing ever arrives at, with the same bounded wait the GEMM
+// pipeline uses: it must give up after `limit_ns`, raise the status word and return normally.
+__global__ void bounded_wait_selftest(uint64_t limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) mbar_wait(smem_u32(&bar), 0, &abort_flag, limit_ns);
+  __syncthreads();
 }
 
 // ------------------------------------------------------------------------
@@ -1181,6 +1197,12 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
   p.kblocks = static_cast<int>((taps * p.cchunks + 7) / 8);
   if (!encode_im2col(&ma, x, d, Cp, 8, false) || !encode_kmajor_granules(&mb, wt, d.O, p.K, bn)) return GL_ERR_CUDA;
   return launch_tc_bn<kIm2colGranule>(bn, ma, mb, dst, p, st);
+}
+
+int gl_selftest_bounded_wait(uint32_t limit_ms, void* stream) {
+  if (limit_ms < 1 || limit_ms > 1000) return GL_ERR_SHAPE;
+  bounded_wait_selftest<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<uint64_t>(limit_ms) * 1000000ull);
+  return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;
 }
 
 int gl_poll_device_status(void* stream) {

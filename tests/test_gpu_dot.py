@@ -303,3 +303,38 @@ def test_full_size_conv_sampled(gl, cfg, layout):
     assert rel_err(got[ns, xs, ys, os_], ref) <= REL_TOL
     # a property that holds at any size: the last image (ragged final tile) is finite and not all zero
     assert np.isfinite(got[-1]).all() and np.abs(got[-1]).max() > 0
+
+
+def test_bounded_wait_reports_timeout_and_context_survives(gl):
+    # a wait that nothing completes gives up after its limit, the status word says so, and the
+    # context keeps working: no trap, no fault, no hang
+    assert gl.gl_poll_device_status() == 0
+    gl.gl_selftest_bounded_wait(20)
+    assert gl.gl_poll_device_status() == 10          # GL_ERR_TIMEOUT
+    assert gl.gl_poll_device_status() == 0           # cleared by the poll
+    a = synth.uniform_int(71, 1, (64, 64), -3, 3)
+    out = gl.gl_cartesian_dot(gl.AccessPattern(to_bf16_device(a), 1), None, gl.AccessPattern(to_bf16_device(a), 1))
+    _ok(gl)
+    assert np.array_equal(out.tensor.cpu().numpy().astype(np.float64), brute.rowdot(a, a))
+    with pytest.raises(gl.GlError):
+        gl.gl_selftest_bounded_wait(5000)
+
+
+def test_workspace_and_flag_errors_launch_nothing(gl):
+    x = to_bf16_device(synth.uniform_int(72, 1, (2, 16, 10, 10), -3, 3))
+    wt = to_bf16_device(synth.uniform_int(72, 2, (8, 16, 3, 3), -3, 3))
+    spec = gl.windows_spec((16, 3, 3), (1, 1, 1), (0, 1, 1), (0, 1, 1))
+    xa, wa = gl.AccessPattern(x, 1), gl.AccessPattern(wt, 1)
+    need = gl.gl_cartesian_dot_workspace(xa, spec, wa)
+    assert need > 0
+    out = gl.output_like(gl.gl_shape_cartesian_dot(tuple(x.shape), 1, spec, tuple(wt.shape), 1), "cuda")
+    out.tensor.fill_(5.0)
+    small = torch.empty(need // 2 + 1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(gl.GlError) as e:
+        gl.gl_cartesian_dot(xa, spec, wa, out=out, workspace=small)
+    assert e.value.code == 8
+    with pytest.raises(gl.GlError) as e:
+        gl.gl_cartesian_dot(xa, spec, wa, out=out, flags=0x40)
+    assert e.value.code == 7
+    torch.cuda.synchronize()
+    assert bool((out.tensor == 5.0).all())
