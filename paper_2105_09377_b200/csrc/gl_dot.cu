@@ -80,7 +80,7 @@ __global__ void __launch_bounds__(256) dot_general(const uint16_t* __restrict__ 
                                                    float* __restrict__ out, const GenA g, int relu) {
   __shared__ float sa[16][64 + 1], sb[16][64 + 1];
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
-  const int64_t m0 = (int64_t)blockIdx.y * 64, o0 = (int64_t)blockIdx.x * 64;
+  const int64_t m0 = (int64_t)blockIdx.x * 64, o0 = (int64_t)blockIdx.y * 64;
   float acc[4][4] = {};
   for (int64_t k0 = 0; k0 < g.K; k0 += 16) {
     for (int e = threadIdx.x; e < 16 * 64; e += 256) {
@@ -753,13 +753,11 @@ const DriverApi& driver_api() {
 }
 
 int num_sms() {
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  }
-  return sms;
+  static int sms[64] = {0};   // per device
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (!sms[dev]) cudaDeviceGetAttribute(&sms[dev], cudaDevAttrMultiProcessorCount, dev);
+  return sms[dev] > 0 ? sms[dev] : 148;
 }
 
 inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -840,7 +838,10 @@ bool encode_rowwin(CUtensorMap* m, const void* base, int64_t rows, int64_t Wo, i
 template <int BN, int MODE, int G, int OCC>
 int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams p, cudaStream_t st) {
   using Cfg = TcCfg<BN, G, OCC>;
-  static bool attr_set = false;   // benign race: the attribute call is idempotent
+  static bool attr_set_dev[64] = {false};   // per device; benign race: the attribute call is idempotent
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return GL_ERR_CUDA;
+  bool& attr_set = attr_set_dev[dev];
   if (!attr_set) {
     if (cudaFuncSetAttribute(dot_tc<BN, MODE, G, OCC>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) !=
         cudaSuccess)
@@ -949,9 +950,9 @@ ConvPlan plan_conv(const DotProblem& d) {
                     d.Kw <= 256 && d.Kh <= 256 && d.Sw <= 8 && d.Sh <= 8 && d.W < (1ll << 30) && d.H < (1ll << 30) &&
                     d.N < (1ll << 30) && d.M < (1ll << 31) && d.O < (1ll << 31) &&
                     d.Kh * d.Kw * pl.Cp < (1ll << 31);
-  pl.tc = fits;
+  pl.tc = fits && ((d.M + 127) / 128) * ((d.O + 63) / 64) < (1ll << 28);
   pl.prepass = !d.channels_last || pl.Cp != d.C;
-  if (fits && pl.Cp < kBK && d.Kw * pl.Cp <= kBK && d.Wo < (1ll << 24) && d.N * (d.H + d.ph_lo + d.ph_hi) < (1ll << 31)) {
+  if (pl.tc && pl.Cp < kBK && d.Kw * pl.Cp <= kBK && d.Wo < (1ll << 24) && d.N * (d.H + d.ph_lo + d.ph_hi) < (1ll << 31)) {
     pl.rowwin = true;
     pl.prepass = true;
     pl.Hp = d.H + d.ph_lo + d.ph_hi;
@@ -976,8 +977,12 @@ bool conv_is_plain_matrix(const DotProblem& d, uint32_t flags) {
          d.ph_hi == 0 && d.pw_lo == 0 && d.pw_hi == 0 && d.C % 8 == 0 && !(flags & GL_OUT_NCHW);
 }
 
+// The kernel counts tiles in 32-bit integers.
+bool tile_count_ok(const DotProblem& d) { return ((d.M + 127) / 128) * ((d.O + 63) / 64) < (1ll << 28); }
+
 bool dense_tc_ok(const DotProblem& d) {
-  return !d.conv && !d.general && d.K % 8 == 0 && d.M < (1ll << 31) && d.O < (1ll << 31) && d.K < (1ll << 31);
+  return !d.conv && !d.general && d.K % 8 == 0 && d.M < (1ll << 31) && d.O < (1ll << 31) && d.K < (1ll << 31) &&
+         tile_count_ok(d);
 }
 
 void fill_general(const gl_ap* a0, const gl_windows* w, const DotProblem& d, GenA* g) {
@@ -1065,7 +1070,7 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     GenA g;
     fill_general(a0, w, d, &g);
     g.out_nchw = out_nchw;
-    const int64_t gx = (d.O + 63) / 64, gy = (d.M + 63) / 64;
+    const int64_t gx = (d.M + 63) / 64, gy = (d.O + 63) / 64;
     if (gy > 65535 || gx > 0x7FFFFFFF) return GL_ERR_UNSUPPORTED;
     dot_general<<<dim3(static_cast<unsigned>(gx), static_cast<unsigned>(gy)), 256, 0, st>>>(pa, pb, dst, g, relu);
     return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;

@@ -708,7 +708,7 @@ void fill_win_params(const gl_ap* in, const gl_windows* w, const gl_ap& A, WinPa
 }
 
 int device_smem_optin() {
-  static int cached = 0;   // same value on every B200 of a node
+  static int cached = 0;   // the same value on every GPU of a node
   if (cached) return cached;
   int dev = 0, v = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return 0;
@@ -759,8 +759,10 @@ int run_windows(const gl_ap* in, const gl_windows* w, const gl_ap& A, gl_ap* out
       p.Wp = static_cast<int>(wp);
       p.pitch = pitch;
       auto kern = vec ? im2col_rows<T, VEC> : im2col_rows<T, 1>;
-      static bool attr_done[2] = {false, false};
-      if (!allow_big_smem(kern, &attr_done[vec ? 1 : 0])) return GL_ERR_CUDA;
+      static bool attr_done[64][2] = {{false}};   // per device and kernel variant
+      int dev = 0;
+      if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return GL_ERR_CUDA;
+      if (!allow_big_smem(kern, &attr_done[dev][vec ? 1 : 0])) return GL_ERR_CUDA;
       kern<<<static_cast<unsigned>(blocks), kThreads, static_cast<size_t>(smem), st>>>(src, dst, p, fill);
       return launch_status();
     }
