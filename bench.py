@@ -258,7 +258,7 @@ def detail_workloads(device, peaks):
         for layout in ("nhwc", "nchw"):
             entry(cfg, layout)
     entry(synth.CONV_SWEEP_3X3[0], "rewritten")   # the materialised im2col form of Section 5.3, for comparison
-    for cfg in (synth.MEM_IM2COL, synth.MEM_TRANSPOSE, synth.MEM_MAXPOOL):
+    for cfg in (synth.MEM_IM2COL, synth.MEM_TRANSPOSE, synth.MEM_MAXPOOL, synth.MEM_RELU, synth.MEM_PAD):
         entry(cfg, "")
     return out
 

@@ -493,6 +493,11 @@ def prepare_compute_reduce_max(a: AccessPattern, w: Optional[GlWindows], out: Ac
     return Prepared(LIB.gl_compute_reduce_max, (ctypes.byref(sa), _wptr(w), ctypes.byref(so)), (sa, so, w, a, out))
 
 
+def prepare_access_pad(a: AccessPattern, dim: int, lo: int, hi: int, pad_kind: int, out: AccessPattern) -> Prepared:
+    sa, so = _struct(a), _struct(out)
+    return Prepared(LIB.gl_access_pad, (ctypes.byref(sa), dim, lo, hi, pad_kind, ctypes.byref(so)), (sa, so, a, out))
+
+
 def prepare_compute_relu(a: AccessPattern, out: AccessPattern) -> Prepared:
     sa, so = _struct(a), _struct(out)
     return Prepared(LIB.gl_compute_relu, (ctypes.byref(sa), ctypes.byref(so)), (sa, so, a, out))

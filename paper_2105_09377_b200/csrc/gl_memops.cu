@@ -253,6 +253,19 @@ __global__ void __launch_bounds__(kThreads) pad_kernel(const V* __restrict__ in,
   }
 }
 
+// pad of the innermost dimension: one warp per row, no divisions.
+template <typename T>
+__global__ void __launch_bounds__(kThreads) pad_rows(const T* __restrict__ in, T* __restrict__ out, int64_t rows,
+                                                     int d_in, int lo, int d_out, T fill) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+  for (int64_t r = blockIdx.x * (int64_t)(blockDim.x >> 5) + (threadIdx.x >> 5); r < rows; r += warps) {
+    const T* src = in + r * d_in - lo;
+    T* dst = out + r * d_out;
+    for (int x = lane; x < d_out; x += 32) dst[x] = (x >= lo && x < lo + d_in) ? src[x] : fill;
+  }
+}
+
 // ------------------------------------------------------------------------
 // windows (materialised) and windows + reduceMax
 // ------------------------------------------------------------------------
@@ -817,6 +830,14 @@ int gl_access_pad(const gl_ap* in, int32_t dim, int64_t lo, int64_t hi, int32_t 
     const int64_t total = outer * d_out * (inner / vec);
     pad_kernel<uint4><<<grid_for(total, kThreads), kThreads, 0, st>>>(
         static_cast<const uint4*>(in->data), static_cast<uint4*>(out->data), outer, d_in, lo, d_out, inner / vec, fill);
+  } else if (inner == 1 && d_out < (1ll << 30)) {
+    const unsigned blocks = static_cast<unsigned>(std::min<int64_t>((outer + 7) / 8, 148 * 32));
+    if (in->dtype == GL_F32)
+      pad_rows<uint32_t><<<blocks, kThreads, 0, st>>>(static_cast<const uint32_t*>(in->data), static_cast<uint32_t*>(out->data),
+                                                      outer, (int)d_in, (int)lo, (int)d_out, Fill<uint32_t>::value(pad_kind));
+    else
+      pad_rows<uint16_t><<<blocks, kThreads, 0, st>>>(static_cast<const uint16_t*>(in->data), static_cast<uint16_t*>(out->data),
+                                                      outer, (int)d_in, (int)lo, (int)d_out, Fill<uint16_t>::value(pad_kind));
   } else if (in->dtype == GL_F32) {
     pad_kernel<uint32_t><<<grid_for(outer * d_out * inner, kThreads), kThreads, 0, st>>>(
         static_cast<const uint32_t*>(in->data), static_cast<uint32_t*>(out->data), outer, d_in, lo, d_out, inner,

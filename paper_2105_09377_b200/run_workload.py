@@ -29,7 +29,8 @@ def _inputs(cfg, seed):
 
 def workloads():
     table = {c.name: c for c in (synth.CONV_TINY,) + synth.CONV_SWEEP_3X3 + synth.CONV_STRIDED_1X1}
-    table.update({c.name: c for c in (synth.MEM_IM2COL, synth.MEM_TRANSPOSE, synth.MEM_MAXPOOL)})
+    table.update({c.name: c for c in (synth.MEM_IM2COL, synth.MEM_TRANSPOSE, synth.MEM_MAXPOOL, synth.MEM_RELU,
+                                      synth.MEM_PAD)})
     table[synth.DENSE_4096.name] = synth.DENSE_4096
     return table
 
@@ -76,6 +77,12 @@ def build_call(cfg, layout: str, device, batch=None, flags=0):
     if cfg.kind == "transpose":
         out = gl.output_like(gl.gl_shape_transpose(cfg.shape, 1, cfg.perm), device)
         return gl.prepare_access_transpose(gl.AccessPattern(x, 1), cfg.perm, out), 0.0, cfg.algorithmic_bytes
+    if cfg.kind == "relu":
+        a = gl.AccessPattern(x, 4)
+        return gl.prepare_compute_relu(a, gl.AccessPattern(torch.empty_like(x), 4)), 0.0, cfg.algorithmic_bytes
+    if cfg.kind == "pad":
+        out = gl.output_like(gl.gl_shape_pad(cfg.shape, 1, 3, cfg.pad, cfg.pad), device)
+        return gl.prepare_access_pad(gl.AccessPattern(x, 1), 3, cfg.pad, cfg.pad, gl.GL_PAD_ZERO, out), 0.0, cfg.algorithmic_bytes
     if cfg.kind == "im2col":
         c = cfg.shape[1]
         spec = gl.windows_spec((c,) + cfg.window, (1, cfg.stride, cfg.stride), (0, cfg.pad, cfg.pad), (0, cfg.pad, cfg.pad))

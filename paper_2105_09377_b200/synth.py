@@ -177,7 +177,7 @@ DENSE_4096 = DenseCase("dense_4096x4096x4096_relu", 4096, 4096, 4096)
 @dataclass(frozen=True)
 class MemCase:
     name: str
-    kind: str                 # "im2col" | "transpose" | "maxpool"
+    kind: str                 # "im2col" | "transpose" | "maxpool" | "relu" | "pad"
     shape: tuple              # NCHW
     window: tuple = ()
     stride: int = 1
@@ -197,8 +197,10 @@ class MemCase:
     def algorithmic_bytes(self):
         n, c, h, w = self.shape
         src = 4 * n * c * h * w
-        if self.kind == "transpose":
+        if self.kind in ("transpose", "relu"):
             return 2 * src
+        if self.kind == "pad":        # one border cell on each side of the last dimension
+            return src + 4 * n * c * h * (w + 2 * self.pad)
         ho, wo = self.out_hw
         if self.kind == "im2col":
             return src + 4 * n * ho * wo * c * self.window[0] * self.window[1]
@@ -207,6 +209,8 @@ class MemCase:
 
 MEM_IM2COL = MemCase("im2col_32x64x56x56_k3p1", "im2col", (32, 64, 56, 56), (3, 3), 1, 1)
 MEM_TRANSPOSE = MemCase("transpose_nchw_nhwc_32x256x56x56", "transpose", (32, 256, 56, 56), perm=(0, 2, 3, 1))
+MEM_RELU = MemCase("relu_4096x4096", "relu", (1, 1, 4096, 4096))
+MEM_PAD = MemCase("pad_w1_32x64x56x56", "pad", (32, 64, 56, 56), pad=1)
 MEM_MAXPOOL = MemCase("maxpool3x3s2p1_32x64x112x112", "maxpool", (32, 64, 112, 112), (3, 3), 2, 1)
 
 
