@@ -299,6 +299,42 @@ __device__ __forceinline__ void tma_load_im2col(uint32_t dst, const CUtensorMap*
       : "memory");
 }
 
+// ---- two-block clusters (CTA pairs): one tcgen05.mma spans the tensor cores and the shared
+// memory of both blocks of a pair; barriers that both blocks feed live in the pair's first block.
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of `saddr` (a shared::cta address of this block) in block `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// Pair forms of the loads: the data lands in this block, the bytes are counted on a barrier that
+// may sit in the other block of the pair (`bar` is a shared::cluster address).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_im2col_pair(uint32_t dst, const CUtensorMap* map, int c, int w, int h, int n,
+                                                     uint16_t kw, uint16_t kh, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.im2col.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%2, %3, %4, %5}], [%6], {%7, %8};"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar), "h"(kw), "h"(kh)
+      : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -313,6 +349,25 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uin
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// Pair forms: issued by one thread of the pair's first block; the commit arrives at the barrier
+// at the same offset in both blocks.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"(static_cast<uint16_t>(3))
+      : "memory");
+}
+// D (256 rows: 128 TMEM lanes in each block) (+)= A (128 rows from each block) * B^T (N/2 rows from each block)
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
@@ -403,10 +458,12 @@ struct TcParams {
 
 // A stage holds G K-blocks of 64 (G A sub-tiles, then G B sub-tiles) behind one pair of barriers.
 // OCC = blocks per SM the configuration is sized for (2 only for BN <= 128: TMEM has 512 columns).
-template <int BN, int G, int OCC>
+// CTAS = 2: two blocks on neighbouring SMs (a cluster) share one 256 x BN tile; each stages its own
+// 128 rows of A and BN/2 rows of B, and one thread of the first block issues MMAs that span both.
+template <int BN, int G, int OCC, int CTAS = 1>
 struct TcCfg {
   static constexpr int kStageA = kBM * kBK * 2;
-  static constexpr int kStageB = BN * kBK * 2;
+  static constexpr int kStageB = (BN / CTAS) * kBK * 2;
   static constexpr int kStage = G * (kStageA + kStageB);
   static constexpr int kEpiBufs = OCC == 2 ? 1 : 2;          // 32x32 fp32 staging tiles per epilogue warp
   static constexpr int kEpiBytes = 4 * kEpiBufs * 4096;
@@ -416,11 +473,12 @@ struct TcCfg {
   static constexpr int kSmemBytes = kStages * kStage + kEpiBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
-template <int BN, int MODE, int G, int OCC>
+template <int BN, int MODE, int G, int OCC, int CTAS>
 __global__ void __launch_bounds__(kTcThreads, OCC)
 dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
        const __grid_constant__ CUtensorMap map_c, float* __restrict__ out, const TcParams p) {
-  using Cfg = TcCfg<BN, G, OCC>;
+  using Cfg = TcCfg<BN, G, OCC, CTAS>;
+  static_assert(CTAS == 1 || (CTAS == 2 && (MODE == kDense || MODE == kIm2col)), "pairs: dense and im2col tiles only");
   static_assert(Cfg::kStages >= 2, "ring too shallow");
   extern __shared__ unsigned char smem_raw[];
   // operand tiles need 1024-byte alignment for the 128-byte swizzle
@@ -437,26 +495,38 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // position in the pair: block 0 owns the barriers both blocks feed and issues the MMAs
+  const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;
 
   if (threadIdx.x == 0) {
+    // full: the two producer threads of block 0 announce the bytes of the whole pair
     for (int s = 0; s < Cfg::kStages; ++s) { mbar_init(bar_full + 8 * s, 2); mbar_init(bar_empty + 8 * s, 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, 4 * CTAS); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(static_cast<uint32_t>(Cfg::kTmemCols))
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (CTAS == 2) {   // the same warp of both blocks allocates the same columns in both tensor memories
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"(static_cast<uint32_t>(Cfg::kTmemCols))
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"(static_cast<uint32_t>(Cfg::kTmemCols))
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
-  __syncthreads();
+  if (CTAS == 2) cluster_sync_all();   // the other block's barriers exist before anything signals them
+  else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  const int num_tiles = p.tiles_m * p.tiles_n * p.ksplit;   // work units
+  const int num_tiles = p.tiles_m * p.tiles_n * p.ksplit;   // work units (p.tiles_m counts 128*CTAS-row tiles)
+  const int unit0 = static_cast<int>(blockIdx.x) / CTAS, unit_step = static_cast<int>(gridDim.x) / CTAS;
 
   if (warp == 0 || warp == 6) {
     // ---------------- TMA producers: warp 0 stages A, warp 6 stages B ----------------
@@ -466,12 +536,14 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
       asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(load_a ? &map_a : &map_b)) : "memory");
       uint32_t s = 0, ph = 0;   // ring slot and its phase, advanced by hand (no division in this thread)
       bool ok = true;
-      for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x) {
+      for (int u = unit0; u < num_tiles && ok; u += unit_step) {
         uint32_t t, ks, tm, tn;
         p.div_ksplit.divmod(static_cast<uint32_t>(u), t, ks);
         p.div_tiles_n.divmod(t, tm, tn);
         const int kb_begin = static_cast<int>(ks) * p.kper, kb_end = min(p.kblocks, kb_begin + p.kper);
-        const int m0 = static_cast<int>(tm) * kBM, n0 = static_cast<int>(tn) * BN;
+        // this block's 128 rows of A and its BN/CTAS rows of B
+        const int m0 = (static_cast<int>(tm) * CTAS + static_cast<int>(rank)) * kBM;
+        const int n0 = static_cast<int>(tn) * BN + static_cast<int>(rank) * (BN / CTAS);
         int wbase = 0, hbase = 0, img = 0;
         if (MODE == kRowWin) {
           if (load_a) {   // tile -> (output row, segment) -> first padded input row
@@ -499,15 +571,27 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
         }
         for (int kb0 = kb_begin; kb0 < kb_end; kb0 += G) {
           if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
-          const uint32_t full = bar_full + 8 * s;
+          const uint32_t full = CTAS == 2 ? map_to_cta(bar_full + 8 * s, 0) : bar_full + 8 * s;
           const uint32_t stage = tiles + s * Cfg::kStage;
           const int nsub = min(G, kb_end - kb0);
-          mbar_expect_tx(full, nsub * (load_a ? Cfg::kStageA : Cfg::kStageB));
+          if (rank == 0) mbar_expect_tx(bar_full + 8 * s, nsub * CTAS * (load_a ? Cfg::kStageA : Cfg::kStageB));
 #pragma unroll 1
           for (int j = 0; j < nsub; ++j) {
             const int kb = kb0 + j;
             const uint32_t sa = stage + j * Cfg::kStageA, sb = stage + G * Cfg::kStageA + j * Cfg::kStageB;
-            if (MODE == kDense) {
+            if (CTAS == 2) {
+              if (MODE == kDense) {
+                if (load_a) tma_load_2d_pair(sa, &map_a, kb * kBK, m0, full);
+                else tma_load_2d_pair(sb, &map_b, kb * kBK, n0, full);
+              } else {
+                if (load_a)
+                  tma_load_im2col_pair(sa, &map_a, cc * kBK, wbase, hbase, img, static_cast<uint16_t>(kw),
+                                       static_cast<uint16_t>(kh), full);
+                else
+                  tma_load_2d_pair(sb, &map_b, (kh * p.Kw + kw) * p.Cp + cc * kBK, n0, full);
+                if (++cc == p.cchunks) { cc = 0; if (++kw == p.Kw) { kw = 0; ++kh; } }
+              }
+            } else if (MODE == kDense) {
               if (load_a) tma_load_2d(sa, &map_a, kb * kBK, m0, full);
               else tma_load_2d(sb, &map_b, kb * kBK, n0, full);
             } else if (MODE == kRowWin) {
@@ -544,14 +628,14 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc(kBM, BN);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = make_idesc(kBM * CTAS, BN);
       const uint64_t desc_a0 = (MODE == kIm2colGranule) ? make_desc(tiles, kBM * 16, 128, 0) : make_desc(tiles, 16, 1024, 2);
       const uint64_t desc_b0 = (MODE == kIm2colGranule) ? make_desc(tiles + G * Cfg::kStageA, BN * 16, 128, 0)
                                                         : make_desc(tiles + G * Cfg::kStageA, 16, 1024, 2);
       uint32_t s = 0, ph = 0, tile_it = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x, ++tile_it) {
+      for (int u = unit0; u < num_tiles && ok; u += unit_step, ++tile_it) {
         const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
         uint32_t t, ks;
         p.div_ksplit.divmod(static_cast<uint32_t>(u), t, ks);
@@ -573,17 +657,24 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
               for (int k = 0; k < kBK / 16; ++k) {
                 constexpr int kStepA = (MODE == kIm2colGranule) ? 2 * (kBM * 16) : 32;
                 constexpr int kStepB = (MODE == kIm2colGranule) ? 2 * (BN * 16) : 32;
-                tc_mma_bf16(d_tmem, da0 + ((j * Cfg::kStageA + k * kStepA) >> 4),
-                            db0 + ((j * Cfg::kStageB + k * kStepB) >> 4), idesc, ((kb0 - kb_begin) | j | k) != 0 ? 1u : 0u);
+                const uint64_t da = da0 + ((j * Cfg::kStageA + k * kStepA) >> 4);
+                const uint64_t db = db0 + ((j * Cfg::kStageB + k * kStepB) >> 4);
+                const uint32_t accumulate = ((kb0 - kb_begin) | j | k) != 0 ? 1u : 0u;
+                if (CTAS == 2) tc_mma_bf16_pair(d_tmem, da, db, idesc, accumulate);
+                else tc_mma_bf16(d_tmem, da, db, idesc, accumulate);
               }
             }
           }
           // one commit per stage (it costs the issuing thread a few hundred cycles): frees the
           // stage once these MMAs have read it
-          tc_commit(bar_empty + 8 * s);
+          if (CTAS == 2) tc_commit_pair(bar_empty + 8 * s);
+          else tc_commit(bar_empty + 8 * s);
           if (++s == Cfg::kStages) { s = 0; ph ^= 1u; }
         }
-        if (ok) tc_commit(bar_tfull + 8 * acc);
+        if (ok) {
+          if (CTAS == 2) tc_commit_pair(bar_tfull + 8 * acc);
+          else tc_commit(bar_tfull + 8 * acc);
+        }
       }
     }
   } else {
@@ -594,11 +685,12 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
     const bool vec_ok = (p.O & 3) == 0;
     const uint32_t stage_buf = epi_base + q * (Cfg::kEpiBufs * 4096);   // this warp's 32 rows x 128 bytes tiles
     if (p.tma_store && lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_c)) : "memory");
-    for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x, ++tile_it) {
+    for (int u = unit0; u < num_tiles && ok; u += unit_step, ++tile_it) {
       const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
       uint32_t t, ks, tmu, tnu;
       p.div_ksplit.divmod(static_cast<uint32_t>(u), t, ks);
       p.div_tiles_n.divmod(t, tmu, tnu);
+      if (CTAS == 2) tmu = tmu * CTAS + rank;   // this block's 128 rows of the pair's tile
       const int tm = static_cast<int>(tmu), tn = static_cast<int>(tnu);
       if (!mbar_wait(bar_tfull + 8 * acc, aph, abort_flag)) { ok = false; break; }
       tc_fence_after();
@@ -660,7 +752,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
                            "r"(static_cast<int>(n0)), "r"(static_cast<int>(oseg) * kBM + q * 32),
                            "r"(static_cast<int>(orow)), "r"(buf)
                            : "memory");
-            else   // (planes, M, O): plane = K-split index, 0 without a split
+            else if (CTAS == 1 || tm * kBM + q * 32 < p.M)   // (planes, M, O): plane = K-split index, 0 without a split
               asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(
                                reinterpret_cast<uint64_t>(&map_c)),
                            "r"(static_cast<int>(n0)), "r"(tm * kBM + q * 32), "r"(static_cast<int>(ks)), "r"(buf)
@@ -682,7 +774,10 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+      if (lane == 0) {
+        if (CTAS == 2) mbar_arrive_cluster(map_to_cta(bar_tempty + 8 * acc, 0));
+        else mbar_arrive(bar_tempty + 8 * acc);
+      }
     }
     if (p.tma_store && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
@@ -694,12 +789,18 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
     while (global_timer() - t0 < 20000000ull) { }
   }
   tc_fence_before();
-  __syncthreads();
+  if (CTAS == 2) cluster_sync_all();   // neither block leaves while the other may still signal it or read its tiles
+  else __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
-                 "r"(static_cast<uint32_t>(Cfg::kTmemCols))
-                 : "memory");
+    if (CTAS == 2)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                   "r"(static_cast<uint32_t>(Cfg::kTmemCols))
+                   : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                   "r"(static_cast<uint32_t>(Cfg::kTmemCols))
+                   : "memory");
   }
 }
 
@@ -835,17 +936,39 @@ bool encode_rowwin(CUtensorMap* m, const void* base, int64_t rows, int64_t Wo, i
                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int MODE, int G, int OCC>
+template <int BN, int MODE, int G, int OCC, int CTAS = 1>
 int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams p, cudaStream_t st) {
-  using Cfg = TcCfg<BN, G, OCC>;
+  using Cfg = TcCfg<BN, G, OCC, CTAS>;
   static bool attr_set_dev[64] = {false};   // per device; benign race: the attribute call is idempotent
+  static int max_pairs_dev[64] = {0};       // CTAS == 2: pairs that can be resident at once
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return GL_ERR_CUDA;
   bool& attr_set = attr_set_dev[dev];
+  cudaLaunchConfig_t cfg;
+  std::memset(&cfg, 0, sizeof(cfg));
+  cudaLaunchAttribute cluster_attr;
+  std::memset(&cluster_attr, 0, sizeof(cluster_attr));
+  cluster_attr.id = cudaLaunchAttributeClusterDimension;
+  cluster_attr.val.clusterDim.x = CTAS;
+  cluster_attr.val.clusterDim.y = 1;
+  cluster_attr.val.clusterDim.z = 1;
+  cfg.blockDim = dim3(kTcThreads);
+  cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+  cfg.stream = st;
+  cfg.attrs = &cluster_attr;
+  cfg.numAttrs = CTAS == 2 ? 1 : 0;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(dot_tc<BN, MODE, G, OCC>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) !=
-        cudaSuccess)
+    if (cudaFuncSetAttribute(dot_tc<BN, MODE, G, OCC, CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Cfg::kSmemBytes) != cudaSuccess)
       return GL_ERR_CUDA;
+    if (CTAS == 2) {
+      // a persistent grid must not exceed what is resident at once (SMs pair up within a GPC)
+      cfg.gridDim = dim3(static_cast<unsigned>(num_sms() / 2 * 2));
+      int pairs = 0;
+      if (cudaOccupancyMaxActiveClusters(&pairs, dot_tc<BN, MODE, G, OCC, CTAS>, &cfg) != cudaSuccess || pairs < 1)
+        return GL_ERR_CUDA;
+      max_pairs_dev[dev] = pairs;
+    }
     attr_set = true;
   }
   if (p.ksplit < 1) { p.ksplit = 1; p.kper = p.kblocks; }
@@ -866,16 +989,34 @@ int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams
     mc = ma;   // unused by the kernel; any valid map
   }
   const int tiles = p.tiles_m * p.tiles_n * p.ksplit;
+  if (CTAS == 2) {
+    const int pairs = std::min(tiles, std::min(max_pairs_dev[dev], num_sms() / 2));
+    cfg.gridDim = dim3(static_cast<unsigned>(2 * pairs));
+    if (cudaLaunchKernelEx(&cfg, dot_tc<BN, MODE, G, OCC, CTAS>, ma, mb, mc, out, p) != cudaSuccess) return GL_ERR_CUDA;
+    return GL_OK;
+  }
   const int grid = tiles < OCC * num_sms() ? tiles : OCC * num_sms();
-  dot_tc<BN, MODE, G, OCC><<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(ma, mb, mc, out, p);
+  dot_tc<BN, MODE, G, OCC, 1><<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(ma, mb, mc, out, p);
   return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+}
+
+// Wide tiles of a large problem are bound by operand traffic from L2 to the SMs; a pair of blocks
+// sharing a 256x256 tile loads a third less per flop.  (The B tensor map then has boxes of bn/2 rows.)
+bool use_pair(int mode, int bn, const TcParams& p) {
+  return bn == 256 && (mode == kDense || mode == kIm2col) && p.ksplit <= 1 && p.tiles_m >= 2;
 }
 
 template <int MODE>
 int launch_tc_bn(int bn, const CUtensorMap& ma, const CUtensorMap& mb, float* out, const TcParams& p,
                  cudaStream_t st) {
   switch (bn) {
-    case 256: return launch_tc<256, MODE, 1, 1>(ma, mb, out, p, st);
+    case 256:
+      if (use_pair(MODE, bn, p)) {
+        TcParams pp = p;
+        pp.tiles_m = (p.tiles_m + 1) / 2;
+        return launch_tc<256, (MODE == kDense || MODE == kIm2col) ? MODE : kDense, 1, 1, 2>(ma, mb, out, pp, st);
+      }
+      return launch_tc<256, MODE, 1, 1>(ma, mb, out, p, st);
     // narrower tiles are bound by the MMA-issuing thread (about 50 cycles per MMA, 250 per commit):
     // 128 wide: two K blocks per stage halve the commits; 64 wide: two blocks per SM interleave
     // their issue threads (measured on the 3x3 and 1x1 convolution shapes)
@@ -1112,7 +1253,9 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
   if (!d.conv) {
     p.K = d.K;
     p.kblocks = static_cast<int>((d.K + kBK - 1) / kBK);
-    if (!encode_kmajor_sw128(&ma, pa, d.M, d.K, kBM) || !encode_kmajor_sw128(&mb, pb, d.O, d.K, bn)) return GL_ERR_CUDA;
+    if (!encode_kmajor_sw128(&ma, pa, d.M, d.K, kBM) ||
+        !encode_kmajor_sw128(&mb, pb, d.O, d.K, use_pair(kDense, bn, p) ? bn / 2 : bn))
+      return GL_ERR_CUDA;
     return finish(launch_tc_bn<kDense>(bn, ma, mb, dst, p, st));
   }
 
@@ -1195,7 +1338,9 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
   if (Cp >= kBK) {
     p.cchunks = static_cast<int>((Cp + kBK - 1) / kBK);
     p.kblocks = static_cast<int>(taps) * p.cchunks;
-    if (!encode_im2col(&ma, x, d, Cp, kBK, true) || !encode_kmajor_sw128(&mb, wt, d.O, p.K, bn)) return GL_ERR_CUDA;
+    if (!encode_im2col(&ma, x, d, Cp, kBK, true) ||
+        !encode_kmajor_sw128(&mb, wt, d.O, p.K, use_pair(kIm2col, bn, p) ? bn / 2 : bn))
+      return GL_ERR_CUDA;
     return finish(launch_tc_bn<kIm2col>(bn, ma, mb, dst, p, st));
   }
   p.cchunks = static_cast<int>(Cp / 8);

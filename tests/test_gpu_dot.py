@@ -241,6 +241,40 @@ def test_dense_integer_bit_exact(gl, m, o, k):
         assert np.array_equal(out.tensor.cpu().numpy().astype(np.float64), ref)
 
 
+# Problems large enough for 256-wide tiles, which run on pairs of blocks sharing a 256x256 tile:
+# an odd number of 128-row tiles (the last pair has an empty half), ragged edges in both directions.
+DENSE_PAIRED = [(2600, 1930, 200), (4001, 1100, 136), (2305, 2309, 72)]
+
+
+@pytest.mark.parametrize("m,o,k", DENSE_PAIRED)
+def test_dense_paired_tiles_bit_exact(gl, m, o, k):
+    a = synth.uniform_int(37, 1, (m, k), -3, 3)
+    b = synth.uniform_int(37, 2, (o, k), -3, 3)
+    ref = brute.rowdot(a, b)
+    aa, bb = gl.AccessPattern(to_bf16_device(a), 1), gl.AccessPattern(to_bf16_device(b), 1)
+    sentinel = torch.full((m + 8, o), -7.0, device="cuda")     # rows around the result must stay untouched
+    out = gl.AccessPattern(sentinel[4:m + 4], 2)
+    for flags in (0, gl.GL_EPILOGUE_RELU):
+        sentinel.fill_(-7.0)
+        gl.gl_cartesian_dot(aa, None, bb, out=out, flags=flags)
+        _ok(gl)
+        want = np.maximum(ref, 0.0) if flags else ref
+        assert np.array_equal(sentinel[4:m + 4].cpu().numpy().astype(np.float64), want)
+        assert bool((sentinel[:4] == -7.0).all()) and bool((sentinel[m + 4:] == -7.0).all())
+
+
+def test_conv_paired_tiles_bit_exact(gl):
+    # 161 row tiles x one 256-wide column tile: the im2col loads of both blocks of a pair
+    n, c, h, w, o = 5, 64, 64, 64, 200
+    x = synth.uniform_int(38, 1, (n, c, h, w), -3, 3)
+    wt = synth.uniform_int(38, 2, (o, c, 3, 3), -3, 3)
+    ref = _conv_ref(x, wt, (1, 1), (1, 1))
+    got = _conv_gpu(gl, x, wt, (1, 1), (1, 1), channels_last=True)
+    assert np.array_equal(got.astype(np.float64), ref)
+    got = _conv_gpu(gl, x, wt, (1, 1), (1, 1), channels_last=True, flags=gl.GL_EPILOGUE_RELU)
+    assert np.array_equal(got.astype(np.float64), np.maximum(ref, 0.0))
+
+
 def test_dense_interpreter_program_with_relu(gl):
     a = synth.uniform_int(32, 1, (20, 16), -3, 3)
     b = synth.uniform_int(32, 2, (12, 16), -3, 3)
