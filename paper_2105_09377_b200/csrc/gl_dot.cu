@@ -804,6 +804,256 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
   }
 }
 
+// ------------------------------------------------------------------------
+// Stride-1 convolutions with the input window tile resident in shared memory
+// ------------------------------------------------------------------------
+//
+// windows (Section 4.2) of a stride-1 convolution overlap: neighbouring filter taps read the same
+// input pixels one position apart.  With one 128-byte shared-memory row per pixel (64 channels),
+// a tile of R output rows of one image needs the (R + Kh - 1) x Wb block of input pixels around it
+// (Wb = W plus the horizontal padding), loaded ONCE by a tiled TMA box whose out-of-range cells
+// read as zeros (the pad).  Number the tile's outputs m = oh * Wb + ow, i.e. in the pitch of the
+// input block: the A operand of filter tap (kh, kw) is then the run of 128 shared-memory rows that
+// starts kh * Wb + kw rows further down - the same bytes, another start address in the matrix
+// descriptor (the 128-byte swizzle is a function of the shared-memory address, so a start on any
+// row is consistent with what the TMA unit wrote).  Outputs with ow >= Wo are computed and dropped.
+// Per tile the activations cross L2 -> SM once instead of Kh*Kw times.
+
+constexpr int kHaloARows = 256;                     // shared-memory rows (pixels) per A stage
+constexpr int kHaloAStage = kHaloARows * 128;
+constexpr int kHaloMaxStages = 16;
+constexpr int kHaloEpiBytes = 4 * 4096;             // one 32x32 fp32 staging tile per epilogue warp
+constexpr int kHaloBarBytes = 640;
+constexpr int kHaloSmemBudget = 232448 - 1024 - kHaloBarBytes - kHaloEpiBytes;
+
+struct HaloParams {
+  int64_t O;
+  int relu;
+  int Ho, Wo, Wb, R, tiles_m, tiles_n;
+  int Kh, Kw, Cp, cchunks;
+  int tg, groups_per_chunk;                 // a B stage holds tg consecutive taps (a filter row, or one tap) of one chunk
+  int ph, pw;
+  int sa_stages, sb_stages, b_resident;     // b_resident: every B stage is loaded once per block and kept
+  uint32_t a_bytes, b_bytes;                // bytes of one input box (64 channels); of one B stage
+  FastDiv div_tiles_n, div_tpi, div_wb;     // tiles per image; padded width
+};
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c, int w, int h, int n,
+                                            uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar)
+      : "memory");
+}
+
+// BN: output channels per tile.  The weights are viewed as (64 channels, O, chunk, tap); one TMA box
+// brings the BN x 64 slices of p.tg consecutive taps of one chunk.
+template <int BN>
+__global__ void __launch_bounds__(kTcThreads, 1)
+conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+          float* __restrict__ out, const HaloParams p) {
+  constexpr int kSubB = BN * kBK * 2;       // one tap of B
+  constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;
+  const uint32_t kStageB = p.b_bytes;
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* gen = smem_raw + (base - raw);
+  const uint32_t a_base = base;
+  const uint32_t b_base = a_base + p.sa_stages * kHaloAStage;
+  const uint32_t epi_base = b_base + p.sb_stages * kStageB;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + (epi_base - base) + kHaloEpiBytes);
+  const uint32_t bar_afull = smem_u32(bars);
+  const uint32_t bar_aempty = bar_afull + 8 * kHaloMaxStages;
+  const uint32_t bar_bfull = bar_aempty + 8 * kHaloMaxStages;
+  const uint32_t bar_bempty = bar_bfull + 8 * kHaloMaxStages;
+  const uint32_t bar_tfull = bar_bempty + 8 * kHaloMaxStages;
+  const uint32_t bar_tempty = bar_tfull + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4 * kHaloMaxStages + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  static_assert((4 * kHaloMaxStages + 4) * 8 + 8 <= kHaloBarBytes, "barrier block too small");
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.sa_stages; ++s) { mbar_init(bar_afull + 8 * s, 1); mbar_init(bar_aempty + 8 * s, 1); }
+    for (int s = 0; s < p.sb_stages; ++s) { mbar_init(bar_bfull + 8 * s, 1); mbar_init(bar_bempty + 8 * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(static_cast<uint32_t>(kTmemCols))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int num_tiles = p.tiles_m * p.tiles_n;
+
+  if (warp == 0) {
+    // ---------------- A producer: one input box per (tile, 64-channel chunk) ----------------
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+      uint32_t s = 0, ph = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x) {
+        uint32_t tm, tn, img, ti;
+        p.div_tiles_n.divmod(static_cast<uint32_t>(u), tm, tn);
+        p.div_tpi.divmod(tm, img, ti);
+        const int h0 = static_cast<int>(ti) * p.R - p.ph;
+        for (int cc = 0; cc < p.cchunks; ++cc) {
+          if (!mbar_wait(bar_aempty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+          mbar_expect_tx(bar_afull + 8 * s, p.a_bytes);
+          tma_load_4d(a_base + s * kHaloAStage, &map_a, cc * kBK, -p.pw, h0, static_cast<int>(img), bar_afull + 8 * s);
+          if (++s == static_cast<uint32_t>(p.sa_stages)) { s = 0; ph ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 6) {
+    // ---------------- B producer: stages in (chunk, tap group) order; once per block when resident ----------------
+    if (lane == 0) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+      uint32_t s = 0, ph = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x) {
+        const int n0 = static_cast<int>(static_cast<uint32_t>(u) - p.div_tiles_n.div(static_cast<uint32_t>(u)) * p.tiles_n) * BN;
+        for (int cc = 0; cc < p.cchunks && ok; ++cc) {
+          for (int g = 0; g < p.groups_per_chunk; ++g) {
+            if (!p.b_resident && !mbar_wait(bar_bempty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
+            mbar_expect_tx(bar_bfull + 8 * s, p.b_bytes);
+            tma_load_4d(b_base + s * kStageB, &map_b, 0, n0, cc, g * p.tg, bar_bfull + 8 * s);
+            if (++s == static_cast<uint32_t>(p.sb_stages)) { s = 0; ph ^= 1u; }
+          }
+        }
+        if (p.b_resident) break;   // the weights stay where they are for every further tile
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    // One thread issues everything, so the loop is kept to the bare sequence: per chunk one wait for the
+    // input box, per B stage one wait, p.tg * 4 MMAs whose descriptors advance by constants, one commit.
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(kBM, BN);
+      const uint64_t desc_a0 = make_desc(a_base, 16, 1024, 2);
+      const uint64_t desc_b0 = make_desc(b_base, 16, 1024, 2);
+      const uint32_t row_step = static_cast<uint32_t>(p.Wb * 128) >> 4;          // next filter row
+      uint32_t sa = 0, pha = 0, sb = 0, phb = 0, tile_it = 0;
+      bool ok = true;
+      for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x, ++tile_it) {
+        const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
+        if (!mbar_wait(bar_tempty + 8 * acc, aph ^ 1u, abort_flag)) { ok = false; break; }
+        const uint32_t d_tmem = tmem_base + acc * BN;
+        const bool wait_b = !p.b_resident || tile_it == 0;
+        uint32_t accumulate = 0;
+        for (int cc = 0; cc < p.cchunks && ok; ++cc) {
+          if (!mbar_wait(bar_afull + 8 * sa, pha, abort_flag)) { ok = false; break; }
+          // tap (kh, kw) reads the box from row kh * Wb + kw on: the group start advances by a filter
+          // row (tg = Kw) or, with one tap per group, by one pixel with a jump at the end of a row
+          uint64_t da_grp = desc_a0 + ((sa * static_cast<uint32_t>(kHaloAStage)) >> 4);
+          int kw = 0;
+          for (int g = 0; g < p.groups_per_chunk; ++g) {
+            if (wait_b && !mbar_wait(bar_bfull + 8 * sb, phb, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            uint64_t da = da_grp, db = desc_b0 + ((sb * kStageB) >> 4);
+#pragma unroll 1
+            for (int t = 0; t < p.tg; ++t, da += 8, db += (kSubB >> 4)) {
+              tc_mma_bf16(d_tmem, da, db, idesc, accumulate);
+              tc_mma_bf16(d_tmem, da + 2, db + 2, idesc, 1u);
+              tc_mma_bf16(d_tmem, da + 4, db + 4, idesc, 1u);
+              tc_mma_bf16(d_tmem, da + 6, db + 6, idesc, 1u);
+              accumulate = 1u;
+            }
+            if (!p.b_resident) tc_commit(bar_bempty + 8 * sb);
+            if (++sb == static_cast<uint32_t>(p.sb_stages)) { sb = 0; phb ^= 1u; }
+            if (p.tg == p.Kw) da_grp += row_step;
+            else { da_grp += 8; if (++kw == p.Kw) { kw = 0; da_grp += row_step - 8u * p.Kw; } }
+          }
+          tc_commit(bar_aempty + 8 * sa);   // the box may be overwritten once these MMAs retire
+          if (++sa == static_cast<uint32_t>(p.sa_stages)) { sa = 0; pha ^= 1u; }
+        }
+        if (ok) tc_commit(bar_tfull + 8 * acc);
+      }
+    }
+  } else {
+    // ---------------- epilogue: TMEM -> registers -> staged 32x32 blocks -> row-predicated global stores ----------------
+    const int q = warp & 3;
+    uint32_t tile_it = 0;
+    bool ok = true;
+    const uint32_t buf = epi_base + q * 4096;
+    const int sub_row = lane >> 3, piece = lane & 7;
+    for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x, ++tile_it) {
+      const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
+      uint32_t tm, tn, img, ti;
+      p.div_tiles_n.divmod(static_cast<uint32_t>(u), tm, tn);
+      p.div_tpi.divmod(tm, img, ti);
+      const int h0 = static_cast<int>(ti) * p.R;
+      // the eight rows this lane stores (one per pass): offset of out[(img, h0 + oh, ow), 0], or -1 for a dropped row
+      int64_t row_off[8];
+#pragma unroll
+      for (int it = 0; it < 8; ++it) {
+        const uint32_t m = static_cast<uint32_t>(q * 32 + it * 4 + sub_row);
+        uint32_t oh, ow;
+        p.div_wb.divmod(m, oh, ow);
+        const bool valid = static_cast<int>(oh) < p.R && h0 + static_cast<int>(oh) < p.Ho && static_cast<int>(ow) < p.Wo;
+        row_off[it] = valid ? ((static_cast<int64_t>(img) * p.Ho + h0 + oh) * p.Wo + ow) * p.O : -1;
+      }
+      if (!mbar_wait(bar_tfull + 8 * acc, aph, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+#pragma unroll 1
+      for (int c = 0; c < BN; c += 32) {
+        const int64_t n0 = static_cast<int64_t>(tn) * BN + c;
+        if (n0 >= p.O) break;   // uniform across the warp
+        uint32_t r[32];
+        tc_load_32cols(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN + c, r);
+        if (p.relu) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(fmaxf(__uint_as_float(r[i]), 0.f));
+        }
+        __syncwarp();   // the previous block has been read back
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(buf + lane * 128 + ((j ^ (lane & 7)) << 4)),
+                       "r"(r[4 * j]), "r"(r[4 * j + 1]), "r"(r[4 * j + 2]), "r"(r[4 * j + 3])
+                       : "memory");
+        __syncwarp();
+        const bool col_ok = n0 + piece * 4 < p.O;   // O is a multiple of 4
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+          const int rr = it * 4 + sub_row;
+          uint32_t v0, v1, v2, v3;
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3)
+                       : "r"(buf + rr * 128 + ((piece ^ (rr & 7)) << 4))
+                       : "memory");
+          if (row_off[it] >= 0 && col_ok)
+            *reinterpret_cast<uint4*>(out + row_off[it] + n0 + piece * 4) = make_uint4(v0, v1, v2, v3);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+    }
+  }
+
+  __syncwarp();
+  if (*abort_flag) {
+    const uint64_t t0 = global_timer();
+    while (global_timer() - t0 < 20000000ull) { }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"(static_cast<uint32_t>(kTmemCols))
+                 : "memory");
+  }
+}
+
 // One block waits on a barrier that nothing ever arrives at, with the same bounded wait the GEMM
 // pipeline uses: it must give up after `limit_ns`, raise the status word and return normally.
 __global__ void bounded_wait_selftest(uint64_t limit_ns) {
@@ -1111,6 +1361,125 @@ ConvPlan plan_conv(const DotProblem& d) {
   return pl;
 }
 
+// Tiling of a stride-1 convolution for conv_halo.
+struct HaloPlan {
+  bool ok = false;
+  int bn = 64, Wb = 0, R = 0, RB = 0, tiles_per_img = 0, sa = 0, sb = 0, resident = 0, tg = 1;
+};
+
+HaloPlan plan_halo(const DotProblem& d, const ConvPlan& pl, uint32_t flags) {
+  HaloPlan hp;
+  if (!d.conv || !pl.tc || pl.rowwin || (flags & GL_OUT_NCHW)) return hp;
+  if (d.Sh != 1 || d.Sw != 1 || pl.Cp % kBK != 0 || d.O % 4 != 0) return hp;
+  if (d.Kh == 1 && d.Kw == 1) return hp;   // no overlap between windows: nothing to keep
+  // 64-wide tiles are bound by the issue rate of N = 64 MMAs either way, and there two blocks per SM
+  // (the im2col-mode kernel) hide start-up and epilogue better than one resident block (measured)
+  if (d.O <= 64) return hp;
+  const int64_t Wb = d.W + d.pw_lo + d.pw_hi;
+  // the MMA of the last tap reads 128 rows starting (Kh-1)*Wb + Kw-1 rows into the stage
+  if (Wb > 256 || (d.Kh - 1) * Wb + d.Kw - 1 + kBM > kHaloARows) return hp;
+  const int64_t R = std::min<int64_t>(d.Ho, (kBM + d.Kw - 1) / Wb);
+  if (R < 1) return hp;
+  const int64_t tpi = (d.Ho + R - 1) / R;
+  // rows of the 128-row tiles that hold real outputs; small images fill too little of a tile
+  if (10 * d.Ho * d.Wo < 6 * tpi * kBM) return hp;
+  if (d.N * tpi * ((d.O + 63) / 64) >= (1ll << 28) || d.N >= (1ll << 30) || d.H >= (1ll << 30)) return hp;
+  hp.bn = 128;
+  hp.Wb = static_cast<int>(Wb);
+  hp.R = static_cast<int>(R);
+  hp.RB = static_cast<int>(R + d.Kh - 1);
+  hp.tiles_per_img = static_cast<int>(tpi);
+  // a B stage holds one filter row of one 64-channel chunk when that stays within 48 KB, else one tap
+  hp.tg = d.Kw * hp.bn * kBK * 2 <= 48 * 1024 ? static_cast<int>(d.Kw) : 1;
+  const int stage_b = hp.tg * hp.bn * kBK * 2;
+  const int64_t groups = (pl.Cp / kBK) * d.Kh * (d.Kw / hp.tg);
+  const int tiles_n = static_cast<int>((d.O + hp.bn - 1) / hp.bn);
+  // weights that fit beside two input boxes stay in shared memory for the whole kernel
+  if (tiles_n == 1 && groups <= kHaloMaxStages && groups * stage_b + 2 * kHaloAStage <= kHaloSmemBudget) {
+    hp.resident = 1;
+    hp.sb = static_cast<int>(groups);
+    hp.sa = std::min<int>(6, (kHaloSmemBudget - hp.sb * stage_b) / kHaloAStage);
+  } else {
+    hp.sa = 2;
+    hp.sb = std::min<int>(8, (kHaloSmemBudget - hp.sa * kHaloAStage) / stage_b);
+    if (hp.sb > 4) { hp.sa = 3; hp.sb = std::min<int>(8, (kHaloSmemBudget - hp.sa * kHaloAStage) / stage_b); }
+  }
+  hp.ok = hp.sa >= 2 && hp.sb >= 2;
+  return hp;
+}
+
+// Channels-last activations (N,H,W,Cp) as a tiled map whose box is the input block of one tile:
+// 64 channels x Wb pixels x RB rows of one image; cells outside the image read as zeros.
+bool encode_halo_box(CUtensorMap* m, const void* base, const DotProblem& d, int64_t Cp, int Wb, int RB) {
+  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(Cp), static_cast<cuuint64_t>(d.W), static_cast<cuuint64_t>(d.H),
+                              static_cast<cuuint64_t>(d.N)};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(Cp) * 2, static_cast<cuuint64_t>(d.W * Cp) * 2,
+                                 static_cast<cuuint64_t>(d.H * d.W * Cp) * 2};
+  const cuuint32_t box[4] = {kBK, static_cast<cuuint32_t>(Wb), static_cast<cuuint32_t>(RB), 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return driver_api().tiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Weights (O, Kh, Kw, Cp) viewed as (64 channels, O, chunk, tap): one box = BN rows x 64 channels of
+// `tg` consecutive taps of one chunk, landing as [tap][row][64].
+bool encode_halo_weights(CUtensorMap* m, const void* base, int64_t O, int64_t taps, int64_t Cp, int bn, int tg) {
+  const cuuint64_t dims[4] = {kBK, static_cast<cuuint64_t>(O), static_cast<cuuint64_t>(Cp / kBK),
+                              static_cast<cuuint64_t>(taps)};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(taps * Cp) * 2, kBK * 2, static_cast<cuuint64_t>(Cp) * 2};
+  const cuuint32_t box[4] = {kBK, static_cast<cuuint32_t>(bn), 1, static_cast<cuuint32_t>(tg)};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return driver_api().tiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN>
+int launch_halo(const CUtensorMap& ma, const CUtensorMap& mb, float* out, const HaloParams& p, cudaStream_t st) {
+  const int smem = p.sa_stages * kHaloAStage + p.sb_stages * static_cast<int>(p.b_bytes) + kHaloEpiBytes + kHaloBarBytes + 1024;
+  static bool attr_set_dev[64] = {false};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return GL_ERR_CUDA;
+  if (!attr_set_dev[dev]) {
+    if (cudaFuncSetAttribute(conv_halo<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448) != cudaSuccess)
+      return GL_ERR_CUDA;
+    attr_set_dev[dev] = true;
+  }
+  const int tiles = p.tiles_m * p.tiles_n;
+  const int grid = std::min(tiles, num_sms());
+  conv_halo<BN><<<grid, kTcThreads, smem, st>>>(ma, mb, out, p);
+  return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+}
+
+int run_halo(const HaloPlan& hp, const DotProblem& d, int64_t Cp, const uint16_t* x, const uint16_t* wt, float* out,
+             int relu, cudaStream_t st) {
+  HaloParams p;
+  std::memset(&p, 0, sizeof(p));
+  p.O = d.O; p.relu = relu;
+  p.Ho = static_cast<int>(d.Ho); p.Wo = static_cast<int>(d.Wo);
+  p.Wb = hp.Wb; p.R = hp.R;
+  p.tiles_m = static_cast<int>(d.N) * hp.tiles_per_img;
+  p.tiles_n = static_cast<int>((d.O + hp.bn - 1) / hp.bn);
+  p.Kh = static_cast<int>(d.Kh); p.Kw = static_cast<int>(d.Kw);
+  p.Cp = static_cast<int>(Cp);
+  p.cchunks = static_cast<int>(Cp / kBK);
+  p.tg = hp.tg;
+  p.groups_per_chunk = p.Kh * (p.Kw / hp.tg);
+  p.ph = static_cast<int>(d.ph_lo); p.pw = static_cast<int>(d.pw_lo);
+  p.sa_stages = hp.sa; p.sb_stages = hp.sb; p.b_resident = hp.resident;
+  p.a_bytes = static_cast<uint32_t>(kBK * 2 * hp.Wb * hp.RB);
+  p.b_bytes = static_cast<uint32_t>(hp.tg * hp.bn * kBK * 2);
+  p.div_tiles_n.set(p.tiles_n);
+  p.div_tpi.set(hp.tiles_per_img);
+  p.div_wb.set(hp.Wb);
+  CUtensorMap ma, mb;
+  if (!encode_halo_box(&ma, x, d, Cp, hp.Wb, hp.RB) ||
+      !encode_halo_weights(&mb, wt, d.O, d.Kh * d.Kw, Cp, hp.bn, hp.tg))
+    return GL_ERR_CUDA;
+  return launch_halo<128>(ma, mb, out, p, st);
+}
+
 // A 1x1, stride-1, unpadded window over channels-last items is no window at all: the activations
 // already are the [N*H*W, C] matrix (the special case "1x1 conv == matmul").
 bool conv_is_plain_matrix(const DotProblem& d, uint32_t flags) {
@@ -1224,7 +1593,9 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
   p.out_nchw = out_nchw;
   // tile width and K split; a K split needs room for its partial planes behind the layout copies
   const size_t pre_bytes = (d.conv && pl.prepass) ? pl.x_bytes + pl.w_bytes : 0;
-  const bool split_mode = (!d.conv || (!pl.rowwin && pl.Cp >= kBK)) && !out_nchw;
+  HaloPlan hp;
+  if (d.conv) hp = plan_halo(d, pl, flags);
+  const bool split_mode = (!d.conv || (!pl.rowwin && pl.Cp >= kBK)) && !out_nchw && !hp.ok;
   const int64_t kblocks_all = !d.conv ? (d.K + kBK - 1) / kBK : d.Kh * d.Kw * ((pl.Cp + kBK - 1) / kBK);
   TilePlan tp = plan_tiles(d.M, d.O, kblocks_all, split_mode);
   if (tp.ksplit > 1 && (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023u) ||
@@ -1329,6 +1700,7 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     wt = ws;
   }
   const int64_t Cp = pl.Cp, taps = d.Kh * d.Kw;
+  if (hp.ok) return run_halo(hp, d, Cp, x, wt, dst, relu, st);
   p.K = taps * Cp;
   p.Cp = static_cast<int>(Cp);
   p.Kh = static_cast<int>(d.Kh); p.Kw = static_cast<int>(d.Kw);

@@ -275,6 +275,31 @@ def test_conv_paired_tiles_bit_exact(gl):
     assert np.array_equal(got.astype(np.float64), np.maximum(ref, 0.0))
 
 
+# Stride-1 convolutions whose input block stays in shared memory across the filter taps: weights that
+# stay resident (one chunk), weights streamed per filter row, per tap (5x5), two channel chunks, no padding.
+CONV_RESIDENT_WINDOWS = [
+    (2, 64, 12, 20, 128, 3, 3, 1, 1),
+    (1, 128, 12, 20, 96, 5, 5, 2, 2),
+    (3, 64, 16, 30, 160, 3, 3, 0, 0),
+    (2, 192, 14, 14, 260, 3, 3, 1, 1),
+    (2, 64, 9, 40, 68, 2, 4, 1, 2),
+]
+
+
+@pytest.mark.parametrize("case", CONV_RESIDENT_WINDOWS, ids=lambda c: "x".join(map(str, c)))
+def test_conv_resident_window_tiles_bit_exact(gl, case):
+    n, c, h, w, o, kh, kw, ph, pw = case
+    x = synth.uniform_int(39, 1, (n, c, h, w), -3, 3)
+    wt = synth.uniform_int(39, 2, (o, c, kh, kw), -3, 3)
+    ref = _conv_ref(x, wt, (1, 1), (ph, pw))
+    for flags in (0, gl.GL_EPILOGUE_RELU):
+        got = _conv_gpu(gl, x, wt, (1, 1), (ph, pw), channels_last=True, flags=flags)
+        assert got.shape == ref.shape
+        assert np.array_equal(got.astype(np.float64), np.maximum(ref, 0.0) if flags else ref)
+    got = _conv_gpu(gl, x, wt, (1, 1), (ph, pw), channels_last=False)
+    assert np.array_equal(got.astype(np.float64), ref)
+
+
 def test_dense_interpreter_program_with_relu(gl):
     a = synth.uniform_int(32, 1, (20, 16), -3, 3)
     b = synth.uniform_int(32, 2, (12, 16), -3, 3)
