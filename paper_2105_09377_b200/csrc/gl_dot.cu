@@ -1054,6 +1054,278 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   }
 }
 
+// ------------------------------------------------------------------------
+// Few input channels: windows read in place from runs of the padded input rows
+// ------------------------------------------------------------------------
+//
+// With pixels padded to Cp = 8 / Sw channels, the windows of neighbouring output columns start exactly
+// 16 bytes apart in a (zero-bordered) row of the input, and a filter row of a window is Kw * Cp
+// consecutive elements of that row.  The rows of the A operand are therefore overlapping pieces of one
+// contiguous run of bytes.  The un-swizzled K-major operand layout of tcgen05.mma places row r of an
+// 8-row group 16 bytes after row r-1 and K chunk j (8 elements) "leading byte offset" bytes after chunk
+// j-1; with a leading byte offset of 16 and 128 bytes between 8-row groups the tensor core reads
+//     A[r][k] = run[8 r + k]
+// which is exactly windows(row, Kw*Cp, stride 8 elements) (Section 4.2) without forming it: shared memory
+// holds each input row run ONCE (2 KB for 128 output columns), copied by one bulk copy per filter row, and
+// cartProd/dotProd run over it as Kh * ceil(Kw*Cp/16) MMAs per tile.  The weights (a few KB) stay resident.
+
+constexpr int kRunThreads = 192;       // warp 0 copies, warp 1 issues MMAs, warps 2-5 store results
+constexpr int kRunMaxStages = 8;
+constexpr int kRunEpiBytes = 4 * 2 * 4096;   // two 32x32 fp32 staging tiles per epilogue warp
+
+struct RowRunParams {
+  int64_t O;
+  int relu;
+  int Ho, Wo, Hp, Sh, Kh;
+  int segs, tiles;              // 128-column segments per output row; tiles = N * Ho * segs
+  int ksteps;                   // MMAs (K = 16) per filter row
+  int bn;                       // MMA N: O rounded up to 16
+  uint32_t seg_bytes;           // bytes of one run: 127 * 16 + ksteps * 32
+  uint32_t slot_bytes;          // shared-memory pitch of a run
+  uint32_t pitch_bytes;         // bytes between padded input rows in global memory
+  uint32_t b_bytes;             // resident weights: Kh * ksteps * 2 chunks * bn rows * 16 bytes
+  int stages;
+  FastDiv div_segs, div_ho;
+};
+
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+__global__ void __launch_bounds__(kRunThreads, 2)
+conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restrict__ wpack,
+            const __grid_constant__ CUtensorMap map_c, const RowRunParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* gen = smem_raw + (base - raw);
+  const uint32_t stage_bytes = static_cast<uint32_t>(p.Kh) * p.slot_bytes;
+  const uint32_t epi_base = base;                                         // 1024-byte aligned staging tiles
+  const uint32_t b_base = epi_base + kRunEpiBytes;
+  const uint32_t a_base = b_base + ((p.b_bytes + 127u) & ~127u);
+  const uint32_t bars_off = (a_base - base) + ((static_cast<uint32_t>(p.stages) * stage_bytes + 7u) & ~7u);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(gen + bars_off);
+  const uint32_t bar_full = smem_u32(bars);                  // [kRunMaxStages]
+  const uint32_t bar_empty = bar_full + 8 * kRunMaxStages;   // [kRunMaxStages]
+  const uint32_t bar_tfull = bar_empty + 8 * kRunMaxStages;  // [2]
+  const uint32_t bar_tempty = bar_tfull + 16;                // [2]
+  const uint32_t bar_b = bar_tempty + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kRunMaxStages + 5);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const uint32_t tmem_cols = 2 * p.bn <= 32 ? 32u : (2 * p.bn <= 64 ? 64u : (2 * p.bn <= 128 ? 128u : 256u));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, 4); }
+    mbar_init(bar_b, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(tmem_cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- producer: the weights once, then Kh row runs per tile ----------------
+    // lane 0 waits for the stage and announces the bytes; lanes 0..Kh-1 then issue one row copy each
+    // (one warp instruction instead of Kh trips through a single-thread loop)
+    if (lane == 0) {
+      mbar_expect_tx(bar_b, p.b_bytes);
+      bulk_copy_g2s(b_base, wpack, p.b_bytes, bar_b);
+    }
+    uint32_t s = 0, ph = 0;
+    int ok = 1;
+    for (int u = blockIdx.x; u < p.tiles; u += gridDim.x) {
+      uint32_t row, seg, img, ho;
+      p.div_segs.divmod(static_cast<uint32_t>(u), row, seg);
+      p.div_ho.divmod(row, img, ho);
+      // filter row `lane` of the tile: padded input row img * Hp + ho * Sh + lane, 16 bytes per output column
+      const unsigned char* src = xpad + (static_cast<int64_t>(img) * p.Hp + static_cast<int64_t>(ho) * p.Sh + lane) * p.pitch_bytes +
+                                 static_cast<int64_t>(seg) * (kBM * 16);
+      if (lane == 0) {
+        ok = mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag) ? 1 : 0;
+        if (ok) mbar_expect_tx(bar_full + 8 * s, static_cast<uint32_t>(p.Kh) * p.seg_bytes);
+      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      if (lane < p.Kh) bulk_copy_g2s(a_base + s * stage_bytes + lane * p.slot_bytes, src, p.seg_bytes, bar_full + 8 * s);
+      if (++s == static_cast<uint32_t>(p.stages)) { s = 0; ph ^= 1u; }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc(kBM, p.bn);
+      const uint64_t desc_a0 = make_desc(a_base, 16, 128, 0);                                   // overlapping rows
+      const uint64_t desc_b0 = make_desc(b_base, static_cast<uint32_t>(p.bn) * 16, 128, 0);    // [chunk][row][16 bytes]
+      const uint32_t b_step = (2u * p.bn * 16u) >> 4;                                           // two K chunks per MMA
+      uint32_t s = 0, ph = 0, tile_it = 0;
+      bool ok = mbar_wait(bar_b, 0, abort_flag);
+      for (int u = blockIdx.x; u < p.tiles && ok; u += gridDim.x, ++tile_it) {
+        const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
+        if (!mbar_wait(bar_tempty + 8 * acc, aph ^ 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * p.bn;
+        uint64_t da_row = desc_a0 + ((s * stage_bytes) >> 4), db = desc_b0;
+        uint32_t accumulate = 0;
+        for (int kh = 0; kh < p.Kh; ++kh, da_row += p.slot_bytes >> 4) {
+          uint64_t da = da_row;
+          for (int k = 0; k < p.ksteps; ++k, da += 2, db += b_step) {
+            tc_mma_bf16(d_tmem, da, db, idesc, accumulate);
+            accumulate = 1u;
+          }
+        }
+        tc_commit(bar_empty + 8 * s);
+        tc_commit(bar_tfull + 8 * acc);
+        if (++s == static_cast<uint32_t>(p.stages)) { s = 0; ph ^= 1u; }
+      }
+    }
+  } else {
+    // ---------------- epilogue: TMEM -> registers -> swizzled 32x32 blocks -> TMA stores ----------------
+    const int q = warp & 3;
+    uint32_t tile_it = 0, chunk_it = 0;
+    bool ok = true;
+    if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_c)) : "memory");
+    for (int u = blockIdx.x; u < p.tiles && ok; u += gridDim.x, ++tile_it) {
+      const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
+      uint32_t row, seg;
+      p.div_segs.divmod(static_cast<uint32_t>(u), row, seg);
+      if (!mbar_wait(bar_tfull + 8 * acc, aph, abort_flag)) { ok = false; break; }
+      tc_fence_after();
+#pragma unroll 1
+      for (int c = 0; c < p.bn; c += 32) {
+        if (c >= p.O) break;   // uniform across the warp
+        uint32_t r[32];
+        tc_load_32cols(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * p.bn + c, r);
+        if (p.relu) {
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(fmaxf(__uint_as_float(r[i]), 0.f));
+        }
+        const uint32_t buf = epi_base + q * 8192 + (chunk_it & 1u) * 4096;
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the store before last has read this buffer
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(buf + lane * 128 + ((j ^ (lane & 7)) << 4)),
+                       "r"(r[4 * j]), "r"(r[4 * j + 1]), "r"(r[4 * j + 2]), "r"(r[4 * j + 3])
+                       : "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {   // result viewed as (N*Ho, Wo, O): columns past Wo and channels past O are clipped
+          asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(
+                           reinterpret_cast<uint64_t>(&map_c)),
+                       "r"(c), "r"(static_cast<int>(seg) * kBM + q * 32), "r"(static_cast<int>(row)), "r"(buf)
+                       : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        }
+        ++chunk_it;
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+    }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+
+  __syncwarp();
+  if (*abort_flag) {
+    const uint64_t t0 = global_timer();
+    while (global_timer() - t0 < 20000000ull) { }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+  }
+}
+
+// Layout pre-pass of conv_rowrun, one launch.
+// Blocks [0, row_blocks): padded copy (N, Hp, Wpa, Cp) with zero borders.  A warp takes one padded row at a
+// time: it stages the pixels of the input row in shared memory (coalesced reads in either item layout) and
+// writes 16-byte chunks (8 / Cp pixels).  Blocks from row_blocks on: the weights in operand order
+// [kh][K chunk j][row o < bn][8 elements], element kw * Cp + c of filter row kh at
+// (j, i) = ((kw * Cp + c) / 8, (kw * Cp + c) % 8); zeros elsewhere.
+constexpr int kPackWarps = 8;
+constexpr int kPackRowsPerWarp = 2;
+
+__global__ void __launch_bounds__(32 * kPackWarps) rowrun_pack(const uint16_t* __restrict__ in, uint16_t* __restrict__ out,
+                                                               const uint16_t* __restrict__ win, uint16_t* __restrict__ wout,
+                                                               int channels_last, int row_blocks, int rows, int C, int H,
+                                                               int W, int Hp, int Wpa, int cp_log2, int ph, int pw, int O,
+                                                               int Kh, int Kw, int chunks, int bn) {
+  extern __shared__ uint16_t pix[];   // [kPackWarps][W * C]
+  const int Cp = 1 << cp_log2;
+  if (static_cast<int>(blockIdx.x) >= row_blocks) {
+    const int total = Kh * chunks * bn * 8;
+    for (int e = (static_cast<int>(blockIdx.x) - row_blocks) * blockDim.x + threadIdx.x; e < total;
+         e += (static_cast<int>(gridDim.x) - row_blocks) * blockDim.x) {
+      const int i = e & 7, t = e >> 3;
+      const int o = t % bn, j = (t / bn) % chunks, kh = t / (bn * chunks);
+      const int el = j * 8 + i, kw = el >> cp_log2, c = el & (Cp - 1);
+      uint16_t val = 0;
+      if (o < O && kw < Kw && c < C)
+        val = channels_last ? win[((static_cast<int64_t>(o) * Kh + kh) * Kw + kw) * C + c]
+                            : win[((static_cast<int64_t>(o) * C + c) * Kh + kh) * Kw + kw];
+      wout[e] = val;
+    }
+    return;
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int WC = W * C;
+  uint16_t* mine = pix + warp * WC;
+  const int nchunks = (Wpa << cp_log2) >> 3;
+  const int ppc = 8 >> cp_log2;   // pixels per 16-byte chunk
+  int rowid = (static_cast<int>(blockIdx.x) * kPackWarps + warp) * kPackRowsPerWarp;
+  int n = rowid / Hp, hp = rowid - n * Hp;
+  for (int r = 0; r < kPackRowsPerWarp && rowid < rows; ++r, ++rowid) {
+    const int h = hp - ph;
+    const bool row_ok = h >= 0 && h < H;
+    __syncwarp();   // the previous row has been written out
+    if (row_ok) {
+      if (channels_last) {
+        const uint16_t* src = in + (static_cast<int64_t>(n) * H + h) * WC;
+#pragma unroll 4
+        for (int e = lane; e < WC; e += 32) mine[e] = src[e];
+      } else {
+        for (int c = 0; c < C; ++c) {
+          const uint16_t* src = in + ((static_cast<int64_t>(n) * C + c) * H + h) * W;
+#pragma unroll 4
+          for (int w = lane; w < W; w += 32) mine[w * C + c] = src[w];
+        }
+      }
+    }
+    __syncwarp();
+    uint4* orow = reinterpret_cast<uint4*>(out + (static_cast<int64_t>(rowid) * Wpa << cp_log2));
+    for (int ch = lane; ch < nchunks; ch += 32) {
+      // 8 elements = ppc pixels of Cp channels; element i of the chunk is channel i % Cp of pixel i / Cp
+      uint32_t word[4] = {0u, 0u, 0u, 0u};
+      for (int px = 0; px < ppc; ++px) {
+        const int w = ch * ppc + px - pw;
+        if (row_ok && w >= 0 && w < W) {
+          const uint16_t* sp = mine + w * C;
+          for (int c = 0; c < C; ++c) {
+            const int i = (px << cp_log2) + c;
+            word[i >> 1] |= static_cast<uint32_t>(sp[c]) << (16 * (i & 1));
+          }
+        }
+      }
+      orow[ch] = make_uint4(word[0], word[1], word[2], word[3]);
+    }
+    if (++hp == Hp) { hp = 0; ++n; }
+  }
+}
+
 // One block waits on a barrier that nothing ever arrives at, with the same bounded wait the GEMM
 // pipeline uses: it must give up after `limit_ns`, raise the status word and return normally.
 __global__ void bounded_wait_selftest(uint64_t limit_ns) {
@@ -1332,9 +1604,13 @@ struct ConvPlan {
   size_t x_bytes = 0, w_bytes = 0;
   bool rowwin = false;   // few channels: row-window layout (always through the workspace)
   int64_t Hp = 0, Wpa = 0;
+  // conv_rowrun: windows read in place from runs of the padded rows (pixels of 8 / Sw channels)
+  bool rowrun = false;
+  int rr_cp = 0, rr_ksteps = 0, rr_bn = 0, rr_stages = 0;
+  uint32_t rr_seg = 0, rr_slot = 0, rr_b_bytes = 0;
 };
 
-ConvPlan plan_conv(const DotProblem& d) {
+ConvPlan plan_conv(const DotProblem& d, uint32_t flags) {
   ConvPlan pl;
   pl.Cp = (d.C + 7) / 8 * 8;
   const bool fits = d.pw_lo <= 128 && d.ph_lo <= 128 && (d.Kw - 1 - d.pw_hi) <= 128 && (d.Kh - 1 - d.ph_hi) <= 128 &&
@@ -1343,6 +1619,31 @@ ConvPlan plan_conv(const DotProblem& d) {
                     d.Kh * d.Kw * pl.Cp < (1ll << 31);
   pl.tc = fits && ((d.M + 127) / 128) * ((d.O + 63) / 64) < (1ll << 28);
   pl.prepass = !d.channels_last || pl.Cp != d.C;
+  if (pl.tc && !(flags & GL_OUT_NCHW) && (d.Sw == 1 || d.Sw == 2 || d.Sw == 4 || d.Sw == 8) && d.C <= 8 / d.Sw &&
+      d.O % 4 == 0 && d.O <= 128 && d.Kh <= 16 && kPackWarps * d.W * d.C * 2 <= 48 * 1024 && d.Wo < (1ll << 24) &&
+      d.N * (d.H + d.ph_lo + d.ph_hi) < (1ll << 31)) {
+    const int cp = static_cast<int>(8 / d.Sw);
+    const int ksteps = static_cast<int>((d.Kw * cp + 15) / 16);
+    const int bn = static_cast<int>((d.O + 15) / 16 * 16);
+    const uint32_t seg = 127 * 16 + ksteps * 32, slot = (seg + 127u) & ~127u;
+    const uint32_t b_bytes = static_cast<uint32_t>(d.Kh) * ksteps * 2 * bn * 16;
+    const int64_t room = 113 * 1024 - 1024 - kRunEpiBytes - 256 - ((b_bytes + 127) & ~127u);   // two blocks per SM
+    const int64_t stages = std::min<int64_t>(kRunMaxStages, room / (d.Kh * slot));
+    if (stages >= 2) {
+      pl.rowrun = true;
+      pl.prepass = true;
+      pl.rr_cp = cp; pl.rr_ksteps = ksteps; pl.rr_bn = bn; pl.rr_stages = static_cast<int>(stages);
+      pl.rr_seg = seg; pl.rr_slot = slot; pl.rr_b_bytes = b_bytes;
+      pl.Hp = d.H + d.ph_lo + d.ph_hi;
+      // every window of a real output column lies inside its row; the row pitch is a multiple of 16 bytes
+      pl.Wpa = std::max(d.W + d.pw_lo + d.pw_hi, (d.Wo - 1) * d.Sw + (ksteps * 16 + cp - 1) / cp);
+      pl.Wpa = (pl.Wpa * cp + 7) / 8 * 8 / cp;
+      // the runs of the columns past Wo (computed, never stored) may reach past the last row: slack
+      pl.x_bytes = round_up(static_cast<size_t>(d.N * pl.Hp * pl.Wpa * cp) * 2 + kBM * 16 + 4096, 1024);
+      pl.w_bytes = round_up(b_bytes, 1024);
+      return pl;
+    }
+  }
   if (pl.tc && pl.Cp < kBK && d.Kw * pl.Cp <= kBK && d.Wo < (1ll << 24) && d.N * (d.H + d.ph_lo + d.ph_hi) < (1ll << 31)) {
     pl.rowwin = true;
     pl.prepass = true;
@@ -1537,7 +1838,7 @@ size_t gl_cartesian_dot_workspace(const gl_ap* a0, const gl_windows* w, const gl
     if (!dense_tc_ok(d)) return 0;
     return plan_tiles(d.M, d.O, (d.K + kBK - 1) / kBK, true).partial_bytes;
   }
-  const ConvPlan pl = plan_conv(d);
+  const ConvPlan pl = plan_conv(d, flags);
   if (!pl.tc) return 0;
   size_t need = pl.prepass ? pl.x_bytes + pl.w_bytes : 0;
   if (!pl.rowwin && pl.Cp >= kBK && !(flags & GL_OUT_NCHW))
@@ -1574,7 +1875,7 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
   const bool force_general = (flags & GL_DOT_GENERAL_KERNEL) != 0;
   if (!force_general && conv_is_plain_matrix(d, flags)) d.conv = false;
   ConvPlan pl;
-  if (d.conv) pl = plan_conv(d);
+  if (d.conv) pl = plan_conv(d, flags);
   const bool use_tc = !force_general && ((d.conv && pl.tc) || dense_tc_ok(d));
   if (!use_tc) {
     GenA g;
@@ -1637,6 +1938,51 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u)) return GL_ERR_WORKSPACE;
     uint16_t* xs = static_cast<uint16_t*>(workspace);
     uint16_t* ws = reinterpret_cast<uint16_t*>(static_cast<unsigned char*>(workspace) + pl.x_bytes);
+    if (pl.rowrun) {
+      const int chunks = 2 * pl.rr_ksteps;
+      int cp_log2 = 0;
+      while ((1 << cp_log2) < pl.rr_cp) ++cp_log2;
+      const int rows = static_cast<int>(d.N * pl.Hp);
+      const int rows_per_block = kPackWarps * kPackRowsPerWarp;
+      const int row_blocks = (rows + rows_per_block - 1) / rows_per_block;
+      const int wblocks = static_cast<int>((pl.rr_b_bytes / 2 + 255) / 256);
+      rowrun_pack<<<static_cast<unsigned>(row_blocks + wblocks), 32 * kPackWarps, static_cast<size_t>(kPackWarps * d.W * d.C * 2), st>>>(
+          pa, xs, pb, ws, d.channels_last ? 1 : 0, row_blocks, rows, static_cast<int>(d.C), static_cast<int>(d.H),
+          static_cast<int>(d.W), static_cast<int>(pl.Hp), static_cast<int>(pl.Wpa), cp_log2, static_cast<int>(d.ph_lo),
+          static_cast<int>(d.pw_lo), static_cast<int>(d.O), static_cast<int>(d.Kh), static_cast<int>(d.Kw), chunks,
+          pl.rr_bn);
+      if (cudaGetLastError() != cudaSuccess) return GL_ERR_CUDA;
+      RowRunParams rp;
+      std::memset(&rp, 0, sizeof(rp));
+      rp.O = d.O; rp.relu = relu;
+      rp.Ho = static_cast<int>(d.Ho); rp.Wo = static_cast<int>(d.Wo); rp.Hp = static_cast<int>(pl.Hp);
+      rp.Sh = static_cast<int>(d.Sh); rp.Kh = static_cast<int>(d.Kh);
+      rp.segs = static_cast<int>((d.Wo + kBM - 1) / kBM);
+      rp.tiles = static_cast<int>(d.N * d.Ho * rp.segs);
+      rp.ksteps = pl.rr_ksteps; rp.bn = pl.rr_bn;
+      rp.seg_bytes = pl.rr_seg; rp.slot_bytes = pl.rr_slot;
+      rp.pitch_bytes = static_cast<uint32_t>(pl.Wpa * pl.rr_cp * 2);
+      rp.b_bytes = pl.rr_b_bytes;
+      rp.stages = pl.rr_stages;
+      rp.div_segs.set(rp.segs);
+      rp.div_ho.set(d.Ho);
+      CUtensorMap mc;
+      if (!encode_result_rows(&mc, dst, d.N * d.Ho, d.Wo, d.O)) return GL_ERR_CUDA;
+      const int smem = 1024 + kRunEpiBytes + static_cast<int>((rp.b_bytes + 127u) & ~127u) +
+                       rp.stages * rp.Kh * static_cast<int>(rp.slot_bytes) + 256;
+      static bool attr_set_dev[64] = {false};
+      int dev = 0;
+      if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return GL_ERR_CUDA;
+      if (!attr_set_dev[dev]) {
+        if (cudaFuncSetAttribute(conv_rowrun, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024) != cudaSuccess)
+          return GL_ERR_CUDA;
+        attr_set_dev[dev] = true;
+      }
+      const int grid = std::min(rp.tiles, 2 * num_sms());
+      conv_rowrun<<<grid, kRunThreads, smem, st>>>(reinterpret_cast<const unsigned char*>(xs),
+                                                    reinterpret_cast<const unsigned char*>(ws), mc, rp);
+      return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+    }
     if (pl.rowwin) {
       rowwin_pack_x<<<static_cast<unsigned>(d.N * pl.Hp), 256, 0, st>>>(
           pa, xs, d.channels_last ? 1 : 0, static_cast<int>(d.C), static_cast<int>(d.H), static_cast<int>(d.W),
