@@ -1252,19 +1252,21 @@ conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restr
 
 // Layout pre-pass of conv_rowrun, one launch.
 // Blocks [0, row_blocks): padded copy (N, Hp, Wpa, Cp) with zero borders.  A warp takes one padded row at a
-// time: it stages the pixels of the input row in shared memory (coalesced reads in either item layout) and
-// writes 16-byte chunks (8 / Cp pixels).  Blocks from row_blocks on: the weights in operand order
+// time and builds it in shared memory: the buffer starts as zeros, the pixels of the input row are dropped
+// at their padded positions (border cells and channels past C are never written, so they stay zero), and
+// the finished row leaves as 16-byte pieces.  Blocks from row_blocks on: the weights in operand order
 // [kh][K chunk j][row o < bn][8 elements], element kw * Cp + c of filter row kh at
 // (j, i) = ((kw * Cp + c) / 8, (kw * Cp + c) % 8); zeros elsewhere.
 constexpr int kPackWarps = 8;
-constexpr int kPackRowsPerWarp = 2;
+constexpr int kPackRowsPerWarp = 1;
 
+template <int C>   // input channels (1..8), a compile-time constant so that the per-pixel loops carry no tests
 __global__ void __launch_bounds__(32 * kPackWarps) rowrun_pack(const uint16_t* __restrict__ in, uint16_t* __restrict__ out,
                                                                const uint16_t* __restrict__ win, uint16_t* __restrict__ wout,
-                                                               int channels_last, int row_blocks, int rows, int C, int H,
+                                                               int channels_last, int row_blocks, int rows, int H,
                                                                int W, int Hp, int Wpa, int cp_log2, int ph, int pw, int O,
                                                                int Kh, int Kw, int chunks, int bn) {
-  extern __shared__ uint16_t pix[];   // [kPackWarps][W * C]
+  extern __shared__ uint4 padded_rows[];   // [kPackWarps][Wpa * Cp / 8] pieces of 16 bytes
   const int Cp = 1 << cp_log2;
   if (static_cast<int>(blockIdx.x) >= row_blocks) {
     const int total = Kh * chunks * bn * 8;
@@ -1282,45 +1284,46 @@ __global__ void __launch_bounds__(32 * kPackWarps) rowrun_pack(const uint16_t* _
     return;
   }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int WC = W * C;
-  uint16_t* mine = pix + warp * WC;
   const int nchunks = (Wpa << cp_log2) >> 3;
-  const int ppc = 8 >> cp_log2;   // pixels per 16-byte chunk
+  uint4* mine = padded_rows + warp * nchunks;
+  uint16_t* cells = reinterpret_cast<uint16_t*>(mine) + (pw << cp_log2);   // pixel 0 of the input row
+  for (int ch = lane; ch < nchunks; ch += 32) mine[ch] = make_uint4(0u, 0u, 0u, 0u);
   int rowid = (static_cast<int>(blockIdx.x) * kPackWarps + warp) * kPackRowsPerWarp;
   int n = rowid / Hp, hp = rowid - n * Hp;
   for (int r = 0; r < kPackRowsPerWarp && rowid < rows; ++r, ++rowid) {
     const int h = hp - ph;
-    const bool row_ok = h >= 0 && h < H;
-    __syncwarp();   // the previous row has been written out
-    if (row_ok) {
-      if (channels_last) {
-        const uint16_t* src = in + (static_cast<int64_t>(n) * H + h) * WC;
-#pragma unroll 4
-        for (int e = lane; e < WC; e += 32) mine[e] = src[e];
-      } else {
-        for (int c = 0; c < C; ++c) {
-          const uint16_t* src = in + ((static_cast<int64_t>(n) * C + c) * H + h) * W;
-#pragma unroll 4
-          for (int w = lane; w < W; w += 32) mine[w * C + c] = src[w];
-        }
-      }
-    }
-    __syncwarp();
     uint4* orow = reinterpret_cast<uint4*>(out + (static_cast<int64_t>(rowid) * Wpa << cp_log2));
-    for (int ch = lane; ch < nchunks; ch += 32) {
-      // 8 elements = ppc pixels of Cp channels; element i of the chunk is channel i % Cp of pixel i / Cp
-      uint32_t word[4] = {0u, 0u, 0u, 0u};
-      for (int px = 0; px < ppc; ++px) {
-        const int w = ch * ppc + px - pw;
-        if (row_ok && w >= 0 && w < W) {
-          const uint16_t* sp = mine + w * C;
+    if (h < 0 || h >= H) {   // a border row
+      for (int ch = lane; ch < nchunks; ch += 32) orow[ch] = make_uint4(0u, 0u, 0u, 0u);
+    } else {
+      __syncwarp();   // the previous row has left the buffer
+      // four pixels per lane per trip, all their channel loads in flight before any is placed
+      const int64_t HW = static_cast<int64_t>(H) * W;
+      const uint16_t* src = channels_last ? in + (static_cast<int64_t>(n) * H + h) * W * C
+                                          : in + (static_cast<int64_t>(n) * C * H + h) * W;
+      const int64_t step_w = channels_last ? C : 1, step_c = channels_last ? 1 : HW;
+      for (int w0 = 0; w0 < W; w0 += 128) {
+        uint16_t v[4][C];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int w = w0 + i * 32 + lane;
+#pragma unroll
           for (int c = 0; c < C; ++c) {
-            const int i = (px << cp_log2) + c;
-            word[i >> 1] |= static_cast<uint32_t>(sp[c]) << (16 * (i & 1));
+            v[i][c] = 0;
+            if (w < W) v[i][c] = src[w * step_w + c * step_c];
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int w = w0 + i * 32 + lane;
+          if (w < W) {
+#pragma unroll
+            for (int c = 0; c < C; ++c) cells[(w << cp_log2) + c] = v[i][c];
           }
         }
       }
-      orow[ch] = make_uint4(word[0], word[1], word[2], word[3]);
+      __syncwarp();
+      for (int ch = lane; ch < nchunks; ch += 32) orow[ch] = mine[ch];
     }
     if (++hp == Hp) { hp = 0; ++n; }
   }
@@ -1620,7 +1623,7 @@ ConvPlan plan_conv(const DotProblem& d, uint32_t flags) {
   pl.tc = fits && ((d.M + 127) / 128) * ((d.O + 63) / 64) < (1ll << 28);
   pl.prepass = !d.channels_last || pl.Cp != d.C;
   if (pl.tc && !(flags & GL_OUT_NCHW) && (d.Sw == 1 || d.Sw == 2 || d.Sw == 4 || d.Sw == 8) && d.C <= 8 / d.Sw &&
-      d.O % 4 == 0 && d.O <= 128 && d.Kh <= 16 && kPackWarps * d.W * d.C * 2 <= 48 * 1024 && d.Wo < (1ll << 24) &&
+      d.O % 4 == 0 && d.O <= 128 && d.Kh <= 16 && kPackWarps * (d.W + d.pw_lo + d.pw_hi + 64) * 16 <= 48 * 1024 && d.Wo < (1ll << 24) &&
       d.N * (d.H + d.ph_lo + d.ph_hi) < (1ll << 31)) {
     const int cp = static_cast<int>(8 / d.Sw);
     const int ksteps = static_cast<int>((d.Kw * cp + 15) / 16);
@@ -1946,11 +1949,24 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
       const int rows_per_block = kPackWarps * kPackRowsPerWarp;
       const int row_blocks = (rows + rows_per_block - 1) / rows_per_block;
       const int wblocks = static_cast<int>((pl.rr_b_bytes / 2 + 255) / 256);
-      rowrun_pack<<<static_cast<unsigned>(row_blocks + wblocks), 32 * kPackWarps, static_cast<size_t>(kPackWarps * d.W * d.C * 2), st>>>(
-          pa, xs, pb, ws, d.channels_last ? 1 : 0, row_blocks, rows, static_cast<int>(d.C), static_cast<int>(d.H),
-          static_cast<int>(d.W), static_cast<int>(pl.Hp), static_cast<int>(pl.Wpa), cp_log2, static_cast<int>(d.ph_lo),
-          static_cast<int>(d.pw_lo), static_cast<int>(d.O), static_cast<int>(d.Kh), static_cast<int>(d.Kw), chunks,
-          pl.rr_bn);
+      const dim3 pgrid(static_cast<unsigned>(row_blocks + wblocks));
+      const size_t psmem = static_cast<size_t>(kPackWarps * pl.Wpa * pl.rr_cp * 2);
+#define GL_ROWRUN_PACK(CT)                                                                                              \
+  rowrun_pack<CT><<<pgrid, 32 * kPackWarps, psmem, st>>>(                                                              \
+      pa, xs, pb, ws, d.channels_last ? 1 : 0, row_blocks, rows, static_cast<int>(d.H), static_cast<int>(d.W),         \
+      static_cast<int>(pl.Hp), static_cast<int>(pl.Wpa), cp_log2, static_cast<int>(d.ph_lo), static_cast<int>(d.pw_lo), \
+      static_cast<int>(d.O), static_cast<int>(d.Kh), static_cast<int>(d.Kw), chunks, pl.rr_bn)
+      switch (d.C) {
+        case 1: GL_ROWRUN_PACK(1); break;
+        case 2: GL_ROWRUN_PACK(2); break;
+        case 3: GL_ROWRUN_PACK(3); break;
+        case 4: GL_ROWRUN_PACK(4); break;
+        case 5: GL_ROWRUN_PACK(5); break;
+        case 6: GL_ROWRUN_PACK(6); break;
+        case 7: GL_ROWRUN_PACK(7); break;
+        default: GL_ROWRUN_PACK(8); break;
+      }
+#undef GL_ROWRUN_PACK
       if (cudaGetLastError() != cudaSuccess) return GL_ERR_CUDA;
       RowRunParams rp;
       std::memset(&rp, 0, sizeof(rp));
