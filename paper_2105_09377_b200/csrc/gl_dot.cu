@@ -152,23 +152,88 @@ __global__ void __launch_bounds__(256) weights_to_channels_last(const uint16_t* 
   }
 }
 
-// Same permutation for (C,Kh,Kw) filters, staged: a block reads 64 channels x T taps of one
-// filter as one contiguous run, and writes T runs of 64 channels.
-__global__ void __launch_bounds__(256) weights_to_channels_last_staged(const uint16_t* __restrict__ in,
-                                                                       uint16_t* __restrict__ out, int C, int T,
-                                                                       int Cp) {
-  extern __shared__ uint16_t wstage[];   // [64][T]
-  const int64_t o = blockIdx.y;
-  const int c0 = blockIdx.x * 64;
-  const int nc = min(64, C - c0);        // channels with data (may be <= 0 in the padded tail)
-  const uint16_t* src = in + (o * C + c0) * T;
-  for (int e = threadIdx.x; e < nc * T; e += blockDim.x) wstage[e] = src[e];
+// Both layout copies of a (C,H,W)-item convolution in ONE launch.
+// Blocks [0, x_blocks): activations (N,C,H,W) -> (N,Hs,Ws,Cp), channels padded with zeros to Cp.  (Hs,Ws) is
+// the whole image, or - for 1x1 windows without padding, which touch only every (Sh,Sw)-th pixel - just
+// those pixels, so that the copy is the [N*H'*W', Cp] matrix itself.  A block moves 64 pixels x 64 channels:
+// pixel-contiguous reads, 16-byte channel-contiguous writes.
+// Blocks from x_blocks on: weights (O,C,T) -> (O,T,Cp), T = Kh*Kw; a block reads 64 channels x T taps of one
+// filter as one contiguous run and writes T runs of 64 channels.
+struct PrepassParams {
+  int C, H, W, Cp, Hs, Ws, Sh, Sw;
+  int tiles_p, tiles_c, x_blocks;   // pixel tiles per image, channel tiles, activation blocks = N * tiles_p * tiles_c
+  int O, T, wtiles_c;               // weight blocks = O * wtiles_c
+};
+
+__global__ void __launch_bounds__(256) nchw_prepass(const uint16_t* __restrict__ x, uint16_t* __restrict__ xs,
+                                                    const uint16_t* __restrict__ w, uint16_t* __restrict__ ws,
+                                                    const PrepassParams p) {
+  extern __shared__ uint16_t pre_smem[];
+  int b = blockIdx.x;
+  if (b >= p.x_blocks) {
+    b -= p.x_blocks;
+    const int o = b / p.wtiles_c, c0 = (b - o * p.wtiles_c) * 64;
+    const int nc = min(64, p.C - c0);        // channels with data (may be <= 0 in the padded tail)
+    const uint16_t* src = w + (static_cast<int64_t>(o) * p.C + c0) * p.T;
+    for (int e = threadIdx.x; e < nc * p.T; e += blockDim.x) pre_smem[e] = src[e];
+    __syncthreads();
+    const int ncp = min(64, p.Cp - c0);
+    uint16_t* dst = ws + static_cast<int64_t>(o) * p.T * p.Cp + c0;
+    for (int e = threadIdx.x; e < p.T * 64; e += blockDim.x) {
+      const int t = e >> 6, c = e & 63;
+      if (c < ncp) dst[static_cast<int64_t>(t) * p.Cp + c] = c < nc ? pre_smem[c * p.T + t] : static_cast<uint16_t>(0);
+    }
+    return;
+  }
+  constexpr int kPitch = 66;                 // elements per staged channel row
+  const int tc = b % p.tiles_c;
+  const int tp = (b / p.tiles_c) % p.tiles_p;
+  const int n = b / (p.tiles_c * p.tiles_p);
+  const int c0 = tc * 64, p0 = tp * 64;
+  const int npix = p.Hs * p.Ws;
+  // reads: a warp takes one channel, its lanes two stretches of 32 consecutive pixels
+  {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    int soff[2];
+    bool pok[2];
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      const int pix = p0 + j * 32 + lane;
+      pok[j] = pix < npix;
+      const int hs = pix / p.Ws, wsx = pix - hs * p.Ws;
+      soff[j] = hs * p.Sh * p.W + wsx * p.Sw;
+    }
+    const int64_t HW = static_cast<int64_t>(p.H) * p.W;
+    uint16_t v[8][2];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int c = c0 + wid + 8 * i;
+#pragma unroll
+      for (int j = 0; j < 2; ++j) {
+        v[i][j] = 0;
+        if (c < p.C && pok[j]) v[i][j] = x[(static_cast<int64_t>(n) * p.C + c) * HW + soff[j]];
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 2; ++j) pre_smem[(wid + 8 * i) * kPitch + j * 32 + lane] = v[i][j];
+  }
   __syncthreads();
-  const int ncp = min(64, Cp - c0);
-  uint16_t* dst = out + o * T * Cp + c0;
-  for (int e = threadIdx.x; e < T * 64; e += blockDim.x) {
-    const int t = e >> 6, c = e & 63;
-    if (c < ncp) dst[static_cast<int64_t>(t) * Cp + c] = c < nc ? wstage[c * T + t] : (uint16_t)0;
+  // writes: a thread takes one pixel and 8 consecutive channels (16 bytes); 512 such pieces per tile
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    const int piece = threadIdx.x + 256 * k;
+    const int pl = piece >> 3, cg = piece & 7;
+    const int pix = p0 + pl, c = c0 + cg * 8;
+    if (pix < npix && c < p.Cp) {
+      uint32_t wd[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        wd[i] = static_cast<uint32_t>(pre_smem[(cg * 8 + 2 * i) * kPitch + pl]) |
+                (static_cast<uint32_t>(pre_smem[(cg * 8 + 2 * i + 1) * kPitch + pl]) << 16);
+      *reinterpret_cast<uint4*>(xs + (static_cast<int64_t>(n) * npix + pix) * p.Cp + c) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+    }
   }
 }
 
@@ -1608,6 +1673,9 @@ struct ConvPlan {
   bool rowwin = false;   // few channels: row-window layout (always through the workspace)
   int64_t Hp = 0, Wpa = 0;
   // conv_rowrun: windows read in place from runs of the padded rows (pixels of 8 / Sw channels)
+  // (C,H,W) items with 1x1 unpadded windows: the copy holds only the pixels the windows touch and is
+  // then the [N*H'*W', Cp] matrix of a plain matrix product
+  bool as_matrix = false;
   bool rowrun = false;
   int rr_cp = 0, rr_ksteps = 0, rr_bn = 0, rr_stages = 0;
   uint32_t rr_seg = 0, rr_slot = 0, rr_b_bytes = 0;
@@ -1656,6 +1724,13 @@ ConvPlan plan_conv(const DotProblem& d, uint32_t flags) {
     pl.Wpa = (pl.Wpa + d.Sw - 1) / d.Sw * d.Sw;
     pl.x_bytes = round_up(static_cast<size_t>(d.N * pl.Hp * pl.Wpa * pl.Cp) * 2, 1024);
     pl.w_bytes = round_up(static_cast<size_t>(d.O * d.Kh * kBK) * 2, 1024);
+    return pl;
+  }
+  pl.as_matrix = pl.tc && !d.channels_last && d.Kh == 1 && d.Kw == 1 && d.ph_lo == 0 && d.ph_hi == 0 && d.pw_lo == 0 &&
+                 d.pw_hi == 0 && !(flags & GL_OUT_NCHW) && pl.Cp >= kBK;
+  if (pl.as_matrix) {
+    pl.x_bytes = round_up(static_cast<size_t>(d.N * d.Ho * d.Wo * pl.Cp) * 2, 1024);
+    pl.w_bytes = round_up(static_cast<size_t>(d.O * pl.Cp) * 2, 1024);
     return pl;
   }
   if (pl.prepass) {
@@ -2029,30 +2104,28 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
       weights_to_channels_last<<<static_cast<unsigned>(std::min<int64_t>((d.O * T * pl.Cp + 255) / 256, 1 << 20)), 256, 0,
                                  st>>>(pb, ws, d.O * T, d.C, 1, pl.Cp);
     } else {
-      if (pl.Cp == d.C) {
-        // no channel padding: (N,C,HW) -> (N,HW,C) is the library's own tiled transpose
-        gl_ap src, dstp;
-        std::memset(&src, 0, sizeof(src));
-        src.data = const_cast<uint16_t*>(pa);
-        src.dtype = GL_BF16; src.ndim = 3; src.access_ndim = 1;
-        src.shape[0] = d.N; src.shape[1] = d.C; src.shape[2] = HW;
-        dstp = src;
-        dstp.data = xs;
-        dstp.shape[1] = HW; dstp.shape[2] = d.C;
-        const int32_t perm[3] = {0, 2, 1};
-        rc = gl_access_transpose(&src, perm, &dstp, stream);
-        if (rc) return rc;
+      PrepassParams pp;
+      std::memset(&pp, 0, sizeof(pp));
+      pp.C = static_cast<int>(d.C); pp.H = static_cast<int>(d.H); pp.W = static_cast<int>(d.W);
+      pp.Cp = static_cast<int>(pl.Cp);
+      pp.Hs = static_cast<int>(pl.as_matrix ? d.Ho : d.H); pp.Ws = static_cast<int>(pl.as_matrix ? d.Wo : d.W);
+      pp.Sh = static_cast<int>(pl.as_matrix ? d.Sh : 1); pp.Sw = static_cast<int>(pl.as_matrix ? d.Sw : 1);
+      pp.O = static_cast<int>(d.O); pp.T = static_cast<int>(T);
+      const int64_t tiles_p = (static_cast<int64_t>(pp.Hs) * pp.Ws + 63) / 64, tiles_c = (pl.Cp + 63) / 64;
+      const int64_t x_blocks = d.N * tiles_p * tiles_c, w_blocks = d.O * tiles_c;
+      if (T <= 256 && x_blocks + w_blocks < (1ll << 31) && d.H * d.W < (1ll << 31) && d.C < (1ll << 24)) {
+        pp.tiles_p = static_cast<int>(tiles_p); pp.tiles_c = static_cast<int>(tiles_c);
+        pp.wtiles_c = static_cast<int>(tiles_c);
+        pp.x_blocks = static_cast<int>(x_blocks);
+        const size_t smem = std::max<size_t>(64 * 66 * 2, static_cast<size_t>(64 * T * 2));
+        nchw_prepass<<<static_cast<unsigned>(x_blocks + w_blocks), 256, smem, st>>>(pa, xs, pb, ws, pp);
+      } else if (pl.as_matrix) {
+        return GL_ERR_UNSUPPORTED;
       } else {
         if (d.N > 65535 || (d.C + 31) / 32 > 65535) return GL_ERR_UNSUPPORTED;
         const dim3 grid(static_cast<unsigned>((HW + 31) / 32), static_cast<unsigned>((pl.Cp + 31) / 32),
                         static_cast<unsigned>(d.N));
         nchw_to_nhwc_pad<<<grid, 256, 0, st>>>(pa, xs, d.C, HW, pl.Cp);
-      }
-      if (T <= 256 && d.O <= 65535 && d.C < (1ll << 30)) {
-        const dim3 grid(static_cast<unsigned>((pl.Cp + 63) / 64), static_cast<unsigned>(d.O));
-        weights_to_channels_last_staged<<<grid, 256, static_cast<size_t>(64 * T * 2), st>>>(
-            pb, ws, static_cast<int>(d.C), static_cast<int>(T), static_cast<int>(pl.Cp));
-      } else {
         weights_to_channels_last<<<static_cast<unsigned>(std::min<int64_t>((d.O * T * pl.Cp + 255) / 256, 1 << 20)), 256,
                                    0, st>>>(pb, ws, d.O, d.C, T, pl.Cp);
       }
@@ -2062,6 +2135,14 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     wt = ws;
   }
   const int64_t Cp = pl.Cp, taps = d.Kh * d.Kw;
+  if (pl.as_matrix) {   // the copy is the [M, Cp] matrix, the weights [O, Cp]
+    p.K = Cp;
+    p.kblocks = static_cast<int>((Cp + kBK - 1) / kBK);
+    if (!encode_kmajor_sw128(&ma, x, d.M, Cp, kBM) ||
+        !encode_kmajor_sw128(&mb, wt, d.O, Cp, use_pair(kDense, bn, p) ? bn / 2 : bn))
+      return GL_ERR_CUDA;
+    return finish(launch_tc_bn<kDense>(bn, ma, mb, dst, p, st));
+  }
   if (hp.ok) return run_halo(hp, d, Cp, x, wt, dst, relu, st);
   p.K = taps * Cp;
   p.Cp = static_cast<int>(Cp);
