@@ -155,13 +155,15 @@ __global__ void __launch_bounds__(256) weights_to_channels_last(const uint16_t* 
 // Both layout copies of a (C,H,W)-item convolution in ONE launch.
 // Blocks [0, x_blocks): activations (N,C,H,W) -> (N,Hs,Ws,Cp), channels padded with zeros to Cp.  (Hs,Ws) is
 // the whole image, or - for 1x1 windows without padding, which touch only every (Sh,Sw)-th pixel - just
-// those pixels, so that the copy is the [N*H'*W', Cp] matrix itself.  A block moves 64 pixels x 64 channels:
-// pixel-contiguous reads, 16-byte channel-contiguous writes.
+// those pixels, so that the copy is the [N*H'*W', Cp] matrix itself.  A block moves 64 pixels (counted
+// across images, so that small images leave no ragged tiles) x 64 channels: pixel-contiguous reads, 16-byte
+// channel-contiguous writes.
 // Blocks from x_blocks on: weights (O,C,T) -> (O,T,Cp), T = Kh*Kw; a block reads 64 channels x T taps of one
 // filter as one contiguous run and writes T runs of 64 channels.
 struct PrepassParams {
   int C, H, W, Cp, Hs, Ws, Sh, Sw;
-  int tiles_p, tiles_c, x_blocks;   // pixel tiles per image, channel tiles, activation blocks = N * tiles_p * tiles_c
+  int tiles_c, x_blocks;            // channel tiles; activation blocks = pixel tiles * tiles_c
+  int64_t total_pix;                // N * Hs * Ws
   int O, T, wtiles_c;               // weight blocks = O * wtiles_c
 };
 
@@ -187,31 +189,32 @@ __global__ void __launch_bounds__(256) nchw_prepass(const uint16_t* __restrict__
   }
   constexpr int kPitch = 66;                 // elements per staged channel row
   const int tc = b % p.tiles_c;
-  const int tp = (b / p.tiles_c) % p.tiles_p;
-  const int n = b / (p.tiles_c * p.tiles_p);
-  const int c0 = tc * 64, p0 = tp * 64;
+  const int64_t g0 = static_cast<int64_t>(b / p.tiles_c) * 64;   // first pixel of the tile, counted over all images
+  const int c0 = tc * 64;
   const int npix = p.Hs * p.Ws;
+  const int64_t HW = static_cast<int64_t>(p.H) * p.W;
   // reads: a warp takes one channel, its lanes two stretches of 32 consecutive pixels
   {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    int soff[2];
+    const uint16_t* src[2];
     bool pok[2];
 #pragma unroll
     for (int j = 0; j < 2; ++j) {
-      const int pix = p0 + j * 32 + lane;
-      pok[j] = pix < npix;
+      const int64_t gp = g0 + j * 32 + lane;
+      pok[j] = gp < p.total_pix;
+      const int64_t n = gp / npix;
+      const int pix = static_cast<int>(gp - n * npix);
       const int hs = pix / p.Ws, wsx = pix - hs * p.Ws;
-      soff[j] = hs * p.Sh * p.W + wsx * p.Sw;
+      src[j] = x + (n * p.C + c0 + wid) * HW + hs * p.Sh * p.W + wsx * p.Sw;
     }
-    const int64_t HW = static_cast<int64_t>(p.H) * p.W;
     uint16_t v[8][2];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-      const int c = c0 + wid + 8 * i;
+      const bool cok = c0 + wid + 8 * i < p.C;
 #pragma unroll
       for (int j = 0; j < 2; ++j) {
         v[i][j] = 0;
-        if (c < p.C && pok[j]) v[i][j] = x[(static_cast<int64_t>(n) * p.C + c) * HW + soff[j]];
+        if (cok && pok[j]) v[i][j] = src[j][8 * i * HW];
       }
     }
 #pragma unroll
@@ -225,14 +228,15 @@ __global__ void __launch_bounds__(256) nchw_prepass(const uint16_t* __restrict__
   for (int k = 0; k < 2; ++k) {
     const int piece = threadIdx.x + 256 * k;
     const int pl = piece >> 3, cg = piece & 7;
-    const int pix = p0 + pl, c = c0 + cg * 8;
-    if (pix < npix && c < p.Cp) {
+    const int64_t gp = g0 + pl;
+    const int c = c0 + cg * 8;
+    if (gp < p.total_pix && c < p.Cp) {
       uint32_t wd[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i)
         wd[i] = static_cast<uint32_t>(pre_smem[(cg * 8 + 2 * i) * kPitch + pl]) |
                 (static_cast<uint32_t>(pre_smem[(cg * 8 + 2 * i + 1) * kPitch + pl]) << 16);
-      *reinterpret_cast<uint4*>(xs + (static_cast<int64_t>(n) * npix + pix) * p.Cp + c) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+      *reinterpret_cast<uint4*>(xs + gp * p.Cp + c) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
     }
   }
 }
@@ -2111,12 +2115,16 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
       pp.Hs = static_cast<int>(pl.as_matrix ? d.Ho : d.H); pp.Ws = static_cast<int>(pl.as_matrix ? d.Wo : d.W);
       pp.Sh = static_cast<int>(pl.as_matrix ? d.Sh : 1); pp.Sw = static_cast<int>(pl.as_matrix ? d.Sw : 1);
       pp.O = static_cast<int>(d.O); pp.T = static_cast<int>(T);
-      const int64_t tiles_p = (static_cast<int64_t>(pp.Hs) * pp.Ws + 63) / 64, tiles_c = (pl.Cp + 63) / 64;
-      const int64_t x_blocks = d.N * tiles_p * tiles_c, w_blocks = d.O * tiles_c;
+      pp.total_pix = d.N * pp.Hs * pp.Ws;
+      const int64_t tiles_p = (pp.total_pix + 63) / 64, tiles_c = (pl.Cp + 63) / 64;
+      // weights of 1x1 windows with an unpadded channel count already are the [O, C] matrix: no copy
+      const bool copy_w = !(T == 1 && pl.Cp == d.C);
+      const int64_t x_blocks = tiles_p * tiles_c, w_blocks = copy_w ? d.O * tiles_c : 0;
       if (T <= 256 && x_blocks + w_blocks < (1ll << 31) && d.H * d.W < (1ll << 31) && d.C < (1ll << 24)) {
-        pp.tiles_p = static_cast<int>(tiles_p); pp.tiles_c = static_cast<int>(tiles_c);
+        pp.tiles_c = static_cast<int>(tiles_c);
         pp.wtiles_c = static_cast<int>(tiles_c);
         pp.x_blocks = static_cast<int>(x_blocks);
+        if (!copy_w) ws = const_cast<uint16_t*>(pb);
         const size_t smem = std::max<size_t>(64 * 66 * 2, static_cast<size_t>(64 * T * 2));
         nchw_prepass<<<static_cast<unsigned>(x_blocks + w_blocks), 256, smem, st>>>(pa, xs, pb, ws, pp);
       } else if (pl.as_matrix) {
