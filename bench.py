@@ -147,15 +147,17 @@ def cpu_baseline_dense(target_seconds: float = 12.0):
     from paper_2105_09377_b200 import synth
     case = synth.DENSE_4096
     a, b = case.inputs(synth.config_seed(1))
-    t0 = time.perf_counter()
-    brute.rowdot(a, b, np.arange(8))
-    probe = max(time.perf_counter() - t0, 1e-4)
-    rows = int(min(case.m, max(8, 8 * target_seconds / probe)))
-    rows -= rows % 8
-    idx = np.arange(rows, dtype=np.int64)
-    t0 = time.perf_counter()
-    brute.rowdot(a, b, idx)
-    dt = time.perf_counter() - t0
+    brute.rowdot(a, b, np.arange(8))          # first call: library load, thread start
+    rows, dt = 64, 0.0
+    for _ in range(3):                        # grow the sample until it takes a fair share of the target
+        idx = np.arange(rows, dtype=np.int64)
+        t0 = time.perf_counter()
+        brute.rowdot(a, b, idx)
+        dt = max(time.perf_counter() - t0, 1e-4)
+        if rows >= case.m or dt >= target_seconds / 3:
+            break
+        rows = int(min(case.m, max(rows * 2, rows * target_seconds / dt)))
+        rows -= rows % 8
     flops = 2.0 * rows * case.o * case.k
     return {"value": flops / dt / 1e12, "unit": "TFLOP/s", "cores": brute.num_threads(), "kind": "oracle",
             "sample": "rows 0..%d of A (of %d) against all %d rows of B, float64 accumulate, %.1f s" % (rows - 1, case.m, case.o, dt),
