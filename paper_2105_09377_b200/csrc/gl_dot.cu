@@ -28,6 +28,14 @@ namespace {
 
 __device__ unsigned int g_status = 0;   // sticky: set when a bounded wait gives up
 
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start
+// while its predecessor in the stream is still draining.  Everything before pdl_wait (barrier set-up,
+// tensor-memory allocation, descriptor prefetch) touches no global data; pdl_wait returns once the
+// predecessor has completed and its writes are visible.  pdl_launch_dependents lets the successor do the same.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+
 // ------------------------------------------------------------------------
 // General SIMT kernel
 // ------------------------------------------------------------------------
@@ -171,6 +179,8 @@ __global__ void __launch_bounds__(256) nchw_prepass(const uint16_t* __restrict__
                                                     const uint16_t* __restrict__ w, uint16_t* __restrict__ ws,
                                                     const PrepassParams p) {
   extern __shared__ uint16_t pre_smem[];
+  pdl_wait();
+  pdl_launch_dependents();
   int b = blockIdx.x;
   if (b >= p.x_blocks) {
     b -= p.x_blocks;
@@ -593,6 +603,8 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
   else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();
+  pdl_launch_dependents();
 
   const int num_tiles = p.tiles_m * p.tiles_n * p.ksplit;   // work units (p.tiles_m counts 128*CTAS-row tiles)
   const int unit0 = static_cast<int>(blockIdx.x) / CTAS, unit_step = static_cast<int>(gridDim.x) / CTAS;
@@ -961,6 +973,8 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();
+  pdl_launch_dependents();
   const int num_tiles = p.tiles_m * p.tiles_n;
 
   if (warp == 0) {
@@ -1203,6 +1217,8 @@ conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restr
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  pdl_wait();
+  pdl_launch_dependents();
 
   if (warp == 0) {
     // ---------------- producer: the weights once, then Kh row runs per tile ----------------
@@ -1336,6 +1352,8 @@ __global__ void __launch_bounds__(32 * kPackWarps) rowrun_pack(const uint16_t* _
                                                                int W, int Hp, int Wpa, int cp_log2, int ph, int pw, int O,
                                                                int Kh, int Kw, int chunks, int bn) {
   extern __shared__ uint4 padded_rows[];   // [kPackWarps][Wpa * Cp / 8] pieces of 16 bytes
+  pdl_wait();
+  pdl_launch_dependents();
   const int Cp = 1 << cp_log2;
   if (static_cast<int>(blockIdx.x) >= row_blocks) {
     const int total = Kh * chunks * bn * 8;
@@ -1445,6 +1463,35 @@ const DriverApi& driver_api() {
     api.ok = true;
   });
   return api;
+}
+
+// Launch with the programmatic-stream-serialisation attribute (every kernel launched this way calls
+// pdl_wait before its first global access), optionally as clusters of `cluster` blocks.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster,
+                       Args&&... args) {
+  cudaLaunchConfig_t cfg;
+  std::memset(&cfg, 0, sizeof(cfg));
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  std::memset(at, 0, sizeof(at));
+  int n = 0;
+  at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[n].val.programmaticStreamSerializationAllowed = 1;
+  ++n;
+  if (cluster > 1) {
+    at[n].id = cudaLaunchAttributeClusterDimension;
+    at[n].val.clusterDim.x = static_cast<unsigned>(cluster);
+    at[n].val.clusterDim.y = 1;
+    at[n].val.clusterDim.z = 1;
+    ++n;
+  }
+  cfg.attrs = at;
+  cfg.numAttrs = static_cast<unsigned>(n);
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
 int num_sms() {
@@ -1585,13 +1632,14 @@ int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams
   const int tiles = p.tiles_m * p.tiles_n * p.ksplit;
   if (CTAS == 2) {
     const int pairs = std::min(tiles, std::min(max_pairs_dev[dev], num_sms() / 2));
-    cfg.gridDim = dim3(static_cast<unsigned>(2 * pairs));
-    if (cudaLaunchKernelEx(&cfg, dot_tc<BN, MODE, G, OCC, CTAS>, ma, mb, mc, out, p) != cudaSuccess) return GL_ERR_CUDA;
+    if (launch_pdl(dot_tc<BN, MODE, G, OCC, CTAS>, dim3(static_cast<unsigned>(2 * pairs)), dim3(kTcThreads),
+                   Cfg::kSmemBytes, st, 2, ma, mb, mc, out, p) != cudaSuccess)
+      return GL_ERR_CUDA;
     return GL_OK;
   }
   const int grid = tiles < OCC * num_sms() ? tiles : OCC * num_sms();
-  dot_tc<BN, MODE, G, OCC, 1><<<grid, kTcThreads, Cfg::kSmemBytes, st>>>(ma, mb, mc, out, p);
-  return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+  return launch_pdl(dot_tc<BN, MODE, G, OCC, 1>, dim3(static_cast<unsigned>(grid)), dim3(kTcThreads), Cfg::kSmemBytes, st,
+                    1, ma, mb, mc, out, p) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
 }
 
 // Wide tiles of a large problem are bound by operand traffic from L2 to the SMs; a pair of blocks
@@ -1634,6 +1682,8 @@ int pick_bn(int64_t M, int64_t O) {
 // added in index order so that the result does not depend on scheduling; relu applied last.
 __global__ void __launch_bounds__(256) splitk_reduce(const float* __restrict__ part, float* __restrict__ out,
                                                      int64_t n, int planes, int relu) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int64_t n4 = n >> 2;
   const float4* p4 = reinterpret_cast<const float4*>(part);
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
@@ -1831,8 +1881,8 @@ int launch_halo(const CUtensorMap& ma, const CUtensorMap& mb, float* out, const 
   }
   const int tiles = p.tiles_m * p.tiles_n;
   const int grid = std::min(tiles, num_sms());
-  conv_halo<BN><<<grid, kTcThreads, smem, st>>>(ma, mb, out, p);
-  return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+  return launch_pdl(conv_halo<BN>, dim3(static_cast<unsigned>(grid)), dim3(kTcThreads), static_cast<size_t>(smem), st, 1,
+                    ma, mb, out, p) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
 }
 
 int run_halo(const HaloPlan& hp, const DotProblem& d, int64_t Cp, const uint16_t* x, const uint16_t* wt, float* out,
@@ -1996,9 +2046,8 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
   auto finish = [&](int rc_launch) -> int {
     if (rc_launch != GL_OK || tp.ksplit == 1) return rc_launch;
     const int64_t n = d.M * d.O;
-    splitk_reduce<<<static_cast<unsigned>(std::min<int64_t>((n / 4 + 255) / 256, 148 * 8)), 256, 0, st>>>(
-        dst, final_dst, n, tp.ksplit, relu);
-    return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+    return launch_pdl(splitk_reduce, dim3(static_cast<unsigned>(std::min<int64_t>((n / 4 + 255) / 256, 148 * 8))), dim3(256),
+                      0, st, 1, static_cast<const float*>(dst), final_dst, n, tp.ksplit, relu) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
   };
   p.tiles_m = static_cast<int>((d.M + kBM - 1) / kBM);
   p.tiles_n = static_cast<int>((d.O + bn - 1) / bn);
@@ -2031,10 +2080,10 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
       const dim3 pgrid(static_cast<unsigned>(row_blocks + wblocks));
       const size_t psmem = static_cast<size_t>(kPackWarps * pl.Wpa * pl.rr_cp * 2);
 #define GL_ROWRUN_PACK(CT)                                                                                              \
-  rowrun_pack<CT><<<pgrid, 32 * kPackWarps, psmem, st>>>(                                                              \
-      pa, xs, pb, ws, d.channels_last ? 1 : 0, row_blocks, rows, static_cast<int>(d.H), static_cast<int>(d.W),         \
-      static_cast<int>(pl.Hp), static_cast<int>(pl.Wpa), cp_log2, static_cast<int>(d.ph_lo), static_cast<int>(d.pw_lo), \
-      static_cast<int>(d.O), static_cast<int>(d.Kh), static_cast<int>(d.Kw), chunks, pl.rr_bn)
+  launch_pdl(rowrun_pack<CT>, pgrid, dim3(32 * kPackWarps), psmem, st, 1, pa, xs, pb, ws, d.channels_last ? 1 : 0,       \
+             row_blocks, rows, static_cast<int>(d.H), static_cast<int>(d.W), static_cast<int>(pl.Hp),                  \
+             static_cast<int>(pl.Wpa), cp_log2, static_cast<int>(d.ph_lo), static_cast<int>(d.pw_lo),                  \
+             static_cast<int>(d.O), static_cast<int>(d.Kh), static_cast<int>(d.Kw), chunks, pl.rr_bn)
       switch (d.C) {
         case 1: GL_ROWRUN_PACK(1); break;
         case 2: GL_ROWRUN_PACK(2); break;
@@ -2074,9 +2123,9 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
         attr_set_dev[dev] = true;
       }
       const int grid = std::min(rp.tiles, 2 * num_sms());
-      conv_rowrun<<<grid, kRunThreads, smem, st>>>(reinterpret_cast<const unsigned char*>(xs),
-                                                    reinterpret_cast<const unsigned char*>(ws), mc, rp);
-      return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+      return launch_pdl(conv_rowrun, dim3(static_cast<unsigned>(grid)), dim3(kRunThreads), static_cast<size_t>(smem), st, 1,
+                        reinterpret_cast<const unsigned char*>(xs), reinterpret_cast<const unsigned char*>(ws), mc,
+                        rp) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
     }
     if (pl.rowwin) {
       rowwin_pack_x<<<static_cast<unsigned>(d.N * pl.Hp), 256, 0, st>>>(
@@ -2126,7 +2175,9 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
         pp.x_blocks = static_cast<int>(x_blocks);
         if (!copy_w) ws = const_cast<uint16_t*>(pb);
         const size_t smem = std::max<size_t>(64 * 66 * 2, static_cast<size_t>(64 * T * 2));
-        nchw_prepass<<<static_cast<unsigned>(x_blocks + w_blocks), 256, smem, st>>>(pa, xs, pb, ws, pp);
+        if (launch_pdl(nchw_prepass, dim3(static_cast<unsigned>(x_blocks + w_blocks)), dim3(256), smem, st, 1, pa, xs, pb,
+                       ws, pp) != cudaSuccess)
+          return GL_ERR_CUDA;
       } else if (pl.as_matrix) {
         return GL_ERR_UNSUPPORTED;
       } else {
