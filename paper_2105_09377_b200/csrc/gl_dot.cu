@@ -21,6 +21,7 @@
 #include <mutex>
 
 #include "gl_internal.h"
+#include "gl_launch.cuh"
 
 using namespace gl;
 
@@ -28,12 +29,6 @@ namespace {
 
 __device__ unsigned int g_status = 0;   // sticky: set when a bounded wait gives up
 
-// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start
-// while its predecessor in the stream is still draining.  Everything before pdl_wait (barrier set-up,
-// tensor-memory allocation, descriptor prefetch) touches no global data; pdl_wait returns once the
-// predecessor has completed and its writes are visible.  pdl_launch_dependents lets the successor do the same.
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 
 // ------------------------------------------------------------------------
@@ -1463,35 +1458,6 @@ const DriverApi& driver_api() {
     api.ok = true;
   });
   return api;
-}
-
-// Launch with the programmatic-stream-serialisation attribute (every kernel launched this way calls
-// pdl_wait before its first global access), optionally as clusters of `cluster` blocks.
-template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, int cluster,
-                       Args&&... args) {
-  cudaLaunchConfig_t cfg;
-  std::memset(&cfg, 0, sizeof(cfg));
-  cfg.gridDim = grid;
-  cfg.blockDim = block;
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cudaLaunchAttribute at[2];
-  std::memset(at, 0, sizeof(at));
-  int n = 0;
-  at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  at[n].val.programmaticStreamSerializationAllowed = 1;
-  ++n;
-  if (cluster > 1) {
-    at[n].id = cudaLaunchAttributeClusterDimension;
-    at[n].val.clusterDim.x = static_cast<unsigned>(cluster);
-    at[n].val.clusterDim.y = 1;
-    at[n].val.clusterDim.z = 1;
-    ++n;
-  }
-  cfg.attrs = at;
-  cfg.numAttrs = static_cast<unsigned>(n);
-  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
 int num_sms() {

@@ -12,6 +12,7 @@
 #include <cstring>
 
 #include "gl_internal.h"
+#include "gl_launch.cuh"
 
 using namespace gl;
 
@@ -73,6 +74,8 @@ __global__ void __launch_bounds__(kThreads) transpose_tiled_vec(const T* __restr
                                                                 const TileParams p) {
   constexpr int TILE = 16 * VEC;
   __shared__ uint4 tile[TILE][16];
+  pdl_wait();
+  pdl_launch_dependents();
   int64_t bid = blockIdx.x;
   const int64_t tileA = bid % p.tilesA; bid /= p.tilesA;
   const int64_t tileB = bid % p.tilesB; bid /= p.tilesB;
@@ -230,7 +233,9 @@ int run_transpose(const gl_ap* in, const int32_t* perm, gl_ap* out, cudaStream_t
   p.tilesB = (p.sizeB + tile - 1) / tile;
   const int64_t blocks = p.tilesA * p.tilesB * nbatch;
   if (blocks > 0x7FFFFFFF) return GL_ERR_UNSUPPORTED;
-  if (vec) transpose_tiled_vec<T, VEC><<<static_cast<unsigned>(blocks), kThreads, 0, st>>>(src, dst, p);
+  if (vec)
+    return launch_pdl(transpose_tiled_vec<T, VEC>, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, st, 1, src, dst,
+                      p) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
   else transpose_tiled_scalar<T><<<static_cast<unsigned>(blocks), kThreads, 0, st>>>(src, dst, p);
   return launch_status();
 }
@@ -257,6 +262,8 @@ __global__ void __launch_bounds__(kThreads) pad_kernel(const V* __restrict__ in,
 template <typename T>
 __global__ void __launch_bounds__(kThreads) pad_rows(const T* __restrict__ in, T* __restrict__ out, int64_t rows,
                                                      int d_in, int lo, int d_out, T fill) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int lane = threadIdx.x & 31;
   const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
   for (int64_t r = blockIdx.x * (int64_t)(blockDim.x >> 5) + (threadIdx.x >> 5); r < rows; r += warps) {
@@ -347,6 +354,8 @@ template <typename T, int VEC>
 __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in, T* __restrict__ out,
                                                         const Im2colParams p, T fill) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  pdl_wait();
+  pdl_launch_dependents();
   int* lut = reinterpret_cast<int*>(smem_raw);                     // K entries: staged offset of column k at w'=0
   T* stage = reinterpret_cast<T*>(smem_raw + (((p.K + p.C * p.Kh) * 4 + 15) / 16) * 16);   // [C*Kh][pitch]
   const int64_t n = blockIdx.x / p.Ho, ho = blockIdx.x % p.Ho;
@@ -579,6 +588,8 @@ struct Pool3s2 {
 template <int R>
 __global__ void __launch_bounds__(256) window_max_3x3s2(const float* __restrict__ in, float* __restrict__ out,
                                                          const Pool3s2 p, float fill) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int64_t u = blockIdx.x * (int64_t)blockDim.y + threadIdx.y;
   if (u >= p.units) return;
   const int64_t plane = u / p.strips;
@@ -634,6 +645,8 @@ __global__ void __launch_bounds__(kThreads) item_max(const float* __restrict__ i
 }
 
 __global__ void __launch_bounds__(kThreads) relu_vec(const float4* __restrict__ in, float4* __restrict__ out, int64_t n4) {
+  pdl_wait();
+  pdl_launch_dependents();
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
     float4 v = in[i];
     v.x = v.x > 0.f ? v.x : 0.f;
@@ -776,8 +789,8 @@ int run_windows(const gl_ap* in, const gl_windows* w, const gl_ap& A, gl_ap* out
       int dev = 0;
       if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return GL_ERR_CUDA;
       if (!allow_big_smem(kern, &attr_done[dev][vec ? 1 : 0])) return GL_ERR_CUDA;
-      kern<<<static_cast<unsigned>(blocks), kThreads, static_cast<size_t>(smem), st>>>(src, dst, p, fill);
-      return launch_status();
+      return launch_pdl(kern, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), static_cast<size_t>(smem), st, 1, src,
+                        dst, p, fill) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
     }
   }
   WinParams p;
@@ -833,11 +846,13 @@ int gl_access_pad(const gl_ap* in, int32_t dim, int64_t lo, int64_t hi, int32_t 
   } else if (inner == 1 && d_out < (1ll << 30)) {
     const unsigned blocks = static_cast<unsigned>(std::min<int64_t>((outer + 7) / 8, 148 * 32));
     if (in->dtype == GL_F32)
-      pad_rows<uint32_t><<<blocks, kThreads, 0, st>>>(static_cast<const uint32_t*>(in->data), static_cast<uint32_t*>(out->data),
-                                                      outer, (int)d_in, (int)lo, (int)d_out, Fill<uint32_t>::value(pad_kind));
+      return launch_pdl(pad_rows<uint32_t>, dim3(blocks), dim3(kThreads), 0, st, 1, static_cast<const uint32_t*>(in->data),
+                        static_cast<uint32_t*>(out->data), outer, (int)d_in, (int)lo, (int)d_out,
+                        Fill<uint32_t>::value(pad_kind)) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
     else
-      pad_rows<uint16_t><<<blocks, kThreads, 0, st>>>(static_cast<const uint16_t*>(in->data), static_cast<uint16_t*>(out->data),
-                                                      outer, (int)d_in, (int)lo, (int)d_out, Fill<uint16_t>::value(pad_kind));
+      return launch_pdl(pad_rows<uint16_t>, dim3(blocks), dim3(kThreads), 0, st, 1, static_cast<const uint16_t*>(in->data),
+                        static_cast<uint16_t*>(out->data), outer, (int)d_in, (int)lo, (int)d_out,
+                        Fill<uint16_t>::value(pad_kind)) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
   } else if (in->dtype == GL_F32) {
     pad_kernel<uint32_t><<<grid_for(outer * d_out * inner, kThreads), kThreads, 0, st>>>(
         static_cast<const uint32_t*>(in->data), static_cast<uint32_t*>(out->data), outer, d_in, lo, d_out, inner,
@@ -903,8 +918,8 @@ int gl_compute_reduce_max(const gl_ap* in, const gl_windows* w, gl_ap* out, void
     t.units = prod(in->shape, 0, na) * t.strips;
     const int64_t blocks = (t.units + 7) / 8;
     if (blocks <= 0x7FFFFFFF) {
-      window_max_3x3s2<kRows><<<static_cast<unsigned>(blocks), dim3(32, 8), 0, st>>>(src, dst, t, fill);
-      return launch_status();
+      return launch_pdl(window_max_3x3s2<kRows>, dim3(static_cast<unsigned>(blocks)), dim3(32, 8), 0, st, 1, src, dst, t,
+                        fill) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
     }
   }
   if (w->n == 2 && in->shape[na] < (1 << 20) && in->shape[na + 1] < (1 << 20) && w->wshape[0] < 1024 &&
@@ -1037,8 +1052,9 @@ int gl_compute_relu(const gl_ap* in, gl_ap* out, void* stream) {
   if (n4) {
     int64_t blocks = (n4 + kThreads - 1) / kThreads;
     if (blocks > 148 * 16) blocks = 148 * 16;
-    relu_vec<<<static_cast<unsigned>(blocks), kThreads, 0, st>>>(reinterpret_cast<const float4*>(src),
-                                                               reinterpret_cast<float4*>(dst), n4);
+    if (launch_pdl(relu_vec, dim3(static_cast<unsigned>(blocks)), dim3(kThreads), 0, st, 1,
+                   reinterpret_cast<const float4*>(src), reinterpret_cast<float4*>(dst), n4) != cudaSuccess)
+      return GL_ERR_CUDA;
   }
   if (n % 4) relu_tail<<<1, 4, 0, st>>>(src, dst, n4 * 4, n);
   return launch_status();
