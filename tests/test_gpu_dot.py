@@ -300,6 +300,57 @@ def test_conv_resident_window_tiles_bit_exact(gl, case):
     assert np.array_equal(got.astype(np.float64), ref)
 
 
+# Few input channels (C <= 8 / Sw): windows read in place from runs of the padded rows.
+# n, c, h, w, o, kh, kw, sh, sw, ph, pw
+CONV_ROW_RUNS = [
+    (2, 3, 30, 300, 64, 7, 7, 2, 2, 3, 3),     # RGB stem, three 128-column segments per output row
+    (1, 8, 12, 40, 128, 3, 3, 1, 1, 1, 1),     # stride 1: 8-channel pixels, widest tile
+    (2, 4, 17, 33, 20, 5, 5, 3, 2, 2, 2),      # odd sizes, O = 20 (MMA N = 32)
+    (2, 2, 16, 64, 12, 3, 6, 1, 4, 1, 0),      # stride 4: 2-channel pixels
+    (1, 1, 20, 80, 8, 2, 20, 2, 8, 0, 4),      # stride 8: 1-channel pixels, two MMAs per filter row
+    (3, 1, 9, 9, 4, 3, 3, 1, 1, 1, 1),         # one channel, stride 1
+]
+
+
+@pytest.mark.parametrize("case", CONV_ROW_RUNS, ids=lambda c: "x".join(map(str, c)))
+def test_conv_row_runs_bit_exact(gl, case):
+    n, c, h, w, o, kh, kw, sh, sw, ph, pw = case
+    x = synth.uniform_int(40, 1, (n, c, h, w), -3, 3)
+    wt = synth.uniform_int(40, 2, (o, c, kh, kw), -3, 3)
+    ref = _conv_ref(x, wt, (sh, sw), (ph, pw))
+    for cl in (False, True):
+        got = _conv_gpu(gl, x, wt, (sh, sw), (ph, pw), channels_last=cl, flags=gl.GL_EPILOGUE_RELU if cl else 0)
+        assert got.shape == ref.shape
+        assert np.array_equal(got.astype(np.float64), np.maximum(ref, 0.0) if cl else ref), "channels_last=%s" % cl
+    again = _conv_gpu(gl, x, wt, (sh, sw), (ph, pw), channels_last=False)
+    assert np.array_equal(again.astype(np.float64), ref)           # the scratch copies are rebuilt on every call
+
+
+# 1x1 unpadded windows over (C,H,W) items: the layout copy keeps only the pixels the windows touch.
+CONV_1X1_CHW = [
+    (2, 64, 9, 11, 72, 2, 3),      # n, c, h, w, o, sh, sw
+    (3, 96, 8, 8, 40, 1, 1),       # C = 96: second chunk half empty
+    (1, 200, 7, 7, 260, 1, 1),     # C not a multiple of 64, O spans tiles
+    (2, 128, 10, 10, 64, 2, 2),
+]
+
+
+@pytest.mark.parametrize("case", CONV_1X1_CHW, ids=lambda c: "x".join(map(str, c)))
+def test_conv_1x1_chw_items_bit_exact(gl, case):
+    n, c, h, w, o, sh, sw = case
+    x = synth.uniform_int(41, 1, (n, c, h, w), -3, 3)
+    wt = synth.uniform_int(41, 2, (o, c, 1, 1), -3, 3)
+    ref = _conv_ref(x, wt, (sh, sw), (0, 0))
+    got = _conv_gpu(gl, x, wt, (sh, sw), (0, 0), channels_last=False)
+    assert got.shape == ref.shape
+    assert np.array_equal(got.astype(np.float64), ref)
+    # with the fused squeeze + transpose the same items take the general window path
+    out = gl.gl_cartesian_dot(gl.AccessPattern(to_bf16_device(x), 1), gl.windows_spec((c, 1, 1), (1, sh, sw)),
+                              gl.AccessPattern(to_bf16_device(wt), 1), flags=gl.GL_OUT_NCHW)
+    _ok(gl)
+    assert np.array_equal(out.tensor.cpu().numpy().astype(np.float64), ref.transpose(0, 3, 1, 2))
+
+
 def test_dense_interpreter_program_with_relu(gl):
     a = synth.uniform_int(32, 1, (20, 16), -3, 3)
     b = synth.uniform_int(32, 2, (12, 16), -3, 3)
