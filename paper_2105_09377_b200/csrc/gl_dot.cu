@@ -161,13 +161,13 @@ __global__ void __launch_bounds__(256) weights_to_channels_last(const uint16_t* 
 // those pixels, so that the copy is the [N*H'*W', Cp] matrix itself.  A block moves 64 pixels (counted
 // across images, so that small images leave no ragged tiles) x 64 channels: pixel-contiguous reads, 16-byte
 // channel-contiguous writes.
-// Blocks from x_blocks on: weights (O,C,T) -> (O,T,Cp), T = Kh*Kw; a block reads 64 channels x T taps of one
-// filter as one contiguous run and writes T runs of 64 channels.
+// Blocks from x_blocks on: weights (O,C,T) -> (O,T,Cp), T = Kh*Kw; a WARP takes 64 channels x T taps of one
+// filter: one contiguous run read with 16-byte loads, T runs of 64 channels written as 16-byte pieces.
 struct PrepassParams {
   int C, H, W, Cp, Hs, Ws, Sh, Sw;
   int tiles_c, x_blocks;            // channel tiles; activation blocks = pixel tiles * tiles_c
   int64_t total_pix;                // N * Hs * Ws
-  int O, T, wtiles_c;               // weight blocks = O * wtiles_c
+  int O, T, wtiles_c, wwarps;       // weight units = O * wtiles_c, wwarps of them per block
 };
 
 __global__ void __launch_bounds__(256) nchw_prepass(const uint16_t* __restrict__ x, uint16_t* __restrict__ xs,
@@ -178,17 +178,34 @@ __global__ void __launch_bounds__(256) nchw_prepass(const uint16_t* __restrict__
   pdl_launch_dependents();
   int b = blockIdx.x;
   if (b >= p.x_blocks) {
-    b -= p.x_blocks;
-    const int o = b / p.wtiles_c, c0 = (b - o * p.wtiles_c) * 64;
-    const int nc = min(64, p.C - c0);        // channels with data (may be <= 0 in the padded tail)
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    if (wid >= p.wwarps) return;
+    const int unit = (b - p.x_blocks) * p.wwarps + wid;
+    if (unit >= p.O * p.wtiles_c) return;
+    const int o = unit / p.wtiles_c, c0 = (unit - o * p.wtiles_c) * 64;
+    const int nc = max(0, min(64, p.C - c0));   // channels with data (none in a fully padded tail)
+    const int run = nc * p.T;                    // contiguous elements of this filter and channel tile
     const uint16_t* src = w + (static_cast<int64_t>(o) * p.C + c0) * p.T;
-    for (int e = threadIdx.x; e < nc * p.T; e += blockDim.x) pre_smem[e] = src[e];
-    __syncthreads();
-    const int ncp = min(64, p.Cp - c0);
-    uint16_t* dst = ws + static_cast<int64_t>(o) * p.T * p.Cp + c0;
-    for (int e = threadIdx.x; e < p.T * 64; e += blockDim.x) {
-      const int t = e >> 6, c = e & 63;
-      if (c < ncp) dst[static_cast<int64_t>(t) * p.Cp + c] = c < nc ? pre_smem[c * p.T + t] : static_cast<uint16_t>(0);
+    uint16_t* mine = pre_smem + wid * 64 * p.T;
+    const bool vec_in = (reinterpret_cast<uintptr_t>(src) & 15u) == 0;
+    const int nvec = vec_in ? run >> 3 : 0;
+    for (int v = lane; v < nvec; v += 32) reinterpret_cast<uint4*>(mine)[v] = reinterpret_cast<const uint4*>(src)[v];
+    for (int e = nvec * 8 + lane; e < run; e += 32) mine[e] = src[e];
+    __syncwarp();
+    // output pieces: tap t, channels c0 + 8 g .. + 7; channels past C are zeros
+    const int groups = (min(64, p.Cp - c0) + 7) >> 3;
+    for (int piece = lane; piece < p.T * 8; piece += 32) {
+      const int t = piece >> 3, g = piece & 7;
+      if (g < groups) {
+        uint32_t wd[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int ca = g * 8 + 2 * i, cb = ca + 1;
+          const uint32_t lo = ca < nc ? mine[ca * p.T + t] : 0u, hi = cb < nc ? mine[cb * p.T + t] : 0u;
+          wd[i] = lo | (hi << 16);
+        }
+        *reinterpret_cast<uint4*>(ws + (static_cast<int64_t>(o) * p.T + t) * p.Cp + c0 + g * 8) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+      }
     }
     return;
   }
@@ -2134,13 +2151,15 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
       const int64_t tiles_p = (pp.total_pix + 63) / 64, tiles_c = (pl.Cp + 63) / 64;
       // weights of 1x1 windows with an unpadded channel count already are the [O, C] matrix: no copy
       const bool copy_w = !(T == 1 && pl.Cp == d.C);
-      const int64_t x_blocks = tiles_p * tiles_c, w_blocks = copy_w ? d.O * tiles_c : 0;
+      const int wwarps = static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(8, (32 * 1024) / (64 * T * 2))));
+      const int64_t x_blocks = tiles_p * tiles_c, w_blocks = copy_w ? (d.O * tiles_c + wwarps - 1) / wwarps : 0;
       if (T <= 256 && x_blocks + w_blocks < (1ll << 31) && d.H * d.W < (1ll << 31) && d.C < (1ll << 24)) {
         pp.tiles_c = static_cast<int>(tiles_c);
         pp.wtiles_c = static_cast<int>(tiles_c);
+        pp.wwarps = wwarps;
         pp.x_blocks = static_cast<int>(x_blocks);
         if (!copy_w) ws = const_cast<uint16_t*>(pb);
-        const size_t smem = std::max<size_t>(64 * 66 * 2, static_cast<size_t>(64 * T * 2));
+        const size_t smem = std::max<size_t>(64 * 66 * 2, static_cast<size_t>(wwarps) * 64 * T * 2);
         if (launch_pdl(nchw_prepass, dim3(static_cast<unsigned>(x_blocks + w_blocks)), dim3(256), smem, st, 1, pa, xs, pb,
                        ws, pp) != cudaSuccess)
           return GL_ERR_CUDA;
