@@ -215,8 +215,29 @@ __global__ void __launch_bounds__(256) nchw_prepass(const uint16_t* __restrict__
   const int c0 = tc * 64;
   const int npix = p.Hs * p.Ws;
   const int64_t HW = static_cast<int64_t>(p.H) * p.W;
-  // reads: a warp takes one channel, its lanes two stretches of 32 consecutive pixels
-  {
+  // reads.  Whole images with a pixel count that is a multiple of 4: a thread loads 4 consecutive pixels
+  // (8 bytes) of 4 channels.  Otherwise: a warp takes one channel, its lanes two stretches of 32 pixels.
+  const bool wide = p.Sh == 1 && p.Sw == 1 && p.Hs == p.H && p.Ws == p.W && (npix & 3) == 0 &&
+                    (reinterpret_cast<uintptr_t>(x) & 7u) == 0;
+  if (wide) {
+    const int pg = threadIdx.x & 15, cs = threadIdx.x >> 4;
+    const int64_t gp = g0 + 4 * pg;
+    const bool pok = gp < p.total_pix;
+    const int64_t n = gp / npix;
+    const uint16_t* src = x + (n * p.C + c0 + cs) * HW + (gp - n * npix);
+    uint2 v[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[i] = make_uint2(0u, 0u);
+      if (pok && c0 + cs + 16 * i < p.C) v[i] = *reinterpret_cast<const uint2*>(src + 16 * i * HW);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint32_t* dst = reinterpret_cast<uint32_t*>(pre_smem + (cs + 16 * i) * kPitch + 4 * pg);
+      dst[0] = v[i].x;
+      dst[1] = v[i].y;
+    }
+  } else {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const uint16_t* src[2];
     bool pok[2];
