@@ -266,10 +266,23 @@ __global__ void __launch_bounds__(kThreads) pad_rows(const T* __restrict__ in, T
   pdl_launch_dependents();
   const int lane = threadIdx.x & 31;
   const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-  for (int64_t r = blockIdx.x * (int64_t)(blockDim.x >> 5) + (threadIdx.x >> 5); r < rows; r += warps) {
-    const T* src = in + r * d_in - lo;
-    T* dst = out + r * d_out;
-    for (int x = lane; x < d_out; x += 32) dst[x] = (x >= lo && x < lo + d_in) ? src[x] : fill;
+  // a warp takes four rows per trip (rows r, r + warps, ...): four loads in flight per lane before any store
+  for (int64_t r = blockIdx.x * (int64_t)(blockDim.x >> 5) + (threadIdx.x >> 5); r < rows; r += 4 * warps) {
+    for (int x = lane; x < d_out; x += 32) {
+      const bool inside = x >= lo && x < lo + d_in;
+      T v[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int64_t rr = r + j * warps;
+        v[j] = fill;
+        if (inside && rr < rows) v[j] = in[rr * d_in - lo + x];
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int64_t rr = r + j * warps;
+        if (rr < rows) out[rr * d_out + x] = v[j];
+      }
+    }
   }
 }
 
@@ -647,13 +660,23 @@ __global__ void __launch_bounds__(kThreads) item_max(const float* __restrict__ i
 __global__ void __launch_bounds__(kThreads) relu_vec(const float4* __restrict__ in, float4* __restrict__ out, int64_t n4) {
   pdl_wait();
   pdl_launch_dependents();
-  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
-    float4 v = in[i];
-    v.x = v.x > 0.f ? v.x : 0.f;
-    v.y = v.y > 0.f ? v.y : 0.f;
-    v.z = v.z > 0.f ? v.z : 0.f;
-    v.w = v.w > 0.f ? v.w : 0.f;
-    out[i] = v;
+  // four independent 16-byte loads in flight per thread
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += 4 * stride) {
+    float4 v[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (i + j * stride < n4) v[j] = in[i + j * stride];
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (i + j * stride < n4) {
+        float4 r = v[j];
+        r.x = r.x > 0.f ? r.x : 0.f;
+        r.y = r.y > 0.f ? r.y : 0.f;
+        r.z = r.z > 0.f ? r.z : 0.f;
+        r.w = r.w > 0.f ? r.w : 0.f;
+        out[i + j * stride] = r;
+      }
   }
 }
 
