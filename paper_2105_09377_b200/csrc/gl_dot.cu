@@ -609,6 +609,12 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // position in the pair: block 0 owns the barriers both blocks feed and issues the MMAs
   const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;
+  // the tensor maps are kernel parameters: their fetch starts now, under the set-up
+  if (threadIdx.x == 32) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+    if (p.tma_store) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_c)) : "memory");
+  }
 
   if (threadIdx.x == 0) {
     // full: the two producer threads of block 0 announce the bytes of the whole pair
@@ -647,7 +653,6 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
     // (issuing one TMA load costs its thread 150-200 cycles; two issuing warps halve that)
     const bool load_a = warp == 0;
     if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(load_a ? &map_a : &map_b)) : "memory");
       uint32_t s = 0, ph = 0;   // ring slot and its phase, advanced by hand (no division in this thread)
       bool ok = true;
       for (int u = unit0; u < num_tiles && ok; u += unit_step) {
@@ -798,7 +803,6 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
     bool ok = true;
     const bool vec_ok = (p.O & 3) == 0;
     const uint32_t stage_buf = epi_base + q * (Cfg::kEpiBufs * 4096);   // this warp's 32 rows x 128 bytes tiles
-    if (p.tma_store && lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_c)) : "memory");
     for (int u = unit0; u < num_tiles && ok; u += unit_step, ++tile_it) {
       const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
       uint32_t t, ks, tmu, tnu;
@@ -988,6 +992,10 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   static_assert((4 * kHaloMaxStages + 4) * 8 + 8 <= kHaloBarBytes, "barrier block too small");
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 32) {   // the tensor maps are kernel parameters: their fetch starts under the set-up
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
+  }
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.sa_stages; ++s) { mbar_init(bar_afull + 8 * s, 1); mbar_init(bar_aempty + 8 * s, 1); }
     for (int s = 0; s < p.sb_stages; ++s) { mbar_init(bar_bfull + 8 * s, 1); mbar_init(bar_bempty + 8 * s, 1); }
@@ -1013,7 +1021,6 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   if (warp == 0) {
     // ---------------- A producer: one input box per (tile, 64-channel chunk) ----------------
     if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
       uint32_t s = 0, ph = 0;
       bool ok = true;
       for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x) {
@@ -1032,7 +1039,6 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   } else if (warp == 6) {
     // ---------------- B producer: stages in (chunk, tap group) order; once per block when resident ----------------
     if (lane == 0) {
-      asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
       uint32_t s = 0, ph = 0;
       bool ok = true;
       for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x) {
@@ -1233,6 +1239,7 @@ conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restr
   const uint32_t tmem_cols = 2 * p.bn <= 32 ? 32u : (2 * p.bn <= 64 ? 64u : (2 * p.bn <= 128 ? 128u : 256u));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 64) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_c)) : "memory");
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, 4); }
@@ -1313,7 +1320,6 @@ conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restr
     const int q = warp & 3;
     uint32_t tile_it = 0, chunk_it = 0;
     bool ok = true;
-    if (lane == 0) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_c)) : "memory");
     for (int u = blockIdx.x; u < p.tiles && ok; u += gridDim.x, ++tile_it) {
       const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
       uint32_t row, seg;
