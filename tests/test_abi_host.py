@@ -164,3 +164,32 @@ def test_blocking_transformer_shapes(gl, golden_dir):
     assert gl.LIB.gl_shape_slice(ct.byref(am), 2, 3, 3, ct.byref(out)) == 4          # empty range
     assert gl.LIB.gl_shape_concat(ct.byref(am), ct.byref(m((2, 4, 4, 5), 2, gl.GL_F32)), 2, ct.byref(out)) == 4
     assert gl.LIB.gl_shape_squeeze(ct.byref(am), 0, ct.byref(out)) == 4
+
+
+def test_scratch_sizes_follow_the_layout_rules(gl):
+    """gl_cartesian_dot_workspace is pure host arithmetic: the bytes it asks for are those of the layout
+    copies each kind of convolution makes (checked against the sizes written out by hand)."""
+    def need(x_shape, w_shape, spec, flags=0):
+        a = gl._meta(x_shape, 1, gl.GL_BF16)
+        b = gl._meta(w_shape, 1, gl.GL_BF16)
+        return int(gl.LIB.gl_cartesian_dot_workspace(ctypes.byref(a), ctypes.byref(spec), ctypes.byref(b), flags))
+
+    def up(v, a=1024):
+        return (v + a - 1) // a * a
+
+    # channels-last items with a channel count that is a multiple of 8: nothing to copy
+    assert need((32, 56, 56, 64), (64, 3, 3, 64), gl.windows_spec((3, 3, 64), (1, 1, 1), (1, 1, 0), (1, 1, 0))) == 0
+    # (C,H,W) items, 3x3: channels-last copies of the activations and of the weights
+    spec = gl.windows_spec((128, 3, 3), (1, 1, 1), (0, 1, 1), (0, 1, 1))
+    assert need((32, 128, 28, 28), (128, 128, 3, 3), spec) == up(32 * 28 * 28 * 128 * 2) + up(128 * 9 * 128 * 2)
+    # (C,H,W) items, 1x1 stride 2, no pad: only the pixels the windows touch, weights [O, C]
+    spec = gl.windows_spec((256, 1, 1), (1, 2, 2))
+    assert need((32, 256, 56, 56), (128, 256, 1, 1), spec) == up(32 * 28 * 28 * 256 * 2) + up(128 * 256 * 2)
+    # RGB stem, stride 2: 4-channel pixels in zero-bordered rows (230 rows of 230 pixels, plus slack for the
+    # runs of the columns past W'), weights as 7 filter rows x 4 chunks x 64 rows x 16 bytes
+    for shape, wshape, spec in (((32, 3, 224, 224), (64, 3, 7, 7), gl.windows_spec((3, 7, 7), (1, 2, 2), (0, 3, 3), (0, 3, 3))),
+                                ((32, 224, 224, 3), (64, 7, 7, 3), gl.windows_spec((7, 7, 3), (2, 2, 1), (3, 3, 0), (3, 3, 0)))):
+        assert need(shape, wshape, spec) == up(32 * 230 * 230 * 4 * 2 + 128 * 16 + 4096) + up(7 * 4 * 64 * 16)
+    # small M, long K: partial planes of the split contraction (26 tiles of 128x256 -> 5 slices of 15 K blocks)
+    spec = gl.windows_spec((3, 3, 512), (1, 1, 1), (1, 1, 0), (1, 1, 0))
+    assert need((32, 7, 7, 512), (512, 3, 3, 512), spec) == up(5 * 1568 * 512 * 4)

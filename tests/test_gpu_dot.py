@@ -332,6 +332,7 @@ CONV_1X1_CHW = [
     (3, 96, 8, 8, 40, 1, 1),       # C = 96: second chunk half empty
     (1, 200, 7, 7, 260, 1, 1),     # C not a multiple of 64, O spans tiles
     (2, 128, 10, 10, 64, 2, 2),
+    (1, 2048, 7, 7, 64, 1, 1),     # one tile, 32 K blocks: the contraction is split and summed by the second kernel
 ]
 
 
