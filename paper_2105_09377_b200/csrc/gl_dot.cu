@@ -966,8 +966,10 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
 
 // BN: output channels per tile.  The weights are viewed as (64 channels, O, chunk, tap); one TMA box
 // brings the BN x 64 slices of p.tg consecutive taps of one chunk.
-template <int BN>
-__global__ void __launch_bounds__(kTcThreads, 1)
+// OCC = 2 (64-wide tiles): two blocks per SM, each with one input-box stage, so that one block's loads and
+// epilogue run under the other's MMAs.
+template <int BN, int OCC>
+__global__ void __launch_bounds__(kTcThreads, OCC)
 conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
           float* __restrict__ out, const HaloParams p) {
   constexpr int kSubB = BN * kBK * 2;       // one tap of B
@@ -1808,6 +1810,7 @@ ConvPlan plan_conv(const DotProblem& d, uint32_t flags) {
 struct HaloPlan {
   bool ok = false;
   int bn = 64, Wb = 0, R = 0, RB = 0, tiles_per_img = 0, sa = 0, sb = 0, resident = 0, tg = 1;
+  int occ = 1;   // blocks per SM the shared-memory plan is made for
 };
 
 HaloPlan plan_halo(const DotProblem& d, const ConvPlan& pl, uint32_t flags) {
@@ -1815,9 +1818,6 @@ HaloPlan plan_halo(const DotProblem& d, const ConvPlan& pl, uint32_t flags) {
   if (!d.conv || !pl.tc || pl.rowwin || (flags & GL_OUT_NCHW)) return hp;
   if (d.Sh != 1 || d.Sw != 1 || pl.Cp % kBK != 0 || d.O % 4 != 0) return hp;
   if (d.Kh == 1 && d.Kw == 1) return hp;   // no overlap between windows: nothing to keep
-  // 64-wide tiles are bound by the issue rate of N = 64 MMAs either way, and there two blocks per SM
-  // (the im2col-mode kernel) hide start-up and epilogue better than one resident block (measured)
-  if (d.O <= 64) return hp;
   const int64_t Wb = d.W + d.pw_lo + d.pw_hi;
   // the MMA of the last tap reads 128 rows starting (Kh-1)*Wb + Kw-1 rows into the stage
   if (Wb > 256 || (d.Kh - 1) * Wb + d.Kw - 1 + kBM > kHaloARows) return hp;
@@ -1827,7 +1827,7 @@ HaloPlan plan_halo(const DotProblem& d, const ConvPlan& pl, uint32_t flags) {
   // rows of the 128-row tiles that hold real outputs; small images fill too little of a tile
   if (10 * d.Ho * d.Wo < 6 * tpi * kBM) return hp;
   if (d.N * tpi * ((d.O + 63) / 64) >= (1ll << 28) || d.N >= (1ll << 30) || d.H >= (1ll << 30)) return hp;
-  hp.bn = 128;
+  hp.bn = d.O > 64 ? 128 : 64;
   hp.Wb = static_cast<int>(Wb);
   hp.R = static_cast<int>(R);
   hp.RB = static_cast<int>(R + d.Kh - 1);
@@ -1837,6 +1837,15 @@ HaloPlan plan_halo(const DotProblem& d, const ConvPlan& pl, uint32_t flags) {
   const int stage_b = hp.tg * hp.bn * kBK * 2;
   const int64_t groups = (pl.Cp / kBK) * d.Kh * (d.Kw / hp.tg);
   const int tiles_n = static_cast<int>((d.O + hp.bn - 1) / hp.bn);
+  if (hp.bn == 64) {
+    // N = 64 MMAs are bound by their issue floor; two blocks per SM with one input-box stage each hide
+    // start-up, loads and epilogue of one block under the MMAs of the other
+    hp.occ = 2;
+    hp.sa = 1;
+    hp.sb = std::min<int>(8, (113 * 1024 - 1024 - kHaloBarBytes - kHaloEpiBytes - kHaloAStage) / stage_b);
+    hp.ok = hp.sb >= 2;
+    return hp;
+  }
   // weights that fit beside two input boxes stay in shared memory for the whole kernel
   if (tiles_n == 1 && groups <= kHaloMaxStages && groups * stage_b + 2 * kHaloAStage <= kHaloSmemBudget) {
     hp.resident = 1;
@@ -1878,20 +1887,21 @@ bool encode_halo_weights(CUtensorMap* m, const void* base, int64_t O, int64_t ta
                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN>
+template <int BN, int OCC>
 int launch_halo(const CUtensorMap& ma, const CUtensorMap& mb, float* out, const HaloParams& p, cudaStream_t st) {
   const int smem = p.sa_stages * kHaloAStage + p.sb_stages * static_cast<int>(p.b_bytes) + kHaloEpiBytes + kHaloBarBytes + 1024;
   static bool attr_set_dev[64] = {false};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return GL_ERR_CUDA;
   if (!attr_set_dev[dev]) {
-    if (cudaFuncSetAttribute(conv_halo<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448) != cudaSuccess)
+    if (cudaFuncSetAttribute(conv_halo<BN, OCC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             OCC == 2 ? 113 * 1024 : 232448) != cudaSuccess)
       return GL_ERR_CUDA;
     attr_set_dev[dev] = true;
   }
   const int tiles = p.tiles_m * p.tiles_n;
-  const int grid = std::min(tiles, num_sms());
-  return launch_pdl(conv_halo<BN>, dim3(static_cast<unsigned>(grid)), dim3(kTcThreads), static_cast<size_t>(smem), st, 1,
+  const int grid = std::min(tiles, OCC * num_sms());
+  return launch_pdl(conv_halo<BN, OCC>, dim3(static_cast<unsigned>(grid)), dim3(kTcThreads), static_cast<size_t>(smem), st, 1,
                     ma, mb, out, p) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
 }
 
@@ -1920,7 +1930,7 @@ int run_halo(const HaloPlan& hp, const DotProblem& d, int64_t Cp, const uint16_t
   if (!encode_halo_box(&ma, x, d, Cp, hp.Wb, hp.RB) ||
       !encode_halo_weights(&mb, wt, d.O, d.Kh * d.Kw, Cp, hp.bn, hp.tg))
     return GL_ERR_CUDA;
-  return launch_halo<128>(ma, mb, out, p, st);
+  return hp.bn == 128 ? launch_halo<128, 1>(ma, mb, out, p, st) : launch_halo<64, 2>(ma, mb, out, p, st);
 }
 
 // A 1x1, stride-1, unpadded window over channels-last items is no window at all: the activations
