@@ -39,3 +39,30 @@ def test_conv_relu_maxpool_chain(gl, n, c, h, w, o):
         prog = gi.maxpool_program(gi.compute("relu", gi.conv2d_program(x, wt, (1, 1), ((1, 1), (1, 1)))).data,
                                   (3, 3), (2, 2), ((1, 1), (1, 1)))
         assert np.array_equal(prog.data, ref.astype(np.float64))
+
+
+def test_conv_relu_maxpool_dense_chain(gl):
+    """The chain continued by the dense layer of Fig. 2b: flatten the pooled activations per image and take
+    dot products with the rows of a weight matrix.  All values stay small integers (three input channels),
+    so the bf16 operands of the dense layer and every sum are exact."""
+    import torch
+    n, c, h, w, o, units = 2, 3, 23, 21, 8, 10
+    x = synth.uniform_int(62, 1, (n, c, h, w), -3, 3)
+    wt = synth.uniform_int(62, 2, (o, c, 3, 3), -3, 3)
+    spec = gl.windows_spec((c, 3, 3), (1, 1, 1), (0, 1, 1), (0, 1, 1))
+    act = gl.gl_cartesian_dot(gl.AccessPattern(to_bf16_device(x), 1), spec, gl.AccessPattern(to_bf16_device(wt), 1),
+                              flags=gl.GL_OUT_NCHW | gl.GL_EPILOGUE_RELU)
+    pooled = gl.gl_compute_reduce_max(gl.AccessPattern(act.tensor, 2),
+                                      gl.windows_spec((3, 3), (2, 2), (1, 1), (1, 1), gl.GL_PAD_NEG_INF))
+    feat = gl.gl_access_flatten(gl.AccessPattern(pooled.tensor, 1))            # ((N), (O*H'*W'))
+    k = feat.tensor.shape[1]
+    assert float(pooled.tensor.abs().max()) <= 256.0                            # exact in bf16
+    dense_w = synth.uniform_int(62, 3, (units, k), -3, 3)
+    feat_bf16 = gl.AccessPattern(feat.tensor.to(torch.bfloat16), 1)             # storage type of the next layer's operand
+    logits = gl.gl_cartesian_dot(feat_bf16, None, gl.AccessPattern(to_bf16_device(dense_w), 1), flags=gl.GL_EPILOGUE_RELU)
+    assert gl.gl_poll_device_status() == 0
+    conv = np.maximum(brute.conv2d(x, wt, (1, 1), ((1, 1), (1, 1))), 0.0)
+    ref_pool = brute.maxpool(conv.astype(np.float32), (3, 3), (2, 2), ((1, 1), (1, 1)))
+    ref = np.maximum(brute.rowdot(ref_pool.reshape(n, -1).astype(np.float32), dense_w), 0.0)
+    assert logits.shape == ((n, units), ())
+    assert np.array_equal(logits.tensor.cpu().numpy().astype(np.float64), ref)
