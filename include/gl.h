@@ -191,7 +191,9 @@ GL_API int gl_compute_reduce_sum(const gl_ap* in, gl_ap* out, void* stream);
  * Everything else runs on a slower general kernel.  The sum over the window is
  * taken in an unspecified order.  `workspace` must hold at least
  * gl_cartesian_dot_workspace() bytes (it may be NULL when that is 0) and must be
- * 1024-byte aligned; its contents are scratch. */
+ * 1024-byte aligned; its contents are scratch.  The kernels are launched with programmatic
+ * stream serialisation: their set-up may run while the preceding kernel of the stream
+ * drains, and they wait for its completion before their first access to memory. */
 GL_API int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w_or_null, const gl_ap* a1, gl_ap* out,
                      uint32_t flags, void* workspace, size_t workspace_bytes, void* stream);
 
