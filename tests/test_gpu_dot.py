@@ -203,6 +203,53 @@ def test_dense_random_shapes_bit_exact(gl, m, o, k):
     assert np.array_equal(out.tensor.cpu().numpy().astype(np.float64), brute.rowdot(a, b))
 
 
+def _random_window_kernel_cases(count, seed):
+    """Seeded shapes aimed at the kernels that keep windows in shared memory: stride-1 convolutions with 64, 128 or
+    192 channels (input block resident across the taps), at most 8 / Sw channels (windows read in place from row
+    runs), and 1x1 windows (the layout copy is the matrix).  Both item layouts are run for each."""
+    rng = np.random.default_rng(seed)
+    cases = []
+    while len(cases) < count:
+        kind = len(cases) % 3
+        if kind == 0:
+            c = int(rng.choice([64, 128, 192]))
+            kh, kw = int(rng.integers(1, 6)), int(rng.integers(2, 6))
+            sh = sw = 1
+            h, w = int(rng.integers(kh, 24)), int(rng.integers(kw, 61))
+            o = int(rng.choice([4, 60, 64, 68, 128, 200]))
+        elif kind == 1:
+            sw = int(rng.choice([1, 2, 4]))
+            c = int(rng.integers(1, 8 // sw + 1))
+            sh = int(rng.integers(1, 4))
+            kh, kw = int(rng.integers(1, 8)), int(rng.integers(1, 9))
+            h, w = int(rng.integers(kh, 40)), int(rng.integers(kw, 180))
+            o = int(rng.choice([4, 8, 36, 64, 128]))
+        else:
+            c = int(rng.choice([64, 72, 128, 320]))
+            kh = kw = 1
+            sh, sw = int(rng.integers(1, 4)), int(rng.integers(1, 4))
+            h, w = int(rng.integers(1, 30)), int(rng.integers(1, 30))
+            o = int(rng.choice([8, 64, 100, 260]))
+        ph, pw = (0, 0) if kind == 2 else (int(rng.integers(0, kh)), int(rng.integers(0, kw)))
+        n = int(rng.integers(1, 4))
+        if n * c * h * w * o * kh * kw > 1.5e8:
+            continue
+        cases.append((n, c, h, w, o, kh, kw, sh, sw, ph, pw))
+    return cases
+
+
+@pytest.mark.parametrize("case", _random_window_kernel_cases(30, 5309), ids=lambda c: "x".join(map(str, c)))
+def test_conv_random_shapes_window_kernels_bit_exact(gl, case):
+    n, c, h, w, o, kh, kw, sh, sw, ph, pw = case
+    x = synth.uniform_int(sum(case) + 7, 1, (n, c, h, w), -3, 3)
+    wt = synth.uniform_int(sum(case) + 7, 2, (o, c, kh, kw), -3, 3)
+    ref = _conv_ref(x, wt, (sh, sw), (ph, pw))
+    for cl in (False, True):
+        got = _conv_gpu(gl, x, wt, (sh, sw), (ph, pw), channels_last=cl)
+        assert got.shape == ref.shape
+        assert np.array_equal(got.astype(np.float64), ref), "layout channels_last=%s" % cl
+
+
 def test_out_nchw_needs_a_conv(gl):
     a = gl.AccessPattern(to_bf16_device(synth.uniform_int(26, 1, (8, 16), -3, 3)), 1)
     out = gl.AccessPattern(torch.empty((8, 8), device="cuda"), 2)
