@@ -88,6 +88,10 @@ typedef struct {
 #define GL_EPILOGUE_RELU 0x2u       /* apply compute relu to every result before it is stored  */
 #define GL_OUT_NCHW 0x4u             /* conv2d only: store transpose(squeeze(...)) of Fig. 2a, i.e.
                                         ((N, O, H', W'),()); see gl_shape_cartesian_dot_nchw      */
+#define GL_OUT_BF16 0x8u             /* store the results rounded to bf16 (nearest even) instead of fp32: `out`
+                                      * must then be GL_BF16.  Sums are still carried in fp32; the rounding is
+                                      * the last step, after relu.  Lets the next layer read its operand as is
+                                      * and halves the bytes written. */
 #define GL_DOT_GENERAL_KERNEL 0x100u /* skip the tensor-core path: run the general kernel, which
                                         takes any shape and sums each window in index order      */
 
@@ -183,7 +187,8 @@ GL_API int gl_compute_reduce_sum(const gl_ap* in, gl_ap* out, void* stream);
 /* out = compute dotProd (cartProd (windows? a0) a1), optionally followed by compute
  * relu (Fig. 2a for conv2d with w given, Fig. 2b / Fig. 6 for matrix products with
  * w NULL).  a0 and a1 are GL_BF16, products and sums are carried in fp32, out is
- * GL_F32 with the access dims of A followed by those of a1, i.e. row-major [M, O].
+ * GL_F32 (GL_BF16 with GL_OUT_BF16) with the access dims of A followed by those of a1,
+ * i.e. row-major [M, O].
  * Two item layouts take the tensor-core path:
  *   - w NULL, a0 ((M),(K)), a1 ((O),(K)) with K a multiple of 8;
  *   - a0 ((N),(C,H,W)) with window (C,Kh,Kw), stride (1,Sh,Sw), or a0 ((N),(H,W,C))

@@ -19,6 +19,7 @@ GL_PAD_ZERO, GL_PAD_NEG_INF = 0, 1
 GL_EPILOGUE_RELU = 0x2
 GL_DOT_GENERAL_KERNEL = 0x100
 GL_OUT_NCHW = 0x4
+GL_OUT_BF16 = 0x8
 GL_OK = 0
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -316,6 +317,8 @@ def gl_cartesian_dot(a0: AccessPattern, w: Optional[GlWindows], a1: AccessPatter
         else:
             _check(LIB.gl_shape_cartesian_dot(ctypes.byref(s0), _wptr(w), ctypes.byref(s1), ctypes.byref(m)),
                    "gl_shape_cartesian_dot")
+        if flags & GL_OUT_BF16:
+            m.dtype = GL_BF16
         out = _alloc(m, a0.tensor.device)
     if workspace is None:
         need = int(LIB.gl_cartesian_dot_workspace(ctypes.byref(s0), _wptr(w), ctypes.byref(s1), flags))

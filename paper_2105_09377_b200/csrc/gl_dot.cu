@@ -48,10 +48,18 @@ struct GenA {            // how to fetch A[m,k]
   int64_t item;
   // result layout: [M,O], or (image, O, H'W') when the squeeze + transpose of Fig. 2a is fused
   int out_nchw;
+  int out_bf16;   // results rounded to bf16 (nearest even) and stored as 2-byte elements
   int64_t HoWo;
 };
 
 __device__ __forceinline__ float bf16_to_f32(uint16_t b) { return __uint_as_float(static_cast<uint32_t>(b) << 16); }
+// Two fp32 values (as bits) rounded to nearest-even bf16 and packed: `lo` at the lower address.
+__device__ __forceinline__ uint32_t pack_bf16x2(uint32_t lo, uint32_t hi) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(__uint_as_float(hi)), "f"(__uint_as_float(lo)));
+  return d;
+}
+__device__ __forceinline__ uint16_t f32_to_bf16(float v) { return static_cast<uint16_t>(pack_bf16x2(__float_as_uint(v), 0u) & 0xFFFFu); }
 
 __device__ float fetch_a(const uint16_t* __restrict__ a, const GenA& g, int64_t m, int64_t k) {
   if (g.mode == 0) return bf16_to_f32(a[m * g.K + k]);
@@ -113,8 +121,9 @@ __global__ void __launch_bounds__(256) dot_general(const uint16_t* __restrict__ 
       if (m < g.M && o < g.O) {
         float v = acc[i][j];
         if (relu) v = v > 0.f ? v : 0.f;
-        if (g.out_nchw) out[((m / g.HoWo) * g.O + o) * g.HoWo + m % g.HoWo] = v;
-        else out[m * g.O + o] = v;
+        const int64_t at = g.out_nchw ? ((m / g.HoWo) * g.O + o) * g.HoWo + m % g.HoWo : m * g.O + o;
+        if (g.out_bf16) reinterpret_cast<uint16_t*>(out)[at] = f32_to_bf16(v);
+        else out[at] = v;
       }
     }
 }
@@ -554,6 +563,8 @@ struct TcParams {
   int relu;
   int out_nchw;           // store (image, O, H'W') instead of [M,O]: squeeze + transpose (0 3 1 2) of Fig. 2a
   int tma_store;          // result rows are 16-byte multiples: the epilogue may use TMA stores
+  int out_bf16;           // results rounded to bf16 and stored as 2-byte elements (never with a K split: the
+                          // partial planes stay fp32 and the summing kernel rounds)
   // conv only
   int Cp, Kh, Kw, Sh, Sw, ph, pw, Ho, Wo;
   int cchunks;            // kIm2col: 64-channel chunks per tap; kIm2colGranule: 8-channel granules per tap
@@ -821,15 +832,19 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
         m = static_cast<int64_t>(orow) * p.Wo + wloc;
         m_ok = wloc < p.Wo;
       }
-      float* row = out + (static_cast<int64_t>(ks) * p.M + m) * p.O;   // partial plane ks (0 without a K split)
-      float* col = out;      // out_nchw: &out[image][0][pixel]; channel o then lies o*H'W' further
+      const int64_t row_at = (static_cast<int64_t>(ks) * p.M + m) * p.O;   // partial plane ks (0 without a K split)
+      float* row = out + row_at;
+      int64_t col_at = 0;    // out_nchw: index of out[image][0][pixel]; channel o then lies o*H'W' further
       if (p.out_nchw && m_ok) {
         uint32_t img_o, pix_o;
         p.div_howo.divmod(static_cast<uint32_t>(m), img_o, pix_o);
-        col = out + static_cast<int64_t>(img_o) * p.O * p.div_howo.d + pix_o;
+        col_at = static_cast<int64_t>(img_o) * p.O * p.div_howo.d + pix_o;
       }
+      float* col = out + col_at;
+      // bf16 results through TMA stores go 64 columns at a time (128 bytes per row, as 32 fp32 columns do)
+      const int cstep = (p.out_bf16 && p.tma_store) ? 64 : 32;
 #pragma unroll 1
-      for (int c = 0; c < BN; c += 32) {
+      for (int c = 0; c < BN; c += cstep) {
         const int64_t n0 = static_cast<int64_t>(tn) * BN + c;
         if (n0 >= p.O) break;   // uniform across the warp
         uint32_t r[32];
@@ -838,13 +853,33 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
 #pragma unroll
           for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(fmaxf(__uint_as_float(r[i]), 0.f));
         }
+        if (cstep == 64) {
+          // pack the first 32 columns, then fetch and pack the next 32: r[0..31] = 64 bf16 values of this row
+#pragma unroll
+          for (int i = 0; i < 16; ++i) r[i] = pack_bf16x2(r[2 * i], r[2 * i + 1]);
+          uint32_t r2[32];
+          tc_load_32cols(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN + c + 32, r2);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            uint32_t a = r2[2 * i], b = r2[2 * i + 1];
+            if (p.relu) { a = __float_as_uint(fmaxf(__uint_as_float(a), 0.f)); b = __float_as_uint(fmaxf(__uint_as_float(b), 0.f)); }
+            r[16 + i] = pack_bf16x2(a, b);
+          }
+        }
         if (p.out_nchw) {
           // lanes hold consecutive pixels: for every channel the warp writes one contiguous run
           if (m_ok) {
             const int64_t plane = p.div_howo.d;
+            if (p.out_bf16) {
+              uint16_t* col16 = reinterpret_cast<uint16_t*>(out) + col_at;
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (n0 + i < p.O) col[(n0 + i) * plane] = __uint_as_float(r[i]);
+              for (int i = 0; i < 32; ++i)
+                if (n0 + i < p.O) col16[(n0 + i) * plane] = f32_to_bf16(__uint_as_float(r[i]));
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (n0 + i < p.O) col[(n0 + i) * plane] = __uint_as_float(r[i]);
+            }
           }
         } else if (p.tma_store) {
           // 32x32 fp32 block: each lane parks its row in shared memory (16-byte pieces XOR-swizzled by
@@ -879,7 +914,12 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
           }
           ++chunk_it;
         } else if (m_ok) {
-          if (vec_ok && n0 + 32 <= p.O) {
+          if (p.out_bf16) {
+            uint16_t* row16 = reinterpret_cast<uint16_t*>(out) + row_at;
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (n0 + i < p.O) row16[n0 + i] = f32_to_bf16(__uint_as_float(r[i]));
+          } else if (vec_ok && n0 + 32 <= p.O) {
 #pragma unroll
             for (int i = 0; i < 32; i += 4)
               *reinterpret_cast<uint4*>(row + n0 + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
@@ -947,6 +987,7 @@ constexpr int kHaloSmemBudget = 232448 - 1024 - kHaloBarBytes - kHaloEpiBytes;
 struct HaloParams {
   int64_t O;
   int relu;
+  int out_bf16;   // results rounded to bf16 (O a multiple of 8)
   int Ho, Wo, Wb, R, tiles_m, tiles_n;
   int Kh, Kw, Cp, cchunks;
   int tg, groups_per_chunk;                 // a B stage holds tg consecutive taps (a filter row, or one tap) of one chunk
@@ -1127,8 +1168,9 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       }
       if (!mbar_wait(bar_tfull + 8 * acc, aph, abort_flag)) { ok = false; break; }
       tc_fence_after();
+      const int cstep = p.out_bf16 ? 64 : 32;   // a staged row is 128 bytes: 32 fp32 or 64 bf16 columns
 #pragma unroll 1
-      for (int c = 0; c < BN; c += 32) {
+      for (int c = 0; c < BN; c += cstep) {
         const int64_t n0 = static_cast<int64_t>(tn) * BN + c;
         if (n0 >= p.O) break;   // uniform across the warp
         uint32_t r[32];
@@ -1137,6 +1179,18 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 #pragma unroll
           for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(fmaxf(__uint_as_float(r[i]), 0.f));
         }
+        if (p.out_bf16) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) r[i] = pack_bf16x2(r[2 * i], r[2 * i + 1]);
+          uint32_t r2[32];
+          tc_load_32cols(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN + c + 32, r2);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            uint32_t a = r2[2 * i], b = r2[2 * i + 1];
+            if (p.relu) { a = __float_as_uint(fmaxf(__uint_as_float(a), 0.f)); b = __float_as_uint(fmaxf(__uint_as_float(b), 0.f)); }
+            r[16 + i] = pack_bf16x2(a, b);
+          }
+        }
         __syncwarp();   // the previous block has been read back
 #pragma unroll
         for (int j = 0; j < 8; ++j)
@@ -1144,7 +1198,8 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                        "r"(r[4 * j]), "r"(r[4 * j + 1]), "r"(r[4 * j + 2]), "r"(r[4 * j + 3])
                        : "memory");
         __syncwarp();
-        const bool col_ok = n0 + piece * 4 < p.O;   // O is a multiple of 4
+        const int per_piece = p.out_bf16 ? 8 : 4;   // elements in 16 bytes; O is a multiple of it
+        const bool col_ok = n0 + piece * per_piece < p.O;
 #pragma unroll
         for (int it = 0; it < 8; ++it) {
           const int rr = it * 4 + sub_row;
@@ -1153,8 +1208,12 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                        : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3)
                        : "r"(buf + rr * 128 + ((piece ^ (rr & 7)) << 4))
                        : "memory");
-          if (row_off[it] >= 0 && col_ok)
-            *reinterpret_cast<uint4*>(out + row_off[it] + n0 + piece * 4) = make_uint4(v0, v1, v2, v3);
+          if (row_off[it] >= 0 && col_ok) {
+            if (p.out_bf16)
+              *reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(out) + row_off[it] + n0 + piece * 8) = make_uint4(v0, v1, v2, v3);
+            else
+              *reinterpret_cast<uint4*>(out + row_off[it] + n0 + piece * 4) = make_uint4(v0, v1, v2, v3);
+          }
         }
       }
       tc_fence_before();
@@ -1200,6 +1259,7 @@ constexpr int kRunEpiBytes = 4 * 2 * 4096;   // two 32x32 fp32 staging tiles per
 struct RowRunParams {
   int64_t O;
   int relu;
+  int out_bf16;   // results rounded to bf16 (O a multiple of 8)
   int Ho, Wo, Hp, Sh, Kh;
   int segs, tiles;              // 128-column segments per output row; tiles = N * Ho * segs
   int ksteps;                   // MMAs (K = 16) per filter row
@@ -1328,14 +1388,30 @@ conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restr
       p.div_segs.divmod(static_cast<uint32_t>(u), row, seg);
       if (!mbar_wait(bar_tfull + 8 * acc, aph, abort_flag)) { ok = false; break; }
       tc_fence_after();
+      const int cstep = p.out_bf16 ? 64 : 32;   // a staged row is 128 bytes: 32 fp32 or 64 bf16 columns
 #pragma unroll 1
-      for (int c = 0; c < p.bn; c += 32) {
+      for (int c = 0; c < p.bn; c += cstep) {
         if (c >= p.O) break;   // uniform across the warp
         uint32_t r[32];
         tc_load_32cols(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * p.bn + c, r);
         if (p.relu) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(fmaxf(__uint_as_float(r[i]), 0.f));
+        }
+        if (p.out_bf16) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) r[i] = pack_bf16x2(r[2 * i], r[2 * i + 1]);
+          uint32_t r2[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) r2[i] = 0u;
+          // the accumulator is bn columns wide: a second half exists only where c + 32 < bn
+          if (c + 32 < p.bn) tc_load_32cols(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * p.bn + c + 32, r2);
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            uint32_t a = r2[2 * i], b = r2[2 * i + 1];
+            if (p.relu) { a = __float_as_uint(fmaxf(__uint_as_float(a), 0.f)); b = __float_as_uint(fmaxf(__uint_as_float(b), 0.f)); }
+            r[16 + i] = pack_bf16x2(a, b);
+          }
         }
         const uint32_t buf = epi_base + q * 8192 + (chunk_it & 1u) * 4096;
         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the store before last has read this buffer
@@ -1555,24 +1631,27 @@ bool encode_im2col(CUtensorMap* m, const void* base, const DotProblem& d, int64_
                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// fp32 result planes [planes, M, O]: 32x32 boxes, 128-byte swizzle (what the epilogue stages).
-bool encode_result(CUtensorMap* m, float* base, int64_t M, int64_t O, int64_t planes) {
+// Result planes [planes, M, O]: boxes of 32 rows x 128 bytes (32 fp32 or 64 bf16 columns), 128-byte swizzle
+// (what the epilogue stages).
+bool encode_result(CUtensorMap* m, float* base, int64_t M, int64_t O, int64_t planes, bool bf16 = false) {
+  const cuuint64_t es = bf16 ? 2 : 4;
   const cuuint64_t dims[3] = {static_cast<cuuint64_t>(O), static_cast<cuuint64_t>(M), static_cast<cuuint64_t>(planes)};
-  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(O) * 4, static_cast<cuuint64_t>(M * O) * 4};
-  const cuuint32_t box[3] = {32, 32, 1};
+  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(O) * es, static_cast<cuuint64_t>(M * O) * es};
+  const cuuint32_t box[3] = {bf16 ? 64u : 32u, 32, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
-  return driver_api().tiled(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr,
+  return driver_api().tiled(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr,
                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                             CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // fp32 result of a row-window convolution viewed as (N*Ho, Wo, O): 32x32 boxes inside one output row.
-bool encode_result_rows(CUtensorMap* m, float* base, int64_t rows, int64_t Wo, int64_t O) {
+bool encode_result_rows(CUtensorMap* m, float* base, int64_t rows, int64_t Wo, int64_t O, bool bf16 = false) {
+  const cuuint64_t es = bf16 ? 2 : 4;
   const cuuint64_t dims[3] = {static_cast<cuuint64_t>(O), static_cast<cuuint64_t>(Wo), static_cast<cuuint64_t>(rows)};
-  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(O) * 4, static_cast<cuuint64_t>(Wo * O) * 4};
-  const cuuint32_t box[3] = {32, 32, 1};
+  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(O) * es, static_cast<cuuint64_t>(Wo * O) * es};
+  const cuuint32_t box[3] = {bf16 ? 64u : 32u, 32, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
-  return driver_api().tiled(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr,
+  return driver_api().tiled(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr,
                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                             CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -1630,13 +1709,14 @@ int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams
   p.div_wo.set(p.Wo > 0 ? p.Wo : 1);
   p.div_howo.set(p.Wo > 0 ? static_cast<int64_t>(p.Wo) * p.Ho : 1);
   CUtensorMap mc;
-  p.tma_store = (p.O % 4 == 0 && !p.out_nchw) ? 1 : 0;
+  p.tma_store = (p.O % (p.out_bf16 ? 8 : 4) == 0 && !p.out_nchw) ? 1 : 0;
   if (MODE == kRowWin) {
     p.div_segs.set(p.segs);
     p.div_ho.set(p.Ho);
   }
   if (p.tma_store) {
-    const bool ok = MODE == kRowWin ? encode_result_rows(&mc, out, p.M / p.Wo, p.Wo, p.O) : encode_result(&mc, out, p.M, p.O, p.ksplit);
+    const bool ok = MODE == kRowWin ? encode_result_rows(&mc, out, p.M / p.Wo, p.Wo, p.O, p.out_bf16 != 0)
+                                    : encode_result(&mc, out, p.M, p.O, p.ksplit, p.out_bf16 != 0);
     if (!ok) return GL_ERR_CUDA;
   } else {
     mc = ma;   // unused by the kernel; any valid map
@@ -1693,7 +1773,7 @@ int pick_bn(int64_t M, int64_t O) {
 // compute reduceSum over the K-split partial planes (Section 5.4, last blocking rewrite), planes
 // added in index order so that the result does not depend on scheduling; relu applied last.
 __global__ void __launch_bounds__(256) splitk_reduce(const float* __restrict__ part, float* __restrict__ out,
-                                                     int64_t n, int planes, int relu) {
+                                                     int64_t n, int planes, int relu, int out_bf16) {
   pdl_wait();
   pdl_launch_dependents();
   const int64_t n4 = n >> 2;
@@ -1705,7 +1785,11 @@ __global__ void __launch_bounds__(256) splitk_reduce(const float* __restrict__ p
       acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
     }
     if (relu) { acc.x = fmaxf(acc.x, 0.f); acc.y = fmaxf(acc.y, 0.f); acc.z = fmaxf(acc.z, 0.f); acc.w = fmaxf(acc.w, 0.f); }
-    reinterpret_cast<float4*>(out)[i] = acc;
+    if (out_bf16)
+      reinterpret_cast<uint2*>(out)[i] = make_uint2(pack_bf16x2(__float_as_uint(acc.x), __float_as_uint(acc.y)),
+                                                    pack_bf16x2(__float_as_uint(acc.z), __float_as_uint(acc.w)));
+    else
+      reinterpret_cast<float4*>(out)[i] = acc;
   }
 }
 
@@ -1757,7 +1841,7 @@ ConvPlan plan_conv(const DotProblem& d, uint32_t flags) {
   pl.tc = fits && ((d.M + 127) / 128) * ((d.O + 63) / 64) < (1ll << 28);
   pl.prepass = !d.channels_last || pl.Cp != d.C;
   if (pl.tc && !(flags & GL_OUT_NCHW) && (d.Sw == 1 || d.Sw == 2 || d.Sw == 4 || d.Sw == 8) && d.C <= 8 / d.Sw &&
-      d.O % 4 == 0 && d.O <= 128 && d.Kh <= 16 && kPackWarps * (d.W + d.pw_lo + d.pw_hi + 64) * 16 <= 48 * 1024 && d.Wo < (1ll << 24) &&
+      d.O % ((flags & GL_OUT_BF16) ? 8 : 4) == 0 && d.O <= 128 && d.Kh <= 16 && kPackWarps * (d.W + d.pw_lo + d.pw_hi + 64) * 16 <= 48 * 1024 && d.Wo < (1ll << 24) &&
       d.N * (d.H + d.ph_lo + d.ph_hi) < (1ll << 31)) {
     const int cp = static_cast<int>(8 / d.Sw);
     const int ksteps = static_cast<int>((d.Kw * cp + 15) / 16);
@@ -1816,7 +1900,7 @@ struct HaloPlan {
 HaloPlan plan_halo(const DotProblem& d, const ConvPlan& pl, uint32_t flags) {
   HaloPlan hp;
   if (!d.conv || !pl.tc || pl.rowwin || (flags & GL_OUT_NCHW)) return hp;
-  if (d.Sh != 1 || d.Sw != 1 || pl.Cp % kBK != 0 || d.O % 4 != 0) return hp;
+  if (d.Sh != 1 || d.Sw != 1 || pl.Cp % kBK != 0 || d.O % ((flags & GL_OUT_BF16) ? 8 : 4) != 0) return hp;
   if (d.Kh == 1 && d.Kw == 1) return hp;   // no overlap between windows: nothing to keep
   const int64_t Wb = d.W + d.pw_lo + d.pw_hi;
   // the MMA of the last tap reads 128 rows starting (Kh-1)*Wb + Kw-1 rows into the stage
@@ -1906,10 +1990,10 @@ int launch_halo(const CUtensorMap& ma, const CUtensorMap& mb, float* out, const 
 }
 
 int run_halo(const HaloPlan& hp, const DotProblem& d, int64_t Cp, const uint16_t* x, const uint16_t* wt, float* out,
-             int relu, cudaStream_t st) {
+             int relu, int out_bf16, cudaStream_t st) {
   HaloParams p;
   std::memset(&p, 0, sizeof(p));
-  p.O = d.O; p.relu = relu;
+  p.O = d.O; p.relu = relu; p.out_bf16 = out_bf16;
   p.Ho = static_cast<int>(d.Ho); p.Wo = static_cast<int>(d.Wo);
   p.Wb = hp.Wb; p.R = hp.R;
   p.tiles_m = static_cast<int>(d.N) * hp.tiles_per_img;
@@ -2006,14 +2090,16 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
   if (rc) return rc;
   if (!out) return GL_ERR_NULL;
   if (a0->dtype != GL_BF16 || a1->dtype != GL_BF16) return GL_ERR_DTYPE;
-  if (flags & ~(GL_EPILOGUE_RELU | GL_DOT_GENERAL_KERNEL | GL_OUT_NCHW)) return GL_ERR_UNSUPPORTED;
+  if (flags & ~(GL_EPILOGUE_RELU | GL_DOT_GENERAL_KERNEL | GL_OUT_NCHW | GL_OUT_BF16)) return GL_ERR_UNSUPPORTED;
   const int out_nchw = (flags & GL_OUT_NCHW) ? 1 : 0;
+  const int out_bf16 = (flags & GL_OUT_BF16) ? 1 : 0;
   DotProblem d;
   rc = classify_dot(a0, w, a1, &d);
   if (rc) return rc;
   gl_ap want = *out;
   rc = out_nchw ? gl_shape_cartesian_dot_nchw(a0, w, a1, &want) : gl_shape_cartesian_dot(a0, w, a1, &want);
   if (rc) return rc;
+  if (out_bf16) want.dtype = GL_BF16;
   rc = check_same_meta(want, out);
   if (rc) return rc;
   rc = check_data(out);
@@ -2033,6 +2119,7 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     GenA g;
     fill_general(a0, w, d, &g);
     g.out_nchw = out_nchw;
+    g.out_bf16 = out_bf16;
     const int64_t gx = (d.M + 63) / 64, gy = (d.O + 63) / 64;
     if (gy > 65535 || gx > 0x7FFFFFFF) return GL_ERR_UNSUPPORTED;
     dot_general<<<dim3(static_cast<unsigned>(gx), static_cast<unsigned>(gy)), 256, 0, st>>>(pa, pb, dst, g, relu);
@@ -2058,16 +2145,18 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
   p.ksplit = tp.ksplit;
   p.kper = tp.kper;
   float* const final_dst = dst;
-  if (tp.ksplit > 1) {
+  p.out_bf16 = out_bf16;
+  if (tp.ksplit > 1) {   // fp32 partial planes; relu and the rounding to bf16 happen in the summing kernel
     dst = reinterpret_cast<float*>(static_cast<unsigned char*>(workspace) + pre_bytes);
     p.relu = 0;
+    p.out_bf16 = 0;
   }
   // the launch of the partial-sum kernel when the contraction was split
   auto finish = [&](int rc_launch) -> int {
     if (rc_launch != GL_OK || tp.ksplit == 1) return rc_launch;
     const int64_t n = d.M * d.O;
     return launch_pdl(splitk_reduce, dim3(static_cast<unsigned>(std::min<int64_t>((n / 4 + 255) / 256, 148 * 8))), dim3(256),
-                      0, st, 1, static_cast<const float*>(dst), final_dst, n, tp.ksplit, relu) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+                      0, st, 1, static_cast<const float*>(dst), final_dst, n, tp.ksplit, relu, out_bf16) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
   };
   p.tiles_m = static_cast<int>((d.M + kBM - 1) / kBM);
   p.tiles_n = static_cast<int>((d.O + bn - 1) / bn);
@@ -2118,7 +2207,7 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
       if (cudaGetLastError() != cudaSuccess) return GL_ERR_CUDA;
       RowRunParams rp;
       std::memset(&rp, 0, sizeof(rp));
-      rp.O = d.O; rp.relu = relu;
+      rp.O = d.O; rp.relu = relu; rp.out_bf16 = out_bf16;
       rp.Ho = static_cast<int>(d.Ho); rp.Wo = static_cast<int>(d.Wo); rp.Hp = static_cast<int>(pl.Hp);
       rp.Sh = static_cast<int>(d.Sh); rp.Kh = static_cast<int>(d.Kh);
       rp.segs = static_cast<int>((d.Wo + kBM - 1) / kBM);
@@ -2131,7 +2220,7 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
       rp.div_segs.set(rp.segs);
       rp.div_ho.set(d.Ho);
       CUtensorMap mc;
-      if (!encode_result_rows(&mc, dst, d.N * d.Ho, d.Wo, d.O)) return GL_ERR_CUDA;
+      if (!encode_result_rows(&mc, dst, d.N * d.Ho, d.Wo, d.O, out_bf16 != 0)) return GL_ERR_CUDA;
       const int smem = 1024 + kRunEpiBytes + static_cast<int>((rp.b_bytes + 127u) & ~127u) +
                        rp.stages * rp.Kh * static_cast<int>(rp.slot_bytes) + 256;
       static bool attr_set_dev[64] = {false};
@@ -2224,7 +2313,7 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
       return GL_ERR_CUDA;
     return finish(launch_tc_bn<kDense>(bn, ma, mb, dst, p, st));
   }
-  if (hp.ok) return run_halo(hp, d, Cp, x, wt, dst, relu, st);
+  if (hp.ok) return run_halo(hp, d, Cp, x, wt, dst, relu, out_bf16, st);
   p.K = taps * Cp;
   p.Cp = static_cast<int>(Cp);
   p.Kh = static_cast<int>(d.Kh); p.Kw = static_cast<int>(d.Kw);

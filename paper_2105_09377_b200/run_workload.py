@@ -41,6 +41,8 @@ def build_call(cfg, layout: str, device, batch=None, flags=0):
         a, b = _inputs(cfg, synth.config_seed(1))
         aa, bb = gl.AccessPattern(_bf16(a, device), 1), gl.AccessPattern(_bf16(b, device), 1)
         out = gl.output_like(gl.gl_shape_cartesian_dot(a.shape, 1, None, b.shape, 1), device)
+        if flags & gl.GL_OUT_BF16:
+            out = gl.AccessPattern(out.tensor.to(torch.bfloat16), out.access_ndim)
         return gl.prepare_cartesian_dot(aa, None, bb, out, flags | gl.GL_EPILOGUE_RELU), cfg.flops, cfg.algorithmic_bytes
     if isinstance(cfg, synth.ConvCase):
         if batch:
@@ -68,6 +70,8 @@ def build_call(cfg, layout: str, device, batch=None, flags=0):
             spec = gl.windows_spec((cfg.c, cfg.kh, cfg.kw), (1, cfg.stride, cfg.stride), (0, cfg.pad, cfg.pad), (0, cfg.pad, cfg.pad))
         xa, wa = gl.AccessPattern(_bf16(x, device), 1), gl.AccessPattern(_bf16(wt, device), 1)
         out = gl.output_like(gl.gl_shape_cartesian_dot(x.shape, 1, spec, wt.shape, 1), device)
+        if flags & gl.GL_OUT_BF16:      # results stored as bf16: half the bytes written
+            out = gl.AccessPattern(out.tensor.to(torch.bfloat16), out.access_ndim)
         need = gl.gl_cartesian_dot_workspace(xa, spec, wa, flags)
         ws = torch.empty(need + 1024, dtype=torch.uint8, device=device) if need else None
         return gl.prepare_cartesian_dot(xa, spec, wa, out, flags, ws), cfg.flops, cfg.algorithmic_bytes
@@ -102,11 +106,12 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="override the leading (batch) extent")
     ap.add_argument("--graph", action="store_true", help="time one CUDA graph holding all iterations")
     ap.add_argument("--general", action="store_true", help="use the general SIMT kernel for dot products")
+    ap.add_argument("--bf16-out", action="store_true", help="store dot-product results as bf16 (GL_OUT_BF16)")
     args = ap.parse_args()
     device = torch.device("cuda", 0)
     torch.cuda.set_device(device)
     call, flops, nbytes = build_call(table[args.workload], args.layout, device, args.batch or None,
-                                     gl.GL_DOT_GENERAL_KERNEL if args.general else 0)
+                                     (gl.GL_DOT_GENERAL_KERNEL if args.general else 0) | (gl.GL_OUT_BF16 if args.bf16_out else 0))
     call()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

@@ -41,7 +41,7 @@ def _conv_gpu(gl, x, wt, stride, pad, channels_last=False, flags=0):
         spec = gl.windows_spec((c, kh, kw), (1, stride[0], stride[1]), (0, pad[0], pad[1]), (0, pad[0], pad[1]))
     out = gl.gl_cartesian_dot(xa, spec, wa, flags=flags)
     _ok(gl)
-    t = out.tensor
+    t = out.tensor.float() if out.tensor.dtype == torch.bfloat16 else out.tensor
     if channels_last:
         assert t.shape[3] == 1
         return t.squeeze(3).cpu().numpy()
@@ -248,6 +248,82 @@ def test_conv_random_shapes_window_kernels_bit_exact(gl, case):
         got = _conv_gpu(gl, x, wt, (sh, sw), (ph, pw), channels_last=cl)
         assert got.shape == ref.shape
         assert np.array_equal(got.astype(np.float64), ref), "layout channels_last=%s" % cl
+
+
+# ---- GL_OUT_BF16: results rounded to bf16 as the last step ----
+
+def _bf16(v):
+    """float64 array -> the bf16 value nearest to each element (ties to even), as float64."""
+    return synth.bf16_round(np.asarray(v, dtype=np.float32)).astype(np.float64)
+
+
+@pytest.mark.parametrize("m,o,k", [(36, 8, 32), (130, 72, 72), (300, 520, 200), (257, 100, 1000), (2600, 1928, 200), (64, 64, 4096)])
+def test_dense_bf16_output_bit_exact(gl, m, o, k):
+    # integer sums are exact in fp32, so rounding them to bf16 gives the same bits on both sides
+    a = synth.uniform_int(43, 1, (m, k), -3, 3)
+    b = synth.uniform_int(43, 2, (o, k), -3, 3)
+    ref = brute.rowdot(a, b)
+    aa, bb = gl.AccessPattern(to_bf16_device(a), 1), gl.AccessPattern(to_bf16_device(b), 1)
+    for flags in (gl.GL_OUT_BF16, gl.GL_OUT_BF16 | gl.GL_EPILOGUE_RELU, gl.GL_OUT_BF16 | gl.GL_DOT_GENERAL_KERNEL):
+        out = gl.gl_cartesian_dot(aa, None, bb, flags=flags)
+        _ok(gl)
+        assert out.tensor.dtype == torch.bfloat16 and out.shape == ((m, o), ())
+        want = _bf16(np.maximum(ref, 0.0) if flags & gl.GL_EPILOGUE_RELU else ref)
+        assert np.array_equal(out.tensor.float().cpu().numpy().astype(np.float64), want)
+
+
+CONV_BF16_OUT = [
+    # n, c, h, w, o, kh, kw, sh, sw, ph, pw
+    (2, 64, 12, 20, 128, 3, 3, 1, 1, 1, 1),    # input block resident, 128-wide tiles
+    (2, 64, 14, 14, 64, 3, 3, 1, 1, 1, 1),     # ... 64-wide tiles, two blocks per SM
+    (2, 3, 30, 40, 64, 7, 7, 2, 2, 3, 3),      # windows read in place from row runs
+    (1, 4, 17, 33, 24, 5, 5, 3, 2, 2, 2),      # ... narrow accumulator (N = 32)
+    (2, 64, 13, 13, 72, 3, 3, 2, 2, 1, 1),     # im2col-mode loads (stride 2)
+    (2, 128, 10, 10, 64, 1, 1, 2, 2, 0, 0),    # 1x1: the copy is the matrix
+    (2, 16, 9, 9, 20, 3, 3, 1, 1, 1, 1),       # granule path, O not a multiple of 8
+    (1, 512, 7, 7, 64, 3, 3, 1, 1, 1, 1),      # split contraction, rounded by the summing kernel
+]
+
+
+@pytest.mark.parametrize("case", CONV_BF16_OUT, ids=lambda c: "x".join(map(str, c)))
+def test_conv_bf16_output_bit_exact(gl, case):
+    n, c, h, w, o, kh, kw, sh, sw, ph, pw = case
+    x = synth.uniform_int(44, 1, (n, c, h, w), -3, 3)
+    wt = synth.uniform_int(44, 2, (o, c, kh, kw), -3, 3)
+    ref = _conv_ref(x, wt, (sh, sw), (ph, pw))
+    for cl in (False, True):
+        for relu in (0, gl.GL_EPILOGUE_RELU):
+            got = _conv_gpu(gl, x, wt, (sh, sw), (ph, pw), channels_last=cl, flags=gl.GL_OUT_BF16 | relu)
+            want = _bf16(np.maximum(ref, 0.0) if relu else ref)
+            assert np.array_equal(np.asarray(got, dtype=np.float64), want), "channels_last=%s relu=%s" % (cl, bool(relu))
+    # fused squeeze + transpose with bf16 results
+    out = gl.gl_cartesian_dot(gl.AccessPattern(to_bf16_device(x), 1),
+                              gl.windows_spec((c, kh, kw), (1, sh, sw), (0, ph, pw), (0, ph, pw)),
+                              gl.AccessPattern(to_bf16_device(wt), 1), flags=gl.GL_OUT_BF16 | gl.GL_OUT_NCHW)
+    _ok(gl)
+    assert np.array_equal(out.tensor.float().cpu().numpy().astype(np.float64), _bf16(ref.transpose(0, 3, 1, 2)))
+
+
+def test_bf16_output_gaussian_within_one_rounding(gl):
+    # N(0,1) inputs: the fp32 sum differs from the float64 one by ~1e-6 relative, so after rounding to bf16 the two
+    # agree or sit on neighbouring bf16 values (2^-8 relative apart)
+    case = synth.DenseCase("d512", 512, 768, 1024)
+    a, b = case.inputs(45)
+    out = gl.gl_cartesian_dot(gl.AccessPattern(to_bf16_device(a), 1), None, gl.AccessPattern(to_bf16_device(b), 1),
+                              flags=gl.GL_OUT_BF16)
+    _ok(gl)
+    got = out.tensor.float().cpu().numpy().astype(np.float64)
+    ref = brute.rowdot(a, b)
+    assert np.max(np.abs(got - ref) / np.maximum(np.abs(ref), np.sqrt(np.mean(ref * ref)))) <= 2.0 ** -8
+    assert np.mean(got == _bf16(ref)) > 0.99
+
+
+def test_bf16_output_wants_a_bf16_tensor(gl):
+    a = gl.AccessPattern(to_bf16_device(synth.uniform_int(46, 1, (16, 32), -3, 3)), 1)
+    with pytest.raises(gl.GlError):
+        gl.gl_cartesian_dot(a, None, a, out=gl.AccessPattern(torch.empty((16, 16), device="cuda"), 2), flags=gl.GL_OUT_BF16)
+    with pytest.raises(gl.GlError):
+        gl.gl_cartesian_dot(a, None, a, out=gl.AccessPattern(torch.empty((16, 16), device="cuda", dtype=torch.bfloat16), 2))
 
 
 def test_out_nchw_needs_a_conv(gl):
