@@ -238,13 +238,17 @@ def detail_workloads(device, peaks):
     from paper_2105_09377_b200 import synth
     out = []
 
-    def entry(cfg, layout):
+    def entry(cfg, layout, bf16_out=False):
+        from paper_2105_09377_b200 import binding as gl
         nsets = max(2, int((2 * L2_BYTES + cfg.algorithmic_bytes - 1) // cfg.algorithmic_bytes))
         nsets = min(nsets, 32)
         calls, flops, nbytes = [], 0.0, 0
         for _ in range(nsets):
-            c, flops, nbytes = rw.build_call(cfg, layout, device)
+            c, flops, nbytes = rw.build_call(cfg, layout, device, None, gl.GL_OUT_BF16 if bf16_out else 0)
             calls.append(c)
+        if bf16_out:                     # results written as 2-byte elements
+            nbytes -= cfg.n * cfg.ho * cfg.wo * cfg.o * 2
+            layout = layout + "+bf16out"
         med, best = time_graph(calls, 20, device)
         e = {"workload": cfg.name, "us": med * 1e6, "us_best": best * 1e6, "gbs": nbytes / med / 1e9,
              "frac_hbm_peak": nbytes / med / 1e9 / peaks["hbm_gbs"], "buffer_sets": nsets}
@@ -260,6 +264,8 @@ def detail_workloads(device, peaks):
         for layout in ("nhwc", "nchw"):
             entry(cfg, layout)
     entry(synth.CONV_SWEEP_3X3[0], "rewritten")   # the materialised im2col form of Section 5.3, for comparison
+    for cfg in (synth.CONV_SWEEP_3X3[0], synth.CONV_STRIDED_1X1[0], synth.CONV_STRIDED_1X1[1]):
+        entry(cfg, "nhwc", bf16_out=True)         # the two bandwidth-bound shapes with bf16 results
     for cfg in (synth.MEM_IM2COL, synth.MEM_TRANSPOSE, synth.MEM_MAXPOOL, synth.MEM_RELU, synth.MEM_PAD):
         entry(cfg, "")
     return out
