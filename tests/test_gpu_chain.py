@@ -66,3 +66,25 @@ def test_conv_relu_maxpool_dense_chain(gl):
     ref = np.maximum(brute.rowdot(ref_pool.reshape(n, -1).astype(np.float32), dense_w), 0.0)
     assert logits.shape == ((n, units), ())
     assert np.array_equal(logits.tensor.cpu().numpy().astype(np.float64), ref)
+
+
+def test_two_convolutions_chained_through_bf16_results(gl):
+    """conv -> relu -> conv with channels-last items: the first layer stores its results as bf16 (GL_OUT_BF16), which
+    is exactly the operand the second layer reads.  Three input channels keep the first layer's results below 256,
+    so they are exact in bf16 and the whole chain is bit for bit the checker's."""
+    n, c, h, w, o1, o2 = 2, 3, 17, 19, 8, 16
+    x = synth.uniform_int(63, 1, (n, c, h, w), -3, 3)
+    w1 = synth.uniform_int(63, 2, (o1, c, 3, 3), -3, 3)
+    w2 = synth.uniform_int(63, 3, (o2, o1, 3, 3), -3, 3)
+    nhwc = lambda t: np.ascontiguousarray(t.transpose(0, 2, 3, 1))
+    spec1 = gl.windows_spec((3, 3, c), (1, 1, 1), (1, 1, 0), (1, 1, 0))
+    y1 = gl.gl_cartesian_dot(gl.AccessPattern(to_bf16_device(nhwc(x)), 1), spec1, gl.AccessPattern(to_bf16_device(nhwc(w1)), 1),
+                             flags=gl.GL_OUT_BF16 | gl.GL_EPILOGUE_RELU)          # ((N,H,W,1,O1),()) in bf16
+    act = gl.AccessPattern(y1.tensor.view(n, h, w, o1), 1)                        # squeeze: items (H,W,O1)
+    spec2 = gl.windows_spec((3, 3, o1), (2, 2, 1), (1, 1, 0), (1, 1, 0))
+    y2 = gl.gl_cartesian_dot(act, spec2, gl.AccessPattern(to_bf16_device(nhwc(w2)), 1))
+    assert gl.gl_poll_device_status() == 0
+    r1 = np.maximum(brute.conv2d(x, w1, (1, 1), ((1, 1), (1, 1))), 0.0)
+    assert r1.max() <= 256.0
+    r2 = brute.conv2d(r1.astype(np.float32), w2, (2, 2), ((1, 1), (1, 1))).transpose(0, 2, 3, 1)
+    assert np.array_equal(y2.tensor.squeeze(3).cpu().numpy().astype(np.float64), r2)
