@@ -258,6 +258,37 @@ __global__ void __launch_bounds__(kThreads) pad_kernel(const V* __restrict__ in,
   }
 }
 
+// pad of the innermost dimension, 4-byte elements, short rows: the output is walked as one flat array in
+// 16-byte pieces (all lanes busy whatever the row length); the row of each element comes from one
+// multiply-high division per piece and a carry test per element.
+__global__ void __launch_bounds__(kThreads) pad_rows_flat(const uint32_t* __restrict__ in, uint32_t* __restrict__ out,
+                                                          int64_t total, int d_in, int lo, int d_out, uint32_t mul,
+                                                          uint32_t shift, uint32_t fill) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const int64_t pieces = total >> 2;
+  for (int64_t pc = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; pc < pieces; pc += (int64_t)gridDim.x * blockDim.x) {
+    const uint32_t o = static_cast<uint32_t>(pc) << 2;         // total < 2^31
+    uint32_t r = d_out == 1 ? o : (__umulhi(o, mul) >> shift);
+    int c = static_cast<int>(o - r * static_cast<uint32_t>(d_out));
+    uint32_t v[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const int x = c - lo;
+      v[i] = (x >= 0 && x < d_in) ? in[static_cast<int64_t>(r) * d_in + x] : fill;
+      if (++c == d_out) { c = 0; ++r; }
+    }
+    reinterpret_cast<uint4*>(out)[pc] = make_uint4(v[0], v[1], v[2], v[3]);
+  }
+  // the last total % 4 elements
+  if (blockIdx.x == 0 && threadIdx.x < (total & 3)) {
+    const int64_t o = (pieces << 2) + threadIdx.x;
+    const int64_t r = o / d_out;
+    const int x = static_cast<int>(o - r * d_out) - lo;
+    out[o] = (x >= 0 && x < d_in) ? in[r * d_in + x] : fill;
+  }
+}
+
 // pad of the innermost dimension: one warp per row, no divisions.
 template <typename T>
 __global__ void __launch_bounds__(kThreads) pad_rows(const T* __restrict__ in, T* __restrict__ out, int64_t rows,
@@ -868,6 +899,17 @@ int gl_access_pad(const gl_ap* in, int32_t dim, int64_t lo, int64_t hi, int32_t 
         static_cast<const uint4*>(in->data), static_cast<uint4*>(out->data), outer, d_in, lo, d_out, inner / vec, fill);
   } else if (inner == 1 && d_out < (1ll << 30)) {
     const unsigned blocks = static_cast<unsigned>(std::min<int64_t>((outer + 7) / 8, 148 * 32));
+    if (in->dtype == GL_F32 && d_out <= 512 && outer * d_out < (1ll << 31)) {
+      // multiply-high division by d_out for n < 2^31: p = ceil(log2 d), m = ceil(2^(31+p) / d), n / d = umulhi(n, m) >> (p - 1)
+      uint32_t pw2 = 0;
+      while ((1ull << pw2) < static_cast<uint64_t>(d_out)) ++pw2;
+      const uint32_t mul = pw2 ? static_cast<uint32_t>(((1ull << (31 + pw2)) + d_out - 1) / d_out) : 0u;
+      const int64_t total = outer * d_out;
+      const unsigned fblocks = static_cast<unsigned>(std::min<int64_t>((total / 4 + kThreads - 1) / kThreads + 1, 148 * 32));
+      return launch_pdl(pad_rows_flat, dim3(fblocks), dim3(kThreads), 0, st, 1, static_cast<const uint32_t*>(in->data),
+                        static_cast<uint32_t*>(out->data), total, (int)d_in, (int)lo, (int)d_out, mul,
+                        pw2 ? pw2 - 1 : 0u, Fill<uint32_t>::value(pad_kind)) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+    }
     if (in->dtype == GL_F32)
       return launch_pdl(pad_rows<uint32_t>, dim3(blocks), dim3(kThreads), 0, st, 1, static_cast<const uint32_t*>(in->data),
                         static_cast<uint32_t*>(out->data), outer, (int)d_in, (int)lo, (int)d_out,

@@ -113,6 +113,7 @@ def test_im2col_full_size(gl):
 @pytest.mark.parametrize("shape,na,dim,lo,hi,kind", [
     ((2, 3, 5, 8), 1, 2, 1, 1, 0), ((2, 3, 5, 8), 1, 3, 2, 0, 0), ((2, 3, 5, 7), 2, 3, 1, 3, 1),
     ((4, 6), 1, 0, 0, 2, 1), ((9,), 0, 0, 3, 3, 0), ((2, 3, 4), 1, 1, 0, 0, 0),
+    ((5, 1), 1, 1, 0, 0, 0), ((7, 3), 1, 1, 0, 2, 1), ((33, 61), 1, 1, 5, 1, 0), ((3, 700), 1, 1, 1, 1, 0),
 ])
 def test_pad(gl, shape, na, dim, lo, hi, kind, dtype):
     x = synth.uniform(9, 1, shape, -1.0, 1.0)
