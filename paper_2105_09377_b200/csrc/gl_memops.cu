@@ -388,10 +388,22 @@ __global__ void __launch_bounds__(kThreads) window_max_generic(const float* __re
 // Indexing is by warp (one staged row, then one output row per warp pass), so
 // the inner loops carry no divisions; the staged row pitch is chosen on the host
 // to spread the (c,kh,kw) gather over the shared-memory banks.
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void st_shared16(uint32_t smem_dst, const uint4& v) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
 struct Im2colParams {
   int64_t N, C, H, W, Kh, Kw, Sh, Sw, ph_lo, pw_lo, Ho, Wo, K;
   int Wp;       // staged row length = W + pw_lo + pw_hi
   int pitch;    // staged row pitch in elements (>= Wp)
+  int aligned;  // rows staged 16-byte aligned behind a margin of one 16-byte piece (W a multiple of it)
+  int cparts;   // blocks per (n, h'): each takes C / cparts channels, i.e. K / cparts of the columns
+  int slide;    // > 0: output columns per sliding-window item (4-byte elements, Sw = 1, Kw >= 3)
 };
 
 template <typename T, int VEC>
@@ -400,63 +412,65 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
   extern __shared__ __align__(16) unsigned char smem_raw[];
   pdl_wait();
   pdl_launch_dependents();
-  int* lut = reinterpret_cast<int*>(smem_raw);                     // K entries: staged offset of column k at w'=0
-  T* stage = reinterpret_cast<T*>(smem_raw + (((p.K + p.C * p.Kh) * 4 + 15) / 16) * 16);   // [C*Kh][pitch]
-  const int64_t n = blockIdx.x / p.Ho, ho = blockIdx.x % p.Ho;
+  // the grid is N * Ho * cparts blocks, below 2^31; this block owns channels [c0, c0 + Cb) = columns [k0, k0 + K)
+  const unsigned Ho32 = static_cast<unsigned>(p.Ho), parts = static_cast<unsigned>(p.cparts);
+  const unsigned part = blockIdx.x % parts, slab_id = blockIdx.x / parts;
+  const int64_t n = slab_id / Ho32, ho = slab_id % Ho32;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-  const int rows = static_cast<int>(p.C * p.Kh), Kw = static_cast<int>(p.Kw), Kh = static_cast<int>(p.Kh);
-  const int K = static_cast<int>(p.K), W = static_cast<int>(p.W), pw = static_cast<int>(p.pw_lo);
-  for (int k = threadIdx.x; k < K; k += blockDim.x) lut[k] = (k / Kw) * p.pitch + k % Kw;
+  const int Cb = static_cast<int>(p.C) / p.cparts, c0 = static_cast<int>(part) * Cb;
+  const int Kw = static_cast<int>(p.Kw), Kh = static_cast<int>(p.Kh), rows = Cb * Kh;
+  const int Kfull = static_cast<int>(p.K), K = Kfull / p.cparts, k0 = static_cast<int>(part) * K;
+  const int W = static_cast<int>(p.W), pw = static_cast<int>(p.pw_lo);
+  int* lut = reinterpret_cast<int*>(smem_raw);                     // K entries: staged offset of column k at w'=0
+  T* stage = reinterpret_cast<T*>(smem_raw + (((K + rows) * 4 + 15) / 16) * 16);   // [Cb*Kh][pitch]
   const int64_t h0 = ho * p.Sh - p.ph_lo;
-  // staging: four rows per warp pass so that several global loads are in flight per thread
-  constexpr int LV = 16 / sizeof(T);   // elements per 128-bit load
-  if (p.W % LV == 0) {
-    // rows are 16-byte multiples.  rowoff[r] = offset of staged row r inside this image, or -1
-    // for a row of border cells; then every thread takes 128-bit pieces of the flattened
-    // (row, piece) space, four loads in flight each.
-    int* rowoff = lut + K;   // the host reserves rows more ints behind the gather table
-    for (int r = threadIdx.x; r < rows; r += blockDim.x) {
-      const int c = r / Kh, kh = r - c * Kh;
-      const int64_t h = h0 + kh;
-      rowoff[r] = (h >= 0 && h < p.H) ? static_cast<int>((c * p.H + h) * p.W) : -1;
-    }
-    const int border = p.Wp - W;
-    for (int e = threadIdx.x; e < rows * border; e += blockDim.x) {
-      const int r = e / border, j = e - r * border;
-      stage[r * p.pitch + (j < pw ? j : W + j)] = fill;
-    }
-    __syncthreads();
-    const T* image = in + n * p.C * p.H * p.W;
-    const int wv = W / LV, slots = rows * wv;
+  constexpr int LV = 16 / sizeof(T);   // elements per 16-byte piece
+  if (p.aligned) {
+    // Rows are 16-byte multiples and staged 16-byte aligned: cell w of a row sits at column LV + w, the
+    // border cells left and right of it.  Every row piece is one asynchronous 16-byte copy, all of them
+    // issued before the gather table is built, so the block waits for one round trip to L2 only.
+    // The loop below is all 32-bit adds: row, channel and addresses advance incrementally.
+    const int wv = W / LV;
+    int lg = 0;
+    while ((1 << lg) < wv && lg < 5) ++lg;            // 2^lg threads per staged row
+    const int lpr = 1 << lg, rpp = blockDim.x >> lg;  // rows per pass
+    const int li = threadIdx.x & (lpr - 1);
+    const int H32 = static_cast<int>(p.H);
+    const unsigned char* image = reinterpret_cast<const unsigned char*>(in + (n * p.C + c0) * p.H * p.W) + li * 16;
     union Vec { uint4 v; T e[LV]; };
-    for (int s0 = threadIdx.x; s0 < slots; s0 += 4 * blockDim.x) {
-      Vec v[4];
-      int at[4];
+    Vec fv;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int sl = s0 + i * blockDim.x;
-        at[i] = -1;
-        if (sl < slots) {
-          const int r = sl / wv, l = sl - r * wv;
-          at[i] = r * p.pitch + pw + l * LV;
-          const int off = rowoff[r];
-          if (off >= 0) {
-            v[i].v = *reinterpret_cast<const uint4*>(image + off + l * LV);
-          } else {
-#pragma unroll
-            for (int e = 0; e < LV; ++e) v[i].e[e] = fill;
-          }
-        }
+    for (int e = 0; e < LV; ++e) fv.e[e] = fill;
+    int r = threadIdx.x >> lg;
+    int c = r / Kh, kh = r - c * Kh;
+    const int dc = rpp / Kh, dkh = rpp - dc * Kh;
+    const int hbase = static_cast<int>(h0);
+    const int rowbytes = W * static_cast<int>(sizeof(T));
+    uint32_t sdst = static_cast<uint32_t>(__cvta_generic_to_shared(stage)) +
+                    static_cast<uint32_t>((r * p.pitch + LV + li * LV) * static_cast<int>(sizeof(T)));
+    const uint32_t sstep = static_cast<uint32_t>(rpp * p.pitch * static_cast<int>(sizeof(T)));
+    for (; r < rows; r += rpp) {
+      const int h = hbase + kh;
+      const bool inside = static_cast<unsigned>(h) < static_cast<unsigned>(H32);
+      const unsigned char* grow = image + static_cast<int64_t>(c * H32 + h) * rowbytes;   // C*H*W fits 31 bits
+      for (int l = li, o = 0; l < wv; l += lpr, o += lpr * 16) {
+        if (inside) cp_async16(sdst + o, grow + o);
+        else st_shared16(sdst + o, fv.v);
       }
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        if (at[i] >= 0) {
-#pragma unroll
-          for (int e = 0; e < LV; ++e) stage[at[i] + e] = v[i].e[e];
-        }
-      }
+      kh += dkh; c += dc;
+      if (kh >= Kh) { kh -= Kh; ++c; }
+      sdst += sstep;
     }
+    const int border = p.Wp - LV - W + pw;            // border cells per row: pw left, the rest right
+    for (int e = threadIdx.x; e < rows * border; e += blockDim.x) {
+      const int rr = e / border, j = e - rr * border;
+      stage[rr * p.pitch + (j < pw ? LV - pw + j : LV + W + (j - pw))] = fill;
+    }
+    cp_async_commit();
+    for (int k = threadIdx.x; k < K; k += blockDim.x) lut[k] = (k / Kw) * p.pitch + k % Kw + (LV - pw);
+    cp_async_wait_all();
   } else {
+    for (int k = threadIdx.x; k < K; k += blockDim.x) lut[k] = (k / Kw) * p.pitch + k % Kw;
     for (int r0 = warp * 4; r0 < rows; r0 += nwarps * 4) {
       for (int x = lane; x < p.Wp; x += 32) {
         const int w = x - pw;
@@ -467,7 +481,7 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
           const int r = r0 + i;
           const int c = r / Kh, kh = r - c * Kh;
           const int64_t h = h0 + kh;
-          v[i] = (r < rows && col_ok && h >= 0 && h < p.H) ? in[((n * p.C + c) * p.H + h) * p.W + w] : fill;
+          v[i] = (r < rows && col_ok && h >= 0 && h < p.H) ? in[((n * p.C + c0 + c) * p.H + h) * p.W + w] : fill;
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i)
@@ -476,9 +490,44 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
     }
   }
   __syncthreads();
-  T* slab = out + (n * p.Ho + ho) * p.Wo * p.K;
+  T* slab = out + (n * p.Ho + ho) * p.Wo * p.K + k0;   // rows of Kfull columns, this block's start at k0
   const int Wo = static_cast<int>(p.Wo), Sw = static_cast<int>(p.Sw);
   union Chunk { uint4 v; T e[VEC]; };
+  if (VEC == 4 && p.slide > 0) {
+    // Sw = 1: the 16-byte piece (columns k..k+3) of output row w'+1 is the piece of row w' moved one
+    // cell along its staged rows.  With Kw >= 3 a piece touches at most two staged rows, so a thread that
+    // keeps its piece in registers and walks along w' reads two new cells per store instead of four.
+    // Work items are (8 pieces, p.slide consecutive w'), one per quarter warp: every store of a quarter is
+    // one whole 128-byte line.  Neighbouring quarters take neighbouring segments; with an odd segment
+    // length their staged columns differ modulo 4, which keeps them on different shared-memory banks
+    // (rows start on 16-byte boundaries, so one column of different rows covers eight banks only).
+    const int L = p.slide, ppr = K / 4, groups = (ppr + 7) / 8, segs = (Wo + L - 1) / L;
+    const int qi = threadIdx.x >> 3, nq = blockDim.x >> 3, ql = threadIdx.x & 7;
+    for (int item = qi; item < groups * segs; item += nq) {
+      const int g = item / segs, seg = item - g * segs;
+      const int piece = g * 8 + ql;
+      if (piece >= ppr) continue;
+      const int k = piece * 4, wo0 = seg * L, cnt = min(L, Wo - wo0);
+      const int4 a = *reinterpret_cast<const int4*>(lut + k);
+      const int la = a.y != a.x + 1 ? 1 : a.z != a.y + 1 ? 2 : a.w != a.z + 1 ? 3 : 4;   // cells in the first staged row
+      const T* srcA = stage + (la == 1 ? a.x : la == 2 ? a.y : la == 3 ? a.z : a.w) + wo0;
+      const T* srcB = stage + a.w + wo0;
+      T* o = slab + static_cast<int64_t>(wo0) * Kfull + k;
+      Chunk ch;
+      ch.e[0] = stage[a.x + wo0]; ch.e[1] = stage[a.y + wo0]; ch.e[2] = stage[a.z + wo0]; ch.e[3] = stage[a.w + wo0];
+      *reinterpret_cast<uint4*>(o) = ch.v;
+      for (int j = 1; j < cnt; ++j) {
+        const T na = srcA[j], nb = srcB[j];
+        ch.e[0] = la == 1 ? na : ch.e[1];
+        ch.e[1] = la == 2 ? na : ch.e[2];
+        ch.e[2] = la == 3 ? na : ch.e[3];
+        ch.e[3] = la == 4 ? na : nb;
+        o += Kfull;
+        *reinterpret_cast<uint4*>(o) = ch.v;
+      }
+    }
+    return;
+  }
   constexpr int kLutPasses = 5;
   int lutreg[kLutPasses][VEC];
   if (VEC > 1 && K <= kLutPasses * 32 * VEC) {
@@ -492,7 +541,7 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
   }
   for (int wo = warp; wo < Wo; wo += nwarps) {
     const T* base = stage + wo * Sw;
-    T* orow = slab + static_cast<int64_t>(wo) * K;
+    T* orow = slab + static_cast<int64_t>(wo) * Kfull;
     if (VEC == 1) {
       for (int k = lane; k < K; k += 32) orow[k] = base[lut[k]];
     } else if (K <= kLutPasses * 32 * VEC) {
@@ -520,9 +569,10 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
 
 // Row pitch (>= Wp, < Wp + 32) with the fewest shared-memory bank conflicts for the
 // gather "lane reads staged[(k/Kw)*pitch + k%Kw], k = VEC*lane + i" (4-byte banks).
-int best_im2col_pitch(int Wp, int Kw, int K, int vec, int elem_bytes) {
-  int best = Wp, best_cost = 1 << 30;
-  for (int pitch = Wp; pitch < Wp + 32; ++pitch) {
+int best_im2col_pitch(int Wp, int Kw, int K, int vec, int elem_bytes, int step = 1) {
+  const int first = (Wp + step - 1) / step * step;   // pitches are multiples of step
+  int best = first, best_cost = 1 << 30;
+  for (int pitch = first; pitch < first + 32; pitch += step) {
     int cost = 0;
     for (int pass = 0; pass * 32 * vec < K && pass < 8; ++pass)
       for (int i = 0; i < vec; ++i) {
@@ -826,18 +876,37 @@ int run_windows(const gl_ap* in, const gl_windows* w, const gl_ap& A, gl_ap* out
     p.ph_lo = w->pad_lo[1]; p.pw_lo = w->pad_lo[2];
     p.Ho = A.shape[na + 1]; p.Wo = A.shape[na + 2];
     p.K = p.C * p.Kh * p.Kw;
-    const int64_t wp = p.W + w->pad_lo[2] + w->pad_hi[2];
-    const bool vec = p.K % VEC == 0;
+    // rows that are whole 16-byte pieces are staged 16-byte aligned behind a margin of one piece
+    const bool aligned = p.W % VEC == 0 && w->pad_lo[2] <= VEC;
+    const int64_t wp = p.W + (aligned ? VEC : w->pad_lo[2]) + w->pad_hi[2];
+    // Two blocks per (n, h'), half the channels each, when the halves of an output row are whole 128-byte
+    // lines: the same work in more, shorter blocks (a shorter last wave, more warps per SM in flight).
+    p.cparts = (p.C % 2 == 0 && (p.K / 2 * sizeof(T)) % 128 == 0 && p.N * p.Ho < (1ll << 30)) ? 2 : 1;
+    const int64_t Kb = p.K / p.cparts, rows_b = p.C / p.cparts * p.Kh;
+    const bool vec = Kb % VEC == 0;
     const int pitch = wp < (1 << 20) && p.K < (1 << 24)
-                          ? best_im2col_pitch(static_cast<int>(wp), static_cast<int>(p.Kw), static_cast<int>(p.K),
-                                              vec ? VEC : 1, static_cast<int>(sizeof(T)))
-                          : static_cast<int>(wp);
-    const int64_t smem = (((p.K + p.C * p.Kh) * 4 + 15) / 16) * 16 + p.C * p.Kh * pitch * (int64_t)sizeof(T);
-    const int64_t blocks = p.N * p.Ho;
+                          ? best_im2col_pitch(static_cast<int>(wp), static_cast<int>(p.Kw), static_cast<int>(Kb),
+                                              vec ? VEC : 1, static_cast<int>(sizeof(T)), aligned ? VEC : 1)
+                          : static_cast<int>((wp + VEC - 1) / VEC * VEC);
+    const int64_t smem = (((Kb + rows_b) * 4 + 15) / 16) * 16 + rows_b * pitch * (int64_t)sizeof(T);
+    const int64_t blocks = p.N * p.Ho * p.cparts;
     if (smem <= kIm2colMaxSmem && smem <= device_smem_optin() && blocks <= 0x7FFFFFFF && p.Wo * p.K < (1ll << 30) &&
         p.C * p.H * p.W < (1ll << 31)) {
       p.Wp = static_cast<int>(wp);
       p.pitch = pitch;
+      p.aligned = aligned ? 1 : 0;
+      p.slide = 0;
+      if (vec && sizeof(T) == 4 && p.Sw == 1 && p.Kw >= 3 && p.Wo >= 2) {
+        // item length that minimises (rounds over the block's quarter warps) x (loads per item); odd
+        // lengths only (see the kernel)
+        const int64_t groups = (Kb / 4 + 7) / 8, nq = kThreads / 8;
+        int64_t best_cost = INT64_MAX;
+        for (int64_t L = p.Wo >= 3 ? 3 : 1; L <= p.Wo; L += 2) {
+          const int64_t items = groups * ((p.Wo + L - 1) / L);
+          const int64_t cost = ((items + nq - 1) / nq) * (2 * L + 2);
+          if (cost < best_cost) { best_cost = cost; p.slide = static_cast<int>(L); }
+        }
+      }
       auto kern = vec ? im2col_rows<T, VEC> : im2col_rows<T, 1>;
       static bool attr_done[64][2] = {{false}};   // per device and kernel variant
       int dev = 0;
