@@ -397,8 +397,28 @@ __device__ __forceinline__ void st_shared16(uint32_t smem_dst, const uint4& v) {
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
+// Division of n < 2^31 by a divisor fixed on the host: p = ceil(log2 d), mul = ceil(2^(31+p) / d),
+// n / d = umulhi(n, mul) >> (p - 1); mul = 0 stands for d = 1.  An integer division on the device costs
+// some twenty-five instructions, and a block of im2col_rows needs a dozen of them per thread.
+struct FastDiv {
+  uint32_t mul, shift;
+};
+inline FastDiv make_fastdiv(int64_t d) {
+  uint32_t pw2 = 0;
+  while ((1ull << pw2) < static_cast<uint64_t>(d)) ++pw2;
+  FastDiv fd;
+  fd.mul = pw2 ? static_cast<uint32_t>(((1ull << (31 + pw2)) + d - 1) / d) : 0u;
+  fd.shift = pw2 ? pw2 - 1 : 0u;
+  return fd;
+}
+__device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& fd) { return fd.mul ? __umulhi(n, fd.mul) >> fd.shift : n; }
+
 struct Im2colParams {
   int64_t N, C, H, W, Kh, Kw, Sh, Sw, ph_lo, pw_lo, Ho, Wo, K;
+  FastDiv by_Ho, by_Kh, by_Kw, by_border, by_segs;   // divisors: Ho, Kh, Kw, border cells per row, segments per row
+  int Cb, Kb;       // channels and columns per block (C / cparts, K / cparts)
+  int lg, dc, dkh;  // aligned staging: 2^lg threads per row; channel and kernel-row step per pass
+  int groups, segs; // sliding gather: 8-piece groups per row part, segments per output row
   int Wp;       // staged row length = W + pw_lo + pw_hi
   int pitch;    // staged row pitch in elements (>= Wp)
   int aligned;  // rows staged 16-byte aligned behind a margin of one 16-byte piece (W a multiple of it)
@@ -413,13 +433,14 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
   pdl_wait();
   pdl_launch_dependents();
   // the grid is N * Ho * cparts blocks, below 2^31; this block owns channels [c0, c0 + Cb) = columns [k0, k0 + K)
-  const unsigned Ho32 = static_cast<unsigned>(p.Ho), parts = static_cast<unsigned>(p.cparts);
-  const unsigned part = blockIdx.x % parts, slab_id = blockIdx.x / parts;
-  const int64_t n = slab_id / Ho32, ho = slab_id % Ho32;
+  const unsigned part = blockIdx.x & static_cast<unsigned>(p.cparts - 1);   // cparts is 1 or 2
+  const unsigned slab_id = blockIdx.x >> (p.cparts - 1);
+  const unsigned n32 = fdiv(slab_id, p.by_Ho);
+  const int64_t n = n32, ho = slab_id - n32 * static_cast<unsigned>(p.Ho);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-  const int Cb = static_cast<int>(p.C) / p.cparts, c0 = static_cast<int>(part) * Cb;
+  const int Cb = p.Cb, c0 = static_cast<int>(part) * Cb;
   const int Kw = static_cast<int>(p.Kw), Kh = static_cast<int>(p.Kh), rows = Cb * Kh;
-  const int Kfull = static_cast<int>(p.K), K = Kfull / p.cparts, k0 = static_cast<int>(part) * K;
+  const int Kfull = static_cast<int>(p.K), K = p.Kb, k0 = static_cast<int>(part) * K;
   const int W = static_cast<int>(p.W), pw = static_cast<int>(p.pw_lo);
   int* lut = reinterpret_cast<int*>(smem_raw);                     // K entries: staged offset of column k at w'=0
   T* stage = reinterpret_cast<T*>(smem_raw + (((K + rows) * 4 + 15) / 16) * 16);   // [Cb*Kh][pitch]
@@ -431,8 +452,7 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
     // issued before the gather table is built, so the block waits for one round trip to L2 only.
     // The loop below is all 32-bit adds: row, channel and addresses advance incrementally.
     const int wv = W / LV;
-    int lg = 0;
-    while ((1 << lg) < wv && lg < 5) ++lg;            // 2^lg threads per staged row
+    const int lg = p.lg;                              // 2^lg threads per staged row
     const int lpr = 1 << lg, rpp = blockDim.x >> lg;  // rows per pass
     const int li = threadIdx.x & (lpr - 1);
     const int H32 = static_cast<int>(p.H);
@@ -442,8 +462,8 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
 #pragma unroll
     for (int e = 0; e < LV; ++e) fv.e[e] = fill;
     int r = threadIdx.x >> lg;
-    int c = r / Kh, kh = r - c * Kh;
-    const int dc = rpp / Kh, dkh = rpp - dc * Kh;
+    int c = static_cast<int>(fdiv(r, p.by_Kh)), kh = r - c * Kh;
+    const int dc = p.dc, dkh = p.dkh;                 // rows per pass = dc * Kh + dkh
     const int hbase = static_cast<int>(h0);
     const int rowbytes = W * static_cast<int>(sizeof(T));
     uint32_t sdst = static_cast<uint32_t>(__cvta_generic_to_shared(stage)) +
@@ -463,11 +483,14 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
     }
     const int border = p.Wp - LV - W + pw;            // border cells per row: pw left, the rest right
     for (int e = threadIdx.x; e < rows * border; e += blockDim.x) {
-      const int rr = e / border, j = e - rr * border;
+      const int rr = static_cast<int>(fdiv(e, p.by_border)), j = e - rr * border;
       stage[rr * p.pitch + (j < pw ? LV - pw + j : LV + W + (j - pw))] = fill;
     }
     cp_async_commit();
-    for (int k = threadIdx.x; k < K; k += blockDim.x) lut[k] = (k / Kw) * p.pitch + k % Kw + (LV - pw);
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+      const int row = static_cast<int>(fdiv(k, p.by_Kw));
+      lut[k] = row * p.pitch + (k - row * Kw) + (LV - pw);
+    }
     cp_async_wait_all();
   } else {
     for (int k = threadIdx.x; k < K; k += blockDim.x) lut[k] = (k / Kw) * p.pitch + k % Kw;
@@ -501,10 +524,10 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
     // one whole 128-byte line.  Neighbouring quarters take neighbouring segments; with an odd segment
     // length their staged columns differ modulo 4, which keeps them on different shared-memory banks
     // (rows start on 16-byte boundaries, so one column of different rows covers eight banks only).
-    const int L = p.slide, ppr = K / 4, groups = (ppr + 7) / 8, segs = (Wo + L - 1) / L;
+    const int L = p.slide, ppr = K / 4, groups = p.groups, segs = p.segs;
     const int qi = threadIdx.x >> 3, nq = blockDim.x >> 3, ql = threadIdx.x & 7;
     for (int item = qi; item < groups * segs; item += nq) {
-      const int g = item / segs, seg = item - g * segs;
+      const int g = static_cast<int>(fdiv(item, p.by_segs)), seg = item - g * segs;
       const int piece = g * 8 + ql;
       if (piece >= ppr) continue;
       const int k = piece * 4, wo0 = seg * L, cnt = min(L, Wo - wo0);
@@ -895,6 +918,16 @@ int run_windows(const gl_ap* in, const gl_windows* w, const gl_ap& A, gl_ap* out
       p.Wp = static_cast<int>(wp);
       p.pitch = pitch;
       p.aligned = aligned ? 1 : 0;
+      p.Cb = static_cast<int>(p.C / p.cparts);
+      p.Kb = static_cast<int>(Kb);
+      p.by_Ho = make_fastdiv(p.Ho); p.by_Kh = make_fastdiv(p.Kh); p.by_Kw = make_fastdiv(p.Kw);
+      p.by_border = make_fastdiv(std::max<int64_t>(1, wp - p.W - (aligned ? VEC : w->pad_lo[2]) + w->pad_lo[2]));
+      p.lg = 0;
+      while ((1 << p.lg) < p.W / VEC && p.lg < 5) ++p.lg;
+      p.dc = static_cast<int>((kThreads >> p.lg) / p.Kh);
+      p.dkh = static_cast<int>((kThreads >> p.lg) - p.dc * p.Kh);
+      p.groups = p.segs = 1;
+      p.by_segs = make_fastdiv(1);
       p.slide = 0;
       if (vec && sizeof(T) == 4 && p.Sw == 1 && p.Kw >= 3 && p.Wo >= 2) {
         // item length that minimises (rounds over the block's quarter warps) x (loads per item); odd
@@ -906,6 +939,9 @@ int run_windows(const gl_ap* in, const gl_windows* w, const gl_ap& A, gl_ap* out
           const int64_t cost = ((items + nq - 1) / nq) * (2 * L + 2);
           if (cost < best_cost) { best_cost = cost; p.slide = static_cast<int>(L); }
         }
+        p.groups = static_cast<int>(groups);
+        p.segs = static_cast<int>((p.Wo + p.slide - 1) / p.slide);
+        p.by_segs = make_fastdiv(p.segs);
       }
       auto kern = vec ? im2col_rows<T, VEC> : im2col_rows<T, 1>;
       static bool attr_done[64][2] = {{false}};   // per device and kernel variant
