@@ -415,7 +415,7 @@ __device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& fd) { return
 
 struct Im2colParams {
   int64_t N, C, H, W, Kh, Kw, Sh, Sw, ph_lo, pw_lo, Ho, Wo, K;
-  FastDiv by_Ho, by_Kh, by_Kw, by_border, by_segs;   // divisors: Ho, Kh, Kw, border cells per row, segments per row
+  FastDiv by_Ho, by_Kh, by_Kw, by_border, by_segs, by_wv;   // divisors: Ho, Kh, Kw, border cells per row, segments per row, 16-byte pieces per input row
   int Cb, Kb;       // channels and columns per block (C / cparts, K / cparts)
   int lg, dc, dkh;  // aligned staging: 2^lg threads per row; channel and kernel-row step per pass
   int groups, segs; // sliding gather: 8-piece groups per row part, segments per output row
@@ -492,6 +492,57 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
       lut[k] = row * p.pitch + (k - row * Kw) + (LV - pw);
     }
     cp_async_wait_all();
+  } else if (p.W % LV == 0) {
+    // Rows are 16-byte multiples, staged unaligned (any pitch, which matters for the 2-byte gather).
+    // rowoff[r] = offset of staged row r inside this image, or -1 for a row of border cells; then every
+    // thread takes 128-bit pieces of the flattened (row, piece) space, four loads in flight each.
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+      const int row = static_cast<int>(fdiv(k, p.by_Kw));
+      lut[k] = row * p.pitch + (k - row * Kw);
+    }
+    int* rowoff = lut + K;   // the host reserves rows more ints behind the gather table
+    for (int r = threadIdx.x; r < rows; r += blockDim.x) {
+      const int c = static_cast<int>(fdiv(r, p.by_Kh)), kh = r - c * Kh;
+      const int64_t h = h0 + kh;
+      rowoff[r] = (h >= 0 && h < p.H) ? static_cast<int>((c * p.H + h) * p.W) : -1;
+    }
+    const int border = p.Wp - W;
+    for (int e = threadIdx.x; e < rows * border; e += blockDim.x) {
+      const int r = static_cast<int>(fdiv(e, p.by_border)), j = e - r * border;
+      stage[r * p.pitch + (j < pw ? j : W + j)] = fill;
+    }
+    __syncthreads();
+    const T* image = in + (n * p.C + c0) * p.H * p.W;
+    const int wv = W / LV, slots = rows * wv;
+    const FastDiv by_wv = p.by_wv;
+    union Vec { uint4 v; T e[LV]; };
+    for (int s0 = threadIdx.x; s0 < slots; s0 += 4 * blockDim.x) {
+      Vec v[4];
+      int at[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int sl = s0 + i * blockDim.x;
+        at[i] = -1;
+        if (sl < slots) {
+          const int r = static_cast<int>(fdiv(sl, by_wv)), l = sl - r * wv;
+          at[i] = r * p.pitch + pw + l * LV;
+          const int off = rowoff[r];
+          if (off >= 0) {
+            v[i].v = *reinterpret_cast<const uint4*>(image + off + l * LV);
+          } else {
+#pragma unroll
+            for (int e = 0; e < LV; ++e) v[i].e[e] = fill;
+          }
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (at[i] >= 0) {
+#pragma unroll
+          for (int e = 0; e < LV; ++e) stage[at[i] + e] = v[i].e[e];
+        }
+      }
+    }
   } else {
     for (int k = threadIdx.x; k < K; k += blockDim.x) lut[k] = (k / Kw) * p.pitch + k % Kw;
     for (int r0 = warp * 4; r0 < rows; r0 += nwarps * 4) {
@@ -900,7 +951,8 @@ int run_windows(const gl_ap* in, const gl_windows* w, const gl_ap& A, gl_ap* out
     p.Ho = A.shape[na + 1]; p.Wo = A.shape[na + 2];
     p.K = p.C * p.Kh * p.Kw;
     // rows that are whole 16-byte pieces are staged 16-byte aligned behind a margin of one piece
-    const bool aligned = p.W % VEC == 0 && w->pad_lo[2] <= VEC;
+    // (4-byte elements only: a pitch of whole pieces puts the 2-byte gather on few banks)
+    const bool aligned = sizeof(T) == 4 && p.W % VEC == 0 && w->pad_lo[2] <= VEC;
     const int64_t wp = p.W + (aligned ? VEC : w->pad_lo[2]) + w->pad_hi[2];
     // Two blocks per (n, h'), half the channels each, when the halves of an output row are whole 128-byte
     // lines: the same work in more, shorter blocks (a shorter last wave, more warps per SM in flight).
@@ -922,6 +974,7 @@ int run_windows(const gl_ap* in, const gl_windows* w, const gl_ap& A, gl_ap* out
       p.Kb = static_cast<int>(Kb);
       p.by_Ho = make_fastdiv(p.Ho); p.by_Kh = make_fastdiv(p.Kh); p.by_Kw = make_fastdiv(p.Kw);
       p.by_border = make_fastdiv(std::max<int64_t>(1, wp - p.W - (aligned ? VEC : w->pad_lo[2]) + w->pad_lo[2]));
+      p.by_wv = make_fastdiv(std::max<int64_t>(1, p.W / VEC));
       p.lg = 0;
       while ((1 << p.lg) < p.W / VEC && p.lg < 5) ++p.lg;
       p.dc = static_cast<int>((kThreads >> p.lg) / p.Kh);
