@@ -72,6 +72,17 @@ WINDOW_CASES = [
     ((3, 10), 1, (4,), (3,), (1,), (2,), 0),                                # 1D windows, uneven pads
     ((2, 5, 6, 7), 1, (2, 3, 2), (2, 1, 3), (1, 0, 1), (0, 2, 0), 0),       # windows over channels too
     ((2, 6, 4), 1, (6, 4), (1, 1), (0, 0), (0, 0), 0),                      # window == whole item
+    # rows of whole 16-byte pieces (aligned staging), stride 1, Kw >= 3 (sliding gather)
+    ((2, 4, 9, 12), 1, (4, 3, 3), (1, 1, 1), (0, 1, 1), (0, 1, 1), 0),      # K = 36
+    ((2, 64, 5, 8), 1, (64, 3, 3), (1, 1, 1), (0, 1, 1), (0, 1, 1), 0),     # K = 576: two channel halves per slab
+    ((2, 64, 5, 8), 1, (64, 3, 3), (1, 1, 1), (0, 1, 1), (0, 1, 1), 1),     # the same with a -inf border
+    ((1, 4, 8, 16), 1, (4, 5, 5), (1, 1, 1), (0, 2, 2), (0, 2, 2), 0),      # Kw = 5: pieces inside one staged row
+    ((1, 8, 6, 8), 1, (8, 2, 4), (1, 1, 1), (0, 0, 1), (0, 1, 2), 1),       # Kw = 4, uneven pads, two halves
+    ((1, 4, 3, 136), 1, (4, 3, 3), (1, 1, 1), (0, 1, 1), (0, 1, 1), 0),     # rows longer than 32 pieces
+    ((2, 4, 9, 16), 1, (4, 3, 3), (1, 2, 2), (0, 1, 1), (0, 1, 1), 0),      # stride 2: aligned staging, table gather
+    ((1, 4, 6, 8), 1, (4, 3, 7), (1, 1, 1), (0, 1, 5), (0, 1, 1), 0),       # left border wider than one piece
+    ((1, 4, 4, 4), 1, (4, 3, 3), (1, 1, 1), (0, 0, 0), (0, 0, 0), 0),       # two output columns
+    ((3, 16, 4, 60), 1, (16, 3, 3), (1, 1, 1), (0, 1, 1), (0, 1, 1), 0),    # segments with a ragged tail (W' = 60)
 ]
 
 
