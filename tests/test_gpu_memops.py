@@ -83,6 +83,8 @@ WINDOW_CASES = [
     ((1, 4, 6, 8), 1, (4, 3, 7), (1, 1, 1), (0, 1, 5), (0, 1, 1), 0),       # left border wider than one piece
     ((1, 4, 4, 4), 1, (4, 3, 3), (1, 1, 1), (0, 0, 0), (0, 0, 0), 0),       # two output columns
     ((3, 16, 4, 60), 1, (16, 3, 3), (1, 1, 1), (0, 1, 1), (0, 1, 1), 0),    # segments with a ragged tail (W' = 60)
+    ((1, 128, 4, 8), 1, (128, 3, 3), (1, 1, 1), (0, 1, 1), (0, 1, 1), 0),   # K = 1152: two halves for 2-byte elements too
+    ((1, 128, 5, 6), 1, (128, 3, 3), (1, 2, 1), (0, 1, 1), (0, 1, 1), 0),   # two halves, rows that are no whole pieces
 ]
 
 
