@@ -395,6 +395,7 @@ __device__ __forceinline__ void st_shared16(uint32_t smem_dst, const uint4& v) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(smem_dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_but_last() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
 // Division of n < 2^31 by a divisor fixed on the host: p = ceil(log2 d), mul = ceil(2^(31+p) / d),
@@ -419,6 +420,7 @@ struct Im2colParams {
   int Cb, Kb;       // channels and columns per block (C / cparts, K / cparts)
   int lg, dc, dkh;  // aligned staging: 2^lg threads per row; channel and kernel-row step per pass
   int groups, segs; // sliding gather: 8-piece groups per row part, segments per output row
+  int rsplit, gsplit;   // gsplit > 0: two phases; groups [0, gsplit) touch staged rows [0, rsplit) only
   int Wp;       // staged row length = W + pw_lo + pw_hi
   int pitch;    // staged row pitch in elements (>= Wp)
   int aligned;  // rows staged 16-byte aligned behind a margin of one 16-byte piece (W a multiple of it)
@@ -469,29 +471,38 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
     uint32_t sdst = static_cast<uint32_t>(__cvta_generic_to_shared(stage)) +
                     static_cast<uint32_t>((r * p.pitch + LV + li * LV) * static_cast<int>(sizeof(T)));
     const uint32_t sstep = static_cast<uint32_t>(rpp * p.pitch * static_cast<int>(sizeof(T)));
-    for (; r < rows; r += rpp) {
-      const int h = hbase + kh;
-      const bool inside = static_cast<unsigned>(h) < static_cast<unsigned>(H32);
-      const unsigned char* grow = image + static_cast<int64_t>(c * H32 + h) * rowbytes;   // C*H*W fits 31 bits
-      for (int l = li, o = 0; l < wv; l += lpr, o += lpr * 16) {
-        if (inside) cp_async16(sdst + o, grow + o);
-        else st_shared16(sdst + o, fv.v);
+    auto stage_rows = [&](int limit) {
+      for (; r < limit; r += rpp) {
+        const int h = hbase + kh;
+        const bool inside = static_cast<unsigned>(h) < static_cast<unsigned>(H32);
+        const unsigned char* grow = image + static_cast<int64_t>(c * H32 + h) * rowbytes;   // C*H*W fits 31 bits
+        for (int l = li, o = 0; l < wv; l += lpr, o += lpr * 16) {
+          if (inside) cp_async16(sdst + o, grow + o);
+          else st_shared16(sdst + o, fv.v);
+        }
+        kh += dkh; c += dc;
+        if (kh >= Kh) { kh -= Kh; ++c; }
+        sdst += sstep;
       }
-      kh += dkh; c += dc;
-      if (kh >= Kh) { kh -= Kh; ++c; }
-      sdst += sstep;
-    }
+    };
+    // two copy groups when the gather below runs in two phases: rows [0, rsplit) first
+    stage_rows(p.gsplit > 0 ? p.rsplit : rows);
     const int border = p.Wp - LV - W + pw;            // border cells per row: pw left, the rest right
     for (int e = threadIdx.x; e < rows * border; e += blockDim.x) {
       const int rr = static_cast<int>(fdiv(e, p.by_border)), j = e - rr * border;
       stage[rr * p.pitch + (j < pw ? LV - pw + j : LV + W + (j - pw))] = fill;
     }
     cp_async_commit();
+    if (p.gsplit > 0) {
+      stage_rows(rows);
+      cp_async_commit();
+    }
     for (int k = threadIdx.x; k < K; k += blockDim.x) {
       const int row = static_cast<int>(fdiv(k, p.by_Kw));
       lut[k] = row * p.pitch + (k - row * Kw) + (LV - pw);
     }
-    cp_async_wait_all();
+    if (p.gsplit > 0) cp_async_wait_but_last();
+    else cp_async_wait_all();
   } else if (p.W % LV == 0) {
     // Rows are 16-byte multiples, staged unaligned (any pitch, which matters for the 2-byte gather).
     // rowoff[r] = offset of staged row r inside this image, or -1 for a row of border cells; then every
@@ -577,29 +588,40 @@ __global__ void __launch_bounds__(kThreads) im2col_rows(const T* __restrict__ in
     // (rows start on 16-byte boundaries, so one column of different rows covers eight banks only).
     const int L = p.slide, ppr = K / 4, groups = p.groups, segs = p.segs;
     const int qi = threadIdx.x >> 3, nq = blockDim.x >> 3, ql = threadIdx.x & 7;
-    for (int item = qi; item < groups * segs; item += nq) {
-      const int g = static_cast<int>(fdiv(item, p.by_segs)), seg = item - g * segs;
-      const int piece = g * 8 + ql;
-      if (piece >= ppr) continue;
-      const int k = piece * 4, wo0 = seg * L, cnt = min(L, Wo - wo0);
-      const int4 a = *reinterpret_cast<const int4*>(lut + k);
-      const int la = a.y != a.x + 1 ? 1 : a.z != a.y + 1 ? 2 : a.w != a.z + 1 ? 3 : 4;   // cells in the first staged row
-      const T* srcA = stage + (la == 1 ? a.x : la == 2 ? a.y : la == 3 ? a.z : a.w) + wo0;
-      const T* srcB = stage + a.w + wo0;
-      T* o = slab + static_cast<int64_t>(wo0) * Kfull + k;
-      Chunk ch;
-      ch.e[0] = stage[a.x + wo0]; ch.e[1] = stage[a.y + wo0]; ch.e[2] = stage[a.z + wo0]; ch.e[3] = stage[a.w + wo0];
-      *reinterpret_cast<uint4*>(o) = ch.v;
-      for (int j = 1; j < cnt; ++j) {
-        const T na = srcA[j], nb = srcB[j];
-        ch.e[0] = la == 1 ? na : ch.e[1];
-        ch.e[1] = la == 2 ? na : ch.e[2];
-        ch.e[2] = la == 3 ? na : ch.e[3];
-        ch.e[3] = la == 4 ? na : nb;
-        o += Kfull;
+    int item = qi;
+    auto run_items = [&](int limit) {
+      for (; item < limit; item += nq) {
+        const int g = static_cast<int>(fdiv(item, p.by_segs)), seg = item - g * segs;
+        const int piece = g * 8 + ql;
+        if (piece >= ppr) continue;
+        const int k = piece * 4, wo0 = seg * L, cnt = min(L, Wo - wo0);
+        const int4 a = *reinterpret_cast<const int4*>(lut + k);
+        const int la = a.y != a.x + 1 ? 1 : a.z != a.y + 1 ? 2 : a.w != a.z + 1 ? 3 : 4;   // cells in the first staged row
+        const T* srcA = stage + (la == 1 ? a.x : la == 2 ? a.y : la == 3 ? a.z : a.w) + wo0;
+        const T* srcB = stage + a.w + wo0;
+        T* o = slab + static_cast<int64_t>(wo0) * Kfull + k;
+        Chunk ch;
+        ch.e[0] = stage[a.x + wo0]; ch.e[1] = stage[a.y + wo0]; ch.e[2] = stage[a.z + wo0]; ch.e[3] = stage[a.w + wo0];
         *reinterpret_cast<uint4*>(o) = ch.v;
+        for (int j = 1; j < cnt; ++j) {
+          const T na = srcA[j], nb = srcB[j];
+          ch.e[0] = la == 1 ? na : ch.e[1];
+          ch.e[1] = la == 2 ? na : ch.e[2];
+          ch.e[2] = la == 3 ? na : ch.e[3];
+          ch.e[3] = la == 4 ? na : nb;
+          o += Kfull;
+          *reinterpret_cast<uint4*>(o) = ch.v;
+        }
       }
+    };
+    if (p.gsplit > 0) {
+      // the first gsplit groups read staged rows below rsplit only: they are written while the second
+      // copy group is still in flight
+      run_items(p.gsplit * segs);
+      cp_async_wait_all();
+      __syncthreads();
     }
+    run_items(groups * segs);
     return;
   }
   constexpr int kLutPasses = 5;
@@ -980,6 +1002,7 @@ int run_windows(const gl_ap* in, const gl_windows* w, const gl_ap& A, gl_ap* out
       p.dc = static_cast<int>((kThreads >> p.lg) / p.Kh);
       p.dkh = static_cast<int>((kThreads >> p.lg) - p.dc * p.Kh);
       p.groups = p.segs = 1;
+      p.rsplit = p.gsplit = 0;
       p.by_segs = make_fastdiv(1);
       p.slide = 0;
       if (vec && sizeof(T) == 4 && p.Sw == 1 && p.Kw >= 3 && p.Wo >= 2) {
@@ -995,6 +1018,10 @@ int run_windows(const gl_ap* in, const gl_windows* w, const gl_ap& A, gl_ap* out
         p.groups = static_cast<int>(groups);
         p.segs = static_cast<int>((p.Wo + p.slide - 1) / p.slide);
         p.by_segs = make_fastdiv(p.segs);
+        if (aligned && p.Cb >= 2) {
+          p.rsplit = static_cast<int>(p.Cb / 2 * p.Kh);
+          p.gsplit = static_cast<int>(p.rsplit * p.Kw / 32);   // a group is 32 columns; column k reads row k / Kw
+        }
       }
       auto kern = vec ? im2col_rows<T, VEC> : im2col_rows<T, 1>;
       static bool attr_done[64][2] = {{false}};   // per device and kernel variant
