@@ -177,6 +177,8 @@ struct PrepassParams {
   int tiles_c, x_blocks;            // channel tiles; activation blocks = pixel tiles * tiles_c
   int64_t total_pix;                // N * Hs * Ws
   int O, T, wtiles_c, wwarps;       // weight units = O * wtiles_c, wwarps of them per block
+  int fast;                         // total_pix + 64 < 2^31: pixel indices divide by multiply-high
+  FastDiv by_tiles_c, by_npix, by_Ws;
 };
 
 __global__ void __launch_bounds__(256) nchw_prepass(const uint16_t* __restrict__ x, uint16_t* __restrict__ xs,
@@ -219,8 +221,9 @@ __global__ void __launch_bounds__(256) nchw_prepass(const uint16_t* __restrict__
     return;
   }
   constexpr int kPitch = 66;                 // elements per staged channel row
-  const int tc = b % p.tiles_c;
-  const int64_t g0 = static_cast<int64_t>(b / p.tiles_c) * 64;   // first pixel of the tile, counted over all images
+  const int pt = static_cast<int>(fdiv(static_cast<uint32_t>(b), p.by_tiles_c));   // pixel tile
+  const int tc = b - pt * p.tiles_c;
+  const int64_t g0 = static_cast<int64_t>(pt) * 64;   // first pixel of the tile, counted over all images
   const int c0 = tc * 64;
   const int npix = p.Hs * p.Ws;
   const int64_t HW = static_cast<int64_t>(p.H) * p.W;
@@ -232,7 +235,7 @@ __global__ void __launch_bounds__(256) nchw_prepass(const uint16_t* __restrict__
     const int pg = threadIdx.x & 15, cs = threadIdx.x >> 4;
     const int64_t gp = g0 + 4 * pg;
     const bool pok = gp < p.total_pix;
-    const int64_t n = gp / npix;
+    const int64_t n = p.fast ? static_cast<int64_t>(fdiv(static_cast<uint32_t>(gp), p.by_npix)) : gp / npix;
     const uint16_t* src = x + (n * p.C + c0 + cs) * HW + (gp - n * npix);
     uint2 v[4];
 #pragma unroll
@@ -254,9 +257,9 @@ __global__ void __launch_bounds__(256) nchw_prepass(const uint16_t* __restrict__
     for (int j = 0; j < 2; ++j) {
       const int64_t gp = g0 + j * 32 + lane;
       pok[j] = gp < p.total_pix;
-      const int64_t n = gp / npix;
+      const int64_t n = p.fast ? static_cast<int64_t>(fdiv(static_cast<uint32_t>(gp), p.by_npix)) : gp / npix;
       const int pix = static_cast<int>(gp - n * npix);
-      const int hs = pix / p.Ws, wsx = pix - hs * p.Ws;
+      const int hs = static_cast<int>(fdiv(static_cast<uint32_t>(pix), p.by_Ws)), wsx = pix - hs * p.Ws;
       src[j] = x + (n * p.C + c0 + wid) * HW + hs * p.Sh * p.W + wsx * p.Sw;
     }
     uint16_t v[8][2];
@@ -2284,6 +2287,10 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
         pp.wtiles_c = static_cast<int>(tiles_c);
         pp.wwarps = wwarps;
         pp.x_blocks = static_cast<int>(x_blocks);
+        pp.fast = pp.total_pix + 64 < (1ll << 31) ? 1 : 0;
+        pp.by_tiles_c = make_fastdiv(tiles_c);
+        pp.by_npix = make_fastdiv(static_cast<int64_t>(pp.Hs) * pp.Ws);
+        pp.by_Ws = make_fastdiv(pp.Ws);
         if (!copy_w) ws = const_cast<uint16_t*>(pb);
         const size_t smem = std::max<size_t>(64 * 66 * 2, static_cast<size_t>(wwarps) * 64 * T * 2);
         if (launch_pdl(nchw_prepass, dim3(static_cast<unsigned>(x_blocks + w_blocks)), dim3(256), smem, st, 1, pa, xs, pb,

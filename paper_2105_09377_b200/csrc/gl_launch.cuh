@@ -8,10 +8,28 @@
 #pragma once
 #include <cuda_runtime.h>
 
+#include <cstdint>
 #include <cstring>
 #include <utility>
 
 namespace gl {
+
+// Division of n < 2^31 by a divisor fixed on the host: p = ceil(log2 d), mul = ceil(2^(31+p) / d),
+// n / d = umulhi(n, mul) >> (p - 1); mul = 0 stands for d = 1.  An integer division on the device costs
+// some twenty-five instructions (over a hundred for 64-bit operands); kernels whose blocks move a few KB
+// each (im2col_rows, nchw_prepass) need several per thread.
+struct FastDiv {
+  uint32_t mul, shift;
+};
+inline FastDiv make_fastdiv(int64_t d) {
+  uint32_t pw2 = 0;
+  while ((1ull << pw2) < static_cast<uint64_t>(d)) ++pw2;
+  FastDiv fd;
+  fd.mul = pw2 ? static_cast<uint32_t>(((1ull << (31 + pw2)) + d - 1) / d) : 0u;
+  fd.shift = pw2 ? pw2 - 1 : 0u;
+  return fd;
+}
+__device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& fd) { return fd.mul ? __umulhi(n, fd.mul) >> fd.shift : n; }
 
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

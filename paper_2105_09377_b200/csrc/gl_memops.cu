@@ -398,22 +398,6 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 __device__ __forceinline__ void cp_async_wait_but_last() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
-// Division of n < 2^31 by a divisor fixed on the host: p = ceil(log2 d), mul = ceil(2^(31+p) / d),
-// n / d = umulhi(n, mul) >> (p - 1); mul = 0 stands for d = 1.  An integer division on the device costs
-// some twenty-five instructions, and a block of im2col_rows needs a dozen of them per thread.
-struct FastDiv {
-  uint32_t mul, shift;
-};
-inline FastDiv make_fastdiv(int64_t d) {
-  uint32_t pw2 = 0;
-  while ((1ull << pw2) < static_cast<uint64_t>(d)) ++pw2;
-  FastDiv fd;
-  fd.mul = pw2 ? static_cast<uint32_t>(((1ull << (31 + pw2)) + d - 1) / d) : 0u;
-  fd.shift = pw2 ? pw2 - 1 : 0u;
-  return fd;
-}
-__device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& fd) { return fd.mul ? __umulhi(n, fd.mul) >> fd.shift : n; }
-
 struct Im2colParams {
   int64_t N, C, H, W, Kh, Kw, Sh, Sw, ph_lo, pw_lo, Ho, Wo, K;
   FastDiv by_Ho, by_Kh, by_Kw, by_border, by_segs, by_wv;   // divisors: Ho, Kh, Kw, border cells per row, segments per row, 16-byte pieces per input row
