@@ -757,6 +757,7 @@ __global__ void __launch_bounds__(kThreads) window_max_2d_tiled(const float* __r
 struct Pool3s2 {
   int H, W, Ho, Wo, R, strips, w4;
   int64_t units;   // planes * strips
+  FastDiv by_strips;   // used when units < 2^31
 };
 
 template <int R>
@@ -766,7 +767,7 @@ __global__ void __launch_bounds__(256) window_max_3x3s2(const float* __restrict_
   pdl_launch_dependents();
   const int64_t u = blockIdx.x * (int64_t)blockDim.y + threadIdx.y;
   if (u >= p.units) return;
-  const int64_t plane = u / p.strips;
+  const int64_t plane = p.units < (1ll << 31) ? static_cast<int64_t>(fdiv(static_cast<uint32_t>(u), p.by_strips)) : u / p.strips;
   const int strip = static_cast<int>(u - plane * p.strips);
   const float* src = in + plane * p.H * p.W;
   float* dst = out + plane * p.Ho * p.Wo;
@@ -1150,6 +1151,7 @@ int gl_compute_reduce_max(const gl_ap* in, const gl_windows* w, gl_ap* out, void
     t.strips = (t.Ho + t.R - 1) / t.R;
     t.w4 = t.W / 4;
     t.units = prod(in->shape, 0, na) * t.strips;
+    t.by_strips = make_fastdiv(t.strips);
     const int64_t blocks = (t.units + 7) / 8;
     if (blocks <= 0x7FFFFFFF) {
       return launch_pdl(window_max_3x3s2<kRows>, dim3(static_cast<unsigned>(blocks)), dim3(32, 8), 0, st, 1, src, dst, t,
