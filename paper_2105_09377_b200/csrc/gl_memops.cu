@@ -53,13 +53,17 @@ struct TileParams {
   BatchDims batch;
 };
 
-__device__ __forceinline__ void batch_offsets(const BatchDims& b, int64_t idx, int64_t& in_off, int64_t& out_off) {
+// idx is a block index (below 2^32, and so is every extent whose product bounds it): 32-bit divisions,
+// a fifth of the instructions of 64-bit ones, which matters for blocks that move one 16 KB tile.
+__device__ __forceinline__ void batch_offsets(const BatchDims& b, uint32_t idx, int64_t& in_off, int64_t& out_off) {
   in_off = 0;
   out_off = 0;
 #pragma unroll 1
   for (int d = b.n - 1; d >= 0; --d) {
-    const int64_t i = idx % b.size[d];
-    idx /= b.size[d];
+    const uint32_t size = static_cast<uint32_t>(b.size[d]);
+    const uint32_t q = idx / size;
+    const int64_t i = idx - q * size;
+    idx = q;
     in_off += i * b.in_stride[d];
     out_off += i * b.out_stride[d];
   }
@@ -76,9 +80,14 @@ __global__ void __launch_bounds__(kThreads) transpose_tiled_vec(const T* __restr
   __shared__ uint4 tile[TILE][16];
   pdl_wait();
   pdl_launch_dependents();
-  int64_t bid = blockIdx.x;
-  const int64_t tileA = bid % p.tilesA; bid /= p.tilesA;
-  const int64_t tileB = bid % p.tilesB; bid /= p.tilesB;
+  uint32_t bid = blockIdx.x;   // tilesA * tilesB * batch = the grid size: every factor is below 2^32
+  const uint32_t nA = static_cast<uint32_t>(p.tilesA), nB = static_cast<uint32_t>(p.tilesB);
+  const uint32_t qA = bid / nA;
+  const int64_t tileA = bid - qA * nA;
+  bid = qA;
+  const uint32_t qB = bid / nB;
+  const int64_t tileB = bid - qB * nB;
+  bid = qB;
   int64_t in_off, out_off;
   batch_offsets(p.batch, bid, in_off, out_off);
   const int ta = threadIdx.x & 15, tb = threadIdx.x >> 4;
@@ -119,9 +128,14 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads) transpose_tiled_scalar(const T* __restrict__ in, T* __restrict__ out,
                                                                    const TileParams p) {
   __shared__ T tile[32][33];
-  int64_t bid = blockIdx.x;
-  const int64_t tileA = bid % p.tilesA; bid /= p.tilesA;
-  const int64_t tileB = bid % p.tilesB; bid /= p.tilesB;
+  uint32_t bid = blockIdx.x;   // tilesA * tilesB * batch = the grid size: every factor is below 2^32
+  const uint32_t nA = static_cast<uint32_t>(p.tilesA), nB = static_cast<uint32_t>(p.tilesB);
+  const uint32_t qA = bid / nA;
+  const int64_t tileA = bid - qA * nA;
+  bid = qA;
+  const uint32_t qB = bid / nB;
+  const int64_t tileB = bid - qB * nB;
+  bid = qB;
   int64_t in_off, out_off;
   batch_offsets(p.batch, bid, in_off, out_off);
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
