@@ -320,6 +320,54 @@ def test_blocked_32x32_is_eight_16x16_matmuls():
     np.testing.assert_array_equal(blocked.data, gi.matmul_program(p, q).data)
 
 
+# ---- the sampled form of the conv2d equation (used on full-size results) ----
+
+SAMPLED_CASES = [
+    # n, c, h, w, o, kh, kw, sh, sw, ph, pw: strides and pads unequal, N and O above 1
+    (2, 3, 13, 10, 5, 7, 7, 2, 1, 3, 2),     # stem-like 7x7, stride 2 only along H, pads 3 and 2
+    (3, 4, 9, 8, 6, 1, 1, 2, 3, 0, 0),       # 1x1 with strides 2 and 3
+    (2, 2, 7, 11, 3, 3, 2, 1, 2, 1, 0),      # lopsided window, one padded dimension
+]
+
+
+@pytest.mark.parametrize("case", SAMPLED_CASES)
+def test_conv2d_sampled_against_full_brute_torch_and_interpreter(case):
+    # every flat (n,o,x,y) offset, then a shuffled subset with repeats: the values must be the cells of
+    # the full brute-force result, of the interpreter's Fig. 2a program and of torch's conv2d
+    n, c, h, w, o, kh, kw, sh, sw, ph, pw = case
+    x = synth.bf16_round(synth.normal(61, 1, (n, c, h, w)))
+    wt = synth.bf16_round(synth.normal(61, 2, (o, c, kh, kw)))
+    pads = ((ph, ph), (pw, pw))
+    full = brute.conv2d(x, wt, (sh, sw), pads)
+    assert full.shape == brute.conv_out_shape(x.shape, wt.shape, (sh, sw), pads)
+    every = np.arange(full.size, dtype=np.int64)
+    got = brute.conv2d_sampled(x, wt, every, (sh, sw), pads)
+    np.testing.assert_array_equal(got, full.ravel())
+    prog = gi.conv2d_program(x.astype(np.float64), wt.astype(np.float64), (sh, sw), pads).data
+    np.testing.assert_allclose(got, prog.ravel(), rtol=1e-12, atol=1e-12)
+    ref = F.conv2d(torch.from_numpy(x.astype(np.float64)), torch.from_numpy(wt.astype(np.float64)), stride=(sh, sw),
+                   padding=(ph, pw)).numpy()
+    np.testing.assert_allclose(got, ref.ravel(), rtol=1e-12, atol=1e-12)
+    rng = np.random.default_rng(3)
+    pick = rng.integers(0, full.size, 257)
+    np.testing.assert_array_equal(brute.conv2d_sampled(x, wt, pick, (sh, sw), pads), full.ravel()[pick])
+
+
+def test_conv2d_sampled_pin_catches_a_wrong_offset_order():
+    # the pin must tell (n,o,x,y) offsets from (n,x,y,o) offsets: feeding offsets of the other order
+    # (a plausible slip in a caller or in the decode) gives different values
+    n, c, h, w, o, kh, kw = 2, 3, 6, 7, 4, 3, 2
+    x = synth.bf16_round(synth.normal(62, 1, (n, c, h, w)))
+    wt = synth.bf16_round(synth.normal(62, 2, (o, c, kh, kw)))
+    full = brute.conv2d(x, wt)
+    _, _, ho, wo = full.shape
+    nn, oo, xx, yy = np.meshgrid(np.arange(n), np.arange(o), np.arange(ho), np.arange(wo), indexing="ij")
+    right = ((nn * o + oo) * ho + xx) * wo + yy
+    wrong = ((nn * ho + xx) * wo + yy) * o + oo
+    np.testing.assert_array_equal(brute.conv2d_sampled(x, wt, right.ravel()), full.ravel())
+    assert not np.array_equal(brute.conv2d_sampled(x, wt, wrong.ravel()), full.ravel())
+
+
 # ---- sensitivity: a planted mistake in the checker is caught --------------
 
 def test_pins_catch_a_planted_mistake(monkeypatch):
