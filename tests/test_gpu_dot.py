@@ -496,47 +496,107 @@ def test_dense_gaussian_1024_full_check(gl):
     assert rel_err(out.tensor.cpu().numpy(), ref) <= REL_TOL
 
 
-def test_dense_4096_sampled_rows_and_relu(gl):
+@pytest.mark.parametrize("kind", ["integer", "gaussian"])
+def test_dense_4096_whole_result_and_relu(gl, kind):
+    # the whole 4096 x 4096 result against the row-vector form of the matMul equation (Section 3.1)
     case = synth.DENSE_4096
-    a, b = case.inputs(synth.config_seed(1))
+    if kind == "integer":
+        a = synth.uniform_int(synth.config_seed(1), 1, (case.m, case.k), -3, 3)
+        b = synth.uniform_int(synth.config_seed(1), 2, (case.o, case.k), -3, 3)
+    else:
+        a, b = case.inputs(synth.config_seed(1))
     aa, bb = gl.AccessPattern(to_bf16_device(a), 1), gl.AccessPattern(to_bf16_device(b), 1)
     out = gl.gl_cartesian_dot(aa, None, bb, flags=gl.GL_EPILOGUE_RELU)
     _ok(gl)
     got = out.tensor.cpu().numpy()
-    rng = np.random.default_rng(5)
-    rows = np.unique(np.concatenate([rng.integers(0, 4096, 48), [0, 127, 128, 255, 256, 4095]]))
-    ref = np.maximum(brute.rowdot(a, b, rows), 0.0)
-    assert rel_err(got[rows], ref) <= REL_TOL
-    cols = np.unique(np.concatenate([rng.integers(0, 4096, 48), [0, 255, 256, 4095]]))
-    refc = np.maximum(brute.rowdot(b, a, cols), 0.0).T          # columns of out = rows of B against all of A
-    assert rel_err(got[:, cols], refc) <= REL_TOL
-    assert (got >= 0).all()
+    ref = np.maximum(brute.rowdot(a, b), 0.0)
+    if kind == "integer":
+        assert np.array_equal(got.astype(np.float64), ref)      # |sums| <= 9 * 4096 < 2^24: exact in any order
+    else:
+        assert rel_err(got, ref) <= REL_TOL
+    plain = gl.gl_cartesian_dot(aa, None, bb)
+    _ok(gl)
+    assert torch.equal(torch.clamp_min(plain.tensor, 0.0), out.tensor)
 
 
-# ---- the convolution sweeps at full size, on sampled outputs ----
+# ---- the convolution sweeps at full size: the whole result, both layouts, both kinds of input ----
 
 FULL_CONVS = list(synth.CONV_SWEEP_3X3) + list(synth.CONV_STRIDED_1X1)
+_FULL = {}
+
+
+def _full_case(cfg, kind):
+    """Inputs and the brute-force (N,H',W',O) result of a full-size workload, computed once per module."""
+    key = (cfg.name, kind)
+    if key not in _FULL:
+        if kind == "integer":
+            x = synth.uniform_int(synth.config_seed(2), 1, (cfg.n, cfg.c, cfg.h, cfg.w), -3, 3)
+            wt = synth.uniform_int(synth.config_seed(2), 2, (cfg.o, cfg.c, cfg.kh, cfg.kw), -3, 3)
+        else:
+            x, wt = cfg.inputs(synth.config_seed(2))
+        ref = _conv_ref(x, wt, (cfg.stride,) * 2, (cfg.pad,) * 2)
+        if kind == "integer":
+            assert np.abs(ref).max() < 2 ** 24
+            ref = ref.astype(np.float32)                       # integers below 2^24: exact
+        _FULL[key] = (x, wt, np.ascontiguousarray(ref))
+    return _FULL[key]
+
+
+@pytest.mark.parametrize("cfg", FULL_CONVS, ids=[c.name for c in FULL_CONVS])
+@pytest.mark.parametrize("kind", ["integer", "gaussian"])
+@pytest.mark.parametrize("layout", ["nhwc", "nchw"])
+def test_full_size_conv_whole_result(gl, cfg, kind, layout):
+    x, wt, ref = _full_case(cfg, kind)
+    got = _conv_gpu(gl, x, wt, (cfg.stride,) * 2, (cfg.pad,) * 2, channels_last=(layout == "nhwc"))
+    assert got.shape == ref.shape == (cfg.n, cfg.ho, cfg.wo, cfg.o)
+    if kind == "integer":
+        assert np.array_equal(got, ref)
+    else:
+        assert rel_err(got, ref) <= REL_TOL
 
 
 @pytest.mark.parametrize("cfg", FULL_CONVS, ids=[c.name for c in FULL_CONVS])
 @pytest.mark.parametrize("layout", ["nhwc", "nchw"])
-def test_full_size_conv_sampled(gl, cfg, layout):
-    x, wt = cfg.inputs(synth.config_seed(2))
-    got = _conv_gpu(gl, x, wt, (cfg.stride,) * 2, (cfg.pad,) * 2, channels_last=(layout == "nhwc"))
-    assert got.shape == (cfg.n, cfg.ho, cfg.wo, cfg.o)
-    rng = np.random.default_rng(9)
-    cnt = 4096
-    ns, os_ = rng.integers(0, cfg.n, cnt), rng.integers(0, cfg.o, cnt)
-    xs, ys = rng.integers(0, cfg.ho, cnt), rng.integers(0, cfg.wo, cnt)
-    # corners, image borders and tile seams are always in the sample
-    xs[:64] = np.where(rng.integers(0, 2, 64) == 0, 0, cfg.ho - 1)
-    ys[64:128] = np.where(rng.integers(0, 2, 64) == 0, 0, cfg.wo - 1)
-    flat = ((ns * cfg.o + os_) * cfg.ho + xs) * cfg.wo + ys
-    pads = ((cfg.pad, cfg.pad), (cfg.pad, cfg.pad))
-    ref = brute.conv2d_sampled(x, wt, flat, (cfg.stride,) * 2, pads)
-    assert rel_err(got[ns, xs, ys, os_], ref) <= REL_TOL
-    # a property that holds at any size: the last image (ragged final tile) is finite and not all zero
-    assert np.isfinite(got[-1]).all() and np.abs(got[-1]).max() > 0
+def test_full_size_conv_fused_squeeze_transpose(gl, cfg, layout):
+    # GL_OUT_NCHW at full size: the whole program of Fig. 2a, result ((N,O,H',W'),())
+    x, wt, ref = _full_case(cfg, "integer")
+    if layout == "nhwc":
+        xa = gl.AccessPattern(to_bf16_device(np.ascontiguousarray(x.transpose(0, 2, 3, 1))), 1)
+        wa = gl.AccessPattern(to_bf16_device(np.ascontiguousarray(wt.transpose(0, 2, 3, 1))), 1)
+        spec = gl.windows_spec((cfg.kh, cfg.kw, cfg.c), (cfg.stride, cfg.stride, 1), (cfg.pad, cfg.pad, 0), (cfg.pad, cfg.pad, 0))
+    else:
+        xa, wa = gl.AccessPattern(to_bf16_device(x), 1), gl.AccessPattern(to_bf16_device(wt), 1)
+        spec = gl.windows_spec((cfg.c, cfg.kh, cfg.kw), (1, cfg.stride, cfg.stride), (0, cfg.pad, cfg.pad), (0, cfg.pad, cfg.pad))
+    out = gl.gl_cartesian_dot(xa, spec, wa, flags=gl.GL_OUT_NCHW)
+    _ok(gl)
+    assert tuple(out.tensor.shape) == (cfg.n, cfg.o, cfg.ho, cfg.wo)
+    assert np.array_equal(out.tensor.cpu().numpy(), ref.transpose(0, 3, 1, 2))
+
+
+@pytest.mark.parametrize("cfg", FULL_CONVS, ids=[c.name for c in FULL_CONVS])
+def test_full_size_conv_bf16_results(gl, cfg):
+    # GL_OUT_BF16 at full size: the exact integer sums rounded once to the nearest-even bf16
+    x, wt, ref = _full_case(cfg, "integer")
+    got = _conv_gpu(gl, x, wt, (cfg.stride,) * 2, (cfg.pad,) * 2, channels_last=True, flags=gl.GL_OUT_BF16 | gl.GL_EPILOGUE_RELU)
+    assert np.array_equal(got, synth.bf16_round(np.maximum(ref, 0.0)))
+
+
+@pytest.mark.parametrize("kind", ["integer", "gaussian"])
+def test_full_size_rewritten_form_equals_direct(gl, kind):
+    # Section 5.3 at full size: windows materialised (bf16), flattened, plain matrix product, reshape
+    cfg = synth.CONV_SWEEP_3X3[0]
+    x, wt, ref = _full_case(cfg, kind)
+    xa, wa = gl.AccessPattern(to_bf16_device(x), 1), gl.AccessPattern(to_bf16_device(wt), 1)
+    spec = gl.windows_spec((cfg.c, cfg.kh, cfg.kw), (1, 1, 1), (0, cfg.pad, cfg.pad), (0, cfg.pad, cfg.pad))
+    cols = gl.gl_access_flatten(gl.gl_access_windows(xa, spec))
+    mm = gl.gl_cartesian_dot(cols, None, gl.gl_access_flatten(wa))
+    _ok(gl)
+    assert mm.shape == ((cfg.m, cfg.o), ())
+    got = mm.tensor.view(cfg.n, cfg.ho, cfg.wo, cfg.o).cpu().numpy()
+    if kind == "integer":
+        assert np.array_equal(got, ref)
+    else:
+        assert rel_err(got, ref) <= REL_TOL
 
 
 def test_bounded_wait_reports_timeout_and_context_survives(gl):
