@@ -17,6 +17,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -459,6 +460,14 @@ __device__ __forceinline__ void tma_load_im2col_pair(uint32_t dst, const CUtenso
       : "memory");
 }
 
+// One lane of the (converged) warp.  The MMA warps run their loops warp-uniformly and predicate only the
+// tcgen05 instructions on this lane: descriptors and barrier addresses then stay warp-uniform values.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.b32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -664,10 +673,13 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
 
   if (warp == 0 || warp == 6) {
     // ---------------- TMA producers: warp 0 stages A, warp 6 stages B ----------------
-    // (issuing one TMA load costs its thread 150-200 cycles; two issuing warps halve that)
+    // The whole warp runs the loop (warp-uniform control flow and values); one elected lane issues the
+    // copies.  Issued from inside a one-lane branch, every TMA or MMA instruction cost its thread 60-150
+    // cycles of operand shuffling; from uniform code it costs 15-30.
     const bool load_a = warp == 0;
-    if (lane == 0) {
-      uint32_t s = 0, ph = 0;   // ring slot and its phase, advanced by hand (no division in this thread)
+    const bool leader = elect_one();
+    {
+      uint32_t s = 0, ph = 0;   // ring slot and its phase, advanced by hand (no division in this loop)
       bool ok = true;
       for (int u = unit0; u < num_tiles && ok; u += unit_step) {
         uint32_t t, ks, tm, tn;
@@ -707,10 +719,11 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
           const uint32_t full = CTAS == 2 ? map_to_cta(bar_full + 8 * s, 0) : bar_full + 8 * s;
           const uint32_t stage = tiles + s * Cfg::kStage;
           const int nsub = min(G, kb_end - kb0);
-          if (rank == 0) mbar_expect_tx(bar_full + 8 * s, nsub * CTAS * (load_a ? Cfg::kStageA : Cfg::kStageB));
+          if (rank == 0 && leader) mbar_expect_tx(bar_full + 8 * s, nsub * CTAS * (load_a ? Cfg::kStageA : Cfg::kStageB));
 #pragma unroll 1
           for (int j = 0; j < nsub; ++j) {
             const int kb = kb0 + j;
+            if (leader) {
             const uint32_t sa = stage + j * Cfg::kStageA, sb = stage + G * Cfg::kStageA + j * Cfg::kStageB;
             if (CTAS == 2) {
               if (MODE == kDense) {
@@ -722,7 +735,6 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
                                        static_cast<uint16_t>(kh), full);
                 else
                   tma_load_2d_pair(sb, &map_b, (kh * p.Kw + kw) * p.Cp + cc * kBK, n0, full);
-                if (++cc == p.cchunks) { cc = 0; if (++kw == p.Kw) { kw = 0; ++kh; } }
               }
             } else if (MODE == kDense) {
               if (load_a) tma_load_2d(sa, &map_a, kb * kBK, m0, full);
@@ -737,7 +749,6 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
                                 static_cast<uint16_t>(kh), full);
               else
                 tma_load_2d(sb, &map_b, (kh * p.Kw + kw) * p.Cp + cc * kBK, n0, full);
-              if (++cc == p.cchunks) { cc = 0; if (++kw == p.Kw) { kw = 0; ++kh; } }
             } else if (load_a) {
               // eight 8-channel granules per K block, each its own (pixels x 16 bytes) box
               const int taps = p.Kh * p.Kw;
@@ -754,6 +765,9 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
             } else {
               tma_load_3d(sb, &map_b, 0, n0, kb * 8, full);
             }
+            }
+            // filter position of the next K block
+            if (MODE == kIm2col) { if (++cc == p.cchunks) { cc = 0; if (++kw == p.Kw) { kw = 0; ++kh; } } }
           }
           if (++s == Cfg::kStages) { s = 0; ph ^= 1u; }
         }
@@ -761,7 +775,8 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
-    if (lane == 0 && rank == 0) {
+    if (rank == 0) {
+      const bool leader = elect_one();   // the loop is warp-uniform; this lane issues the MMAs and commits
       constexpr uint32_t idesc = make_idesc(kBM * CTAS, BN);
       const uint64_t desc_a0 = (MODE == kIm2colGranule) ? make_desc(tiles, kBM * 16, 128, 0) : make_desc(tiles, 16, 1024, 2);
       const uint64_t desc_b0 = (MODE == kIm2colGranule) ? make_desc(tiles + G * Cfg::kStageA, BN * 16, 128, 0)
@@ -793,18 +808,22 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
                 const uint64_t da = da0 + ((j * Cfg::kStageA + k * kStepA) >> 4);
                 const uint64_t db = db0 + ((j * Cfg::kStageB + k * kStepB) >> 4);
                 const uint32_t accumulate = ((kb0 - kb_begin) | j | k) != 0 ? 1u : 0u;
-                if (CTAS == 2) tc_mma_bf16_pair(d_tmem, da, db, idesc, accumulate);
-                else tc_mma_bf16(d_tmem, da, db, idesc, accumulate);
+                if (leader) {
+                  if (CTAS == 2) tc_mma_bf16_pair(d_tmem, da, db, idesc, accumulate);
+                  else tc_mma_bf16(d_tmem, da, db, idesc, accumulate);
+                }
               }
             }
           }
           // one commit per stage (it costs the issuing thread a few hundred cycles): frees the
           // stage once these MMAs have read it
-          if (CTAS == 2) tc_commit_pair(bar_empty + 8 * s);
-          else tc_commit(bar_empty + 8 * s);
+          if (leader) {
+            if (CTAS == 2) tc_commit_pair(bar_empty + 8 * s);
+            else tc_commit(bar_empty + 8 * s);
+          }
           if (++s == Cfg::kStages) { s = 0; ph ^= 1u; }
         }
-        if (ok) {
+        if (ok && leader) {
           if (CTAS == 2) tc_commit_pair(bar_tfull + 8 * acc);
           else tc_commit(bar_tfull + 8 * acc);
         }
@@ -813,6 +832,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
   } else {
     // ---------------- epilogue: TMEM -> registers -> (shared memory -> TMA store | global) ----------------
     const int q = warp & 3;   // TMEM lane quarter this warp may read
+    const bool leader = elect_one();   // issues this warp's TMA stores (always the same lane: it owns the bulk groups)
     uint32_t tile_it = 0, chunk_it = 0;
     bool ok = true;
     const bool vec_ok = (p.O & 3) == 0;
@@ -889,7 +909,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
           // row, the 128-byte swizzle of the tensor map), then one lane hands the block to the TMA unit,
           // which writes whole 128-byte rows and clips at the matrix edge.
           const uint32_t buf = stage_buf + (Cfg::kEpiBufs == 2 ? (chunk_it & 1u) * 4096 : 0u);
-          if (lane == 0) {   // the store that last used this buffer has read it
+          if (leader) {   // the store that last used this buffer has read it
             if (Cfg::kEpiBufs == 2) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
             else asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
           }
@@ -901,7 +921,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
                          : "memory");
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           __syncwarp();
-          if (lane == 0) {
+          if (leader) {
             if (MODE == kRowWin)   // result viewed as (N*Ho, Wo, O): columns past Wo are clipped
               asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(
                                reinterpret_cast<uint64_t>(&map_c)),
@@ -940,7 +960,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
         else mbar_arrive(bar_tempty + 8 * acc);
       }
     }
-    if (p.tma_store && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (p.tma_store && leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   // teardown: a block that gave up lets its copies in flight land before it leaves
@@ -991,7 +1011,7 @@ struct HaloParams {
   int64_t O;
   int relu;
   int out_bf16;   // results rounded to bf16 (O a multiple of 8)
-  int Ho, Wo, Wb, R, tiles_m, tiles_n;
+  int N, Ho, Wo, Wb, R, tiles_m, tiles_n;   // tiles_m: M tiles, or pairs of them
   int Kh, Kw, Cp, cchunks;
   int tg, groups_per_chunk;                 // a B stage holds tg consecutive taps (a filter row, or one tap) of one chunk
   int ph, pw;
@@ -1008,15 +1028,27 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       : "memory");
 }
 
+__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap* map, int c, int w, int h, int n,
+                                                 uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar)
+      : "memory");
+}
+
 // BN: output channels per tile.  The weights are viewed as (64 channels, O, chunk, tap); one TMA box
 // brings the BN x 64 slices of p.tg consecutive taps of one chunk.
 // OCC = 2 (64-wide tiles): two blocks per SM, each with one input-box stage, so that one block's loads and
 // epilogue run under the other's MMAs.
-template <int BN, int OCC>
+// CTAS = 2: two blocks on neighbouring SMs (a cluster) take two M tiles of the same column tile.  Each block
+// stages the input box of its own tile and BN/2 rows of every weight box; one thread of the first block issues
+// tcgen05.mma.cta_group::2 (M = 256), which reads both halves of the weights.  Per SM and MMA the shared
+// memory then serves 4 KB of A and BN/2 rows of B instead of BN rows, and half the weight bytes cross L2 -> SM.
+template <int BN, int OCC, int CTAS>
 __global__ void __launch_bounds__(kTcThreads, OCC)
 conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
           float* __restrict__ out, const HaloParams p) {
-  constexpr int kSubB = BN * kBK * 2;       // one tap of B
+  constexpr int kSubB = (BN / CTAS) * kBK * 2;       // one tap of B (this block's rows)
   constexpr int kTmemCols = 2 * BN < 32 ? 32 : 2 * BN;
   const uint32_t kStageB = p.b_bytes;
   extern __shared__ unsigned char smem_raw[];
@@ -1038,62 +1070,96 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   static_assert((4 * kHaloMaxStages + 4) * 8 + 8 <= kHaloBarBytes, "barrier block too small");
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // position in the pair: block 0 owns the barriers both blocks feed and issues the MMAs
+  const uint32_t rank = CTAS == 2 ? cluster_ctarank() : 0u;
   if (threadIdx.x == 32) {   // the tensor maps are kernel parameters: their fetch starts under the set-up
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_a)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_b)) : "memory");
   }
   if (threadIdx.x == 0) {
+    // full: one arrival, by the producer of block 0, which announces the bytes of the whole pair
     for (int s = 0; s < p.sa_stages; ++s) { mbar_init(bar_afull + 8 * s, 1); mbar_init(bar_aempty + 8 * s, 1); }
     for (int s = 0; s < p.sb_stages; ++s) { mbar_init(bar_bfull + 8 * s, 1); mbar_init(bar_bempty + 8 * s, 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, 4 * CTAS); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(static_cast<uint32_t>(kTmemCols))
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (CTAS == 2) {   // the same warp of both blocks allocates the same columns in both tensor memories
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"(static_cast<uint32_t>(kTmemCols))
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"(static_cast<uint32_t>(kTmemCols))
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
-  __syncthreads();
+  if (CTAS == 2) cluster_sync_all();   // the other block's barriers exist before anything signals them
+  else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   pdl_wait();
   pdl_launch_dependents();
+  // work units: p.tiles_m counts tiles of CTAS M tiles; this block takes M tile tm * CTAS + rank
   const int num_tiles = p.tiles_m * p.tiles_n;
+  const int unit0 = static_cast<int>(blockIdx.x) / CTAS, unit_step = static_cast<int>(gridDim.x) / CTAS;
 
   if (warp == 0) {
     // ---------------- A producer: one input box per (tile, 64-channel chunk) ----------------
-    if (lane == 0) {
+    // (warp-uniform loop, one elected lane issues: see dot_tc)
+    const bool leader = elect_one();
+    {
       uint32_t s = 0, ph = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x) {
+      for (int u = unit0; u < num_tiles && ok; u += unit_step) {
         uint32_t tm, tn, img, ti;
         p.div_tiles_n.divmod(static_cast<uint32_t>(u), tm, tn);
-        p.div_tpi.divmod(tm, img, ti);
+        // an M tile past the last one (odd tile count) has img >= N: its box lies outside the tensor and reads as zeros
+        p.div_tpi.divmod(tm * CTAS + rank, img, ti);
         const int h0 = static_cast<int>(ti) * p.R - p.ph;
         for (int cc = 0; cc < p.cchunks; ++cc) {
           if (!mbar_wait(bar_aempty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
-          mbar_expect_tx(bar_afull + 8 * s, p.a_bytes);
-          tma_load_4d(a_base + s * kHaloAStage, &map_a, cc * kBK, -p.pw, h0, static_cast<int>(img), bar_afull + 8 * s);
+          if (leader) {
+            if (CTAS == 2) {
+              if (rank == 0) mbar_expect_tx(bar_afull + 8 * s, 2 * p.a_bytes);
+              tma_load_4d_pair(a_base + s * kHaloAStage, &map_a, cc * kBK, -p.pw, h0, static_cast<int>(img),
+                               map_to_cta(bar_afull + 8 * s, 0));
+            } else {
+              mbar_expect_tx(bar_afull + 8 * s, p.a_bytes);
+              tma_load_4d(a_base + s * kHaloAStage, &map_a, cc * kBK, -p.pw, h0, static_cast<int>(img), bar_afull + 8 * s);
+            }
+          }
           if (++s == static_cast<uint32_t>(p.sa_stages)) { s = 0; ph ^= 1u; }
         }
       }
     }
   } else if (warp == 6) {
     // ---------------- B producer: stages in (chunk, tap group) order; once per block when resident ----------------
-    if (lane == 0) {
+    const bool leader = elect_one();
+    {
       uint32_t s = 0, ph = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x) {
-        const int n0 = static_cast<int>(static_cast<uint32_t>(u) - p.div_tiles_n.div(static_cast<uint32_t>(u)) * p.tiles_n) * BN;
+      for (int u = unit0; u < num_tiles && ok; u += unit_step) {
+        // this block's BN / CTAS rows of the column tile
+        const int n0 = static_cast<int>(static_cast<uint32_t>(u) - p.div_tiles_n.div(static_cast<uint32_t>(u)) * p.tiles_n) * BN +
+                       static_cast<int>(rank) * (BN / CTAS);
         for (int cc = 0; cc < p.cchunks && ok; ++cc) {
           for (int g = 0; g < p.groups_per_chunk; ++g) {
             if (!p.b_resident && !mbar_wait(bar_bempty + 8 * s, ph ^ 1u, abort_flag)) { ok = false; break; }
-            mbar_expect_tx(bar_bfull + 8 * s, p.b_bytes);
-            tma_load_4d(b_base + s * kStageB, &map_b, 0, n0, cc, g * p.tg, bar_bfull + 8 * s);
+            if (leader) {
+              if (CTAS == 2) {
+                if (rank == 0) mbar_expect_tx(bar_bfull + 8 * s, 2 * p.b_bytes);
+                tma_load_4d_pair(b_base + s * kStageB, &map_b, 0, n0, cc, g * p.tg, map_to_cta(bar_bfull + 8 * s, 0));
+              } else {
+                mbar_expect_tx(bar_bfull + 8 * s, p.b_bytes);
+                tma_load_4d(b_base + s * kStageB, &map_b, 0, n0, cc, g * p.tg, bar_bfull + 8 * s);
+              }
+            }
             if (++s == static_cast<uint32_t>(p.sb_stages)) { s = 0; ph ^= 1u; }
           }
         }
@@ -1104,14 +1170,15 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     // ---------------- MMA issuer ----------------
     // One thread issues everything, so the loop is kept to the bare sequence: per chunk one wait for the
     // input box, per B stage one wait, p.tg * 4 MMAs whose descriptors advance by constants, one commit.
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc(kBM, BN);
+    if (rank == 0) {
+      const bool leader = elect_one();
+      constexpr uint32_t idesc = make_idesc(kBM * CTAS, BN);
       const uint64_t desc_a0 = make_desc(a_base, 16, 1024, 2);
       const uint64_t desc_b0 = make_desc(b_base, 16, 1024, 2);
       const uint32_t row_step = static_cast<uint32_t>(p.Wb * 128) >> 4;          // next filter row
       uint32_t sa = 0, pha = 0, sb = 0, phb = 0, tile_it = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x, ++tile_it) {
+      for (int u = unit0; u < num_tiles && ok; u += unit_step, ++tile_it) {
         const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
         if (!mbar_wait(bar_tempty + 8 * acc, aph ^ 1u, abort_flag)) { ok = false; break; }
         const uint32_t d_tmem = tmem_base + acc * BN;
@@ -1129,21 +1196,31 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
             uint64_t da = da_grp, db = desc_b0 + ((sb * kStageB) >> 4);
 #pragma unroll 1
             for (int t = 0; t < p.tg; ++t, da += 8, db += (kSubB >> 4)) {
-              tc_mma_bf16(d_tmem, da, db, idesc, accumulate);
-              tc_mma_bf16(d_tmem, da + 2, db + 2, idesc, 1u);
-              tc_mma_bf16(d_tmem, da + 4, db + 4, idesc, 1u);
-              tc_mma_bf16(d_tmem, da + 6, db + 6, idesc, 1u);
+              if (leader) {
+              if (CTAS == 2) {
+                tc_mma_bf16_pair(d_tmem, da, db, idesc, accumulate);
+                tc_mma_bf16_pair(d_tmem, da + 2, db + 2, idesc, 1u);
+                tc_mma_bf16_pair(d_tmem, da + 4, db + 4, idesc, 1u);
+                tc_mma_bf16_pair(d_tmem, da + 6, db + 6, idesc, 1u);
+              } else {
+                tc_mma_bf16(d_tmem, da, db, idesc, accumulate);
+                tc_mma_bf16(d_tmem, da + 2, db + 2, idesc, 1u);
+                tc_mma_bf16(d_tmem, da + 4, db + 4, idesc, 1u);
+                tc_mma_bf16(d_tmem, da + 6, db + 6, idesc, 1u);
+              }
+              }
               accumulate = 1u;
             }
-            if (!p.b_resident) tc_commit(bar_bempty + 8 * sb);
+            if (!p.b_resident && leader) { if (CTAS == 2) tc_commit_pair(bar_bempty + 8 * sb); else tc_commit(bar_bempty + 8 * sb); }
             if (++sb == static_cast<uint32_t>(p.sb_stages)) { sb = 0; phb ^= 1u; }
             if (p.tg == p.Kw) da_grp += row_step;
             else { da_grp += 8; if (++kw == p.Kw) { kw = 0; da_grp += row_step - 8u * p.Kw; } }
           }
-          tc_commit(bar_aempty + 8 * sa);   // the box may be overwritten once these MMAs retire
+          // the box may be overwritten once these MMAs retire
+          if (leader) { if (CTAS == 2) tc_commit_pair(bar_aempty + 8 * sa); else tc_commit(bar_aempty + 8 * sa); }
           if (++sa == static_cast<uint32_t>(p.sa_stages)) { sa = 0; pha ^= 1u; }
         }
-        if (ok) tc_commit(bar_tfull + 8 * acc);
+        if (ok && leader) { if (CTAS == 2) tc_commit_pair(bar_tfull + 8 * acc); else tc_commit(bar_tfull + 8 * acc); }
       }
     }
   } else {
@@ -1153,11 +1230,12 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     bool ok = true;
     const uint32_t buf = epi_base + q * 4096;
     const int sub_row = lane >> 3, piece = lane & 7;
-    for (int u = blockIdx.x; u < num_tiles && ok; u += gridDim.x, ++tile_it) {
+    for (int u = unit0; u < num_tiles && ok; u += unit_step, ++tile_it) {
       const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
       uint32_t tm, tn, img, ti;
       p.div_tiles_n.divmod(static_cast<uint32_t>(u), tm, tn);
-      p.div_tpi.divmod(tm, img, ti);
+      p.div_tpi.divmod(tm * CTAS + rank, img, ti);
+      const bool tile_ok = static_cast<int>(img) < p.N;   // false for the filler tile of an odd tile count
       const int h0 = static_cast<int>(ti) * p.R;
       // the eight rows this lane stores (one per pass): offset of out[(img, h0 + oh, ow), 0], or -1 for a dropped row
       int64_t row_off[8];
@@ -1166,7 +1244,7 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         const uint32_t m = static_cast<uint32_t>(q * 32 + it * 4 + sub_row);
         uint32_t oh, ow;
         p.div_wb.divmod(m, oh, ow);
-        const bool valid = static_cast<int>(oh) < p.R && h0 + static_cast<int>(oh) < p.Ho && static_cast<int>(ow) < p.Wo;
+        const bool valid = tile_ok && static_cast<int>(oh) < p.R && h0 + static_cast<int>(oh) < p.Ho && static_cast<int>(ow) < p.Wo;
         row_off[it] = valid ? ((static_cast<int64_t>(img) * p.Ho + h0 + oh) * p.Wo + ow) * p.O : -1;
       }
       if (!mbar_wait(bar_tfull + 8 * acc, aph, abort_flag)) { ok = false; break; }
@@ -1221,7 +1299,10 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+      if (lane == 0) {
+        if (CTAS == 2) mbar_arrive_cluster(map_to_cta(bar_tempty + 8 * acc, 0));
+        else mbar_arrive(bar_tempty + 8 * acc);
+      }
     }
   }
 
@@ -1231,12 +1312,18 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     while (global_timer() - t0 < 20000000ull) { }
   }
   tc_fence_before();
-  __syncthreads();
+  if (CTAS == 2) cluster_sync_all();   // neither block leaves while the other may still signal it or read its tiles
+  else __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
-                 "r"(static_cast<uint32_t>(kTmemCols))
-                 : "memory");
+    if (CTAS == 2)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                   "r"(static_cast<uint32_t>(kTmemCols))
+                   : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                   "r"(static_cast<uint32_t>(kTmemCols))
+                   : "memory");
   }
 }
 
@@ -1353,7 +1440,8 @@ conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restr
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
-    if (lane == 0) {
+    {
+      const bool leader = elect_one();   // warp-uniform loop, one elected lane issues (see dot_tc)
       const uint32_t idesc = make_idesc(kBM, p.bn);
       const uint64_t desc_a0 = make_desc(a_base, 16, 128, 0);                                   // overlapping rows
       const uint64_t desc_b0 = make_desc(b_base, static_cast<uint32_t>(p.bn) * 16, 128, 0);    // [chunk][row][16 bytes]
@@ -1371,18 +1459,21 @@ conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restr
         for (int kh = 0; kh < p.Kh; ++kh, da_row += p.slot_bytes >> 4) {
           uint64_t da = da_row;
           for (int k = 0; k < p.ksteps; ++k, da += 2, db += b_step) {
-            tc_mma_bf16(d_tmem, da, db, idesc, accumulate);
+            if (leader) tc_mma_bf16(d_tmem, da, db, idesc, accumulate);
             accumulate = 1u;
           }
         }
-        tc_commit(bar_empty + 8 * s);
-        tc_commit(bar_tfull + 8 * acc);
+        if (leader) {
+          tc_commit(bar_empty + 8 * s);
+          tc_commit(bar_tfull + 8 * acc);
+        }
         if (++s == static_cast<uint32_t>(p.stages)) { s = 0; ph ^= 1u; }
       }
     }
   } else {
     // ---------------- epilogue: TMEM -> registers -> swizzled 32x32 blocks -> TMA stores ----------------
     const int q = warp & 3;
+    const bool leader = elect_one();   // issues this warp's TMA stores (always the same lane: it owns the bulk groups)
     uint32_t tile_it = 0, chunk_it = 0;
     bool ok = true;
     for (int u = blockIdx.x; u < p.tiles && ok; u += gridDim.x, ++tile_it) {
@@ -1417,7 +1508,7 @@ conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restr
           }
         }
         const uint32_t buf = epi_base + q * 8192 + (chunk_it & 1u) * 4096;
-        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the store before last has read this buffer
+        if (leader) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the store before last has read this buffer
         __syncwarp();
 #pragma unroll
         for (int j = 0; j < 8; ++j)
@@ -1426,7 +1517,7 @@ conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restr
                        : "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
-        if (lane == 0) {   // result viewed as (N*Ho, Wo, O): columns past Wo and channels past O are clipped
+        if (leader) {   // result viewed as (N*Ho, Wo, O): columns past Wo and channels past O are clipped
           asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(
                            reinterpret_cast<uint64_t>(&map_c)),
                        "r"(c), "r"(static_cast<int>(seg) * kBM + q * 32), "r"(static_cast<int>(row)), "r"(buf)
@@ -1439,7 +1530,7 @@ conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restr
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
     }
-    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   __syncwarp();
@@ -1898,6 +1989,7 @@ struct HaloPlan {
   bool ok = false;
   int bn = 64, Wb = 0, R = 0, RB = 0, tiles_per_img = 0, sa = 0, sb = 0, resident = 0, tg = 1;
   int occ = 1;   // blocks per SM the shared-memory plan is made for
+  int ctas = 1;  // 2: pairs of blocks share a column tile (each stages half of every weight box)
 };
 
 HaloPlan plan_halo(const DotProblem& d, const ConvPlan& pl, uint32_t flags) {
@@ -1919,11 +2011,23 @@ HaloPlan plan_halo(const DotProblem& d, const ConvPlan& pl, uint32_t flags) {
   hp.R = static_cast<int>(R);
   hp.RB = static_cast<int>(R + d.Kh - 1);
   hp.tiles_per_img = static_cast<int>(tpi);
+  {
+    const char* e = getenv("GL_HALO_PAIR");
+    if (e && e[0] == '1' && d.N * tpi >= 2) hp.ctas = 2;
+  }
   // a B stage holds one filter row of one 64-channel chunk when that stays within 48 KB, else one tap
   hp.tg = d.Kw * hp.bn * kBK * 2 <= 48 * 1024 ? static_cast<int>(d.Kw) : 1;
-  const int stage_b = hp.tg * hp.bn * kBK * 2;
+  const int stage_b = hp.tg * (hp.bn / hp.ctas) * kBK * 2;
   const int64_t groups = (pl.Cp / kBK) * d.Kh * (d.Kw / hp.tg);
   const int tiles_n = static_cast<int>((d.O + hp.bn - 1) / hp.bn);
+  if (hp.ctas == 2) {
+    const char* e2 = getenv("GL_HALO_SA");
+    hp.occ = 1;
+    hp.sa = e2 ? atoi(e2) : 2;
+    hp.sb = std::min<int>(kHaloMaxStages, (kHaloSmemBudget - hp.sa * kHaloAStage) / stage_b);
+    hp.ok = hp.sb >= 2;
+    return hp;
+  }
   if (hp.bn == 64) {
     // N = 64 MMAs are bound by their issue floor; two blocks per SM with one input-box stage each hide
     // start-up, loads and epilogue of one block under the MMAs of the other
@@ -1963,7 +2067,7 @@ bool encode_halo_box(CUtensorMap* m, const void* base, const DotProblem& d, int6
 
 // Weights (O, Kh, Kw, Cp) viewed as (64 channels, O, chunk, tap): one box = BN rows x 64 channels of
 // `tg` consecutive taps of one chunk, landing as [tap][row][64].
-bool encode_halo_weights(CUtensorMap* m, const void* base, int64_t O, int64_t taps, int64_t Cp, int bn, int tg) {
+bool encode_halo_weights(CUtensorMap* m, const void* base, int64_t O, int64_t taps, int64_t Cp, int bn, int tg) {   // bn: rows per box
   const cuuint64_t dims[4] = {kBK, static_cast<cuuint64_t>(O), static_cast<cuuint64_t>(Cp / kBK),
                               static_cast<cuuint64_t>(taps)};
   const cuuint64_t strides[3] = {static_cast<cuuint64_t>(taps * Cp) * 2, kBK * 2, static_cast<cuuint64_t>(Cp) * 2};
@@ -1974,21 +2078,47 @@ bool encode_halo_weights(CUtensorMap* m, const void* base, int64_t O, int64_t ta
                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int OCC>
+template <int BN, int OCC, int CTAS>
 int launch_halo(const CUtensorMap& ma, const CUtensorMap& mb, float* out, const HaloParams& p, cudaStream_t st) {
   const int smem = p.sa_stages * kHaloAStage + p.sb_stages * static_cast<int>(p.b_bytes) + kHaloEpiBytes + kHaloBarBytes + 1024;
   static bool attr_set_dev[64] = {false};
+  static int max_pairs_dev[64] = {0};       // CTAS == 2: pairs that can be resident at once
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return GL_ERR_CUDA;
   if (!attr_set_dev[dev]) {
-    if (cudaFuncSetAttribute(conv_halo<BN, OCC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (cudaFuncSetAttribute(conv_halo<BN, OCC, CTAS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              OCC == 2 ? 113 * 1024 : 232448) != cudaSuccess)
       return GL_ERR_CUDA;
+    if (CTAS == 2) {
+      // a persistent grid must not exceed what is resident at once (SMs pair up within a GPC)
+      cudaLaunchConfig_t cfg;
+      std::memset(&cfg, 0, sizeof(cfg));
+      cudaLaunchAttribute cluster_attr;
+      std::memset(&cluster_attr, 0, sizeof(cluster_attr));
+      cluster_attr.id = cudaLaunchAttributeClusterDimension;
+      cluster_attr.val.clusterDim.x = 2;
+      cluster_attr.val.clusterDim.y = 1;
+      cluster_attr.val.clusterDim.z = 1;
+      cfg.gridDim = dim3(static_cast<unsigned>(OCC * (num_sms() / 2 * 2)));
+      cfg.blockDim = dim3(kTcThreads);
+      cfg.dynamicSmemBytes = OCC == 2 ? 113 * 1024 : 232448;
+      cfg.attrs = &cluster_attr;
+      cfg.numAttrs = 1;
+      int pairs = 0;
+      if (cudaOccupancyMaxActiveClusters(&pairs, conv_halo<BN, OCC, CTAS>, &cfg) != cudaSuccess || pairs < 1)
+        return GL_ERR_CUDA;
+      max_pairs_dev[dev] = pairs;
+    }
     attr_set_dev[dev] = true;
   }
   const int tiles = p.tiles_m * p.tiles_n;
+  if (CTAS == 2) {
+    const int pairs = std::min(tiles, std::min(max_pairs_dev[dev], OCC * (num_sms() / 2)));
+    return launch_pdl(conv_halo<BN, OCC, CTAS>, dim3(static_cast<unsigned>(2 * pairs)), dim3(kTcThreads),
+                      static_cast<size_t>(smem), st, 2, ma, mb, out, p) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+  }
   const int grid = std::min(tiles, OCC * num_sms());
-  return launch_pdl(conv_halo<BN, OCC>, dim3(static_cast<unsigned>(grid)), dim3(kTcThreads), static_cast<size_t>(smem), st, 1,
+  return launch_pdl(conv_halo<BN, OCC, CTAS>, dim3(static_cast<unsigned>(grid)), dim3(kTcThreads), static_cast<size_t>(smem), st, 1,
                     ma, mb, out, p) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
 }
 
@@ -1997,9 +2127,10 @@ int run_halo(const HaloPlan& hp, const DotProblem& d, int64_t Cp, const uint16_t
   HaloParams p;
   std::memset(&p, 0, sizeof(p));
   p.O = d.O; p.relu = relu; p.out_bf16 = out_bf16;
+  p.N = static_cast<int>(d.N);
   p.Ho = static_cast<int>(d.Ho); p.Wo = static_cast<int>(d.Wo);
   p.Wb = hp.Wb; p.R = hp.R;
-  p.tiles_m = static_cast<int>(d.N) * hp.tiles_per_img;
+  p.tiles_m = (static_cast<int>(d.N) * hp.tiles_per_img + hp.ctas - 1) / hp.ctas;
   p.tiles_n = static_cast<int>((d.O + hp.bn - 1) / hp.bn);
   p.Kh = static_cast<int>(d.Kh); p.Kw = static_cast<int>(d.Kw);
   p.Cp = static_cast<int>(Cp);
@@ -2009,15 +2140,17 @@ int run_halo(const HaloPlan& hp, const DotProblem& d, int64_t Cp, const uint16_t
   p.ph = static_cast<int>(d.ph_lo); p.pw = static_cast<int>(d.pw_lo);
   p.sa_stages = hp.sa; p.sb_stages = hp.sb; p.b_resident = hp.resident;
   p.a_bytes = static_cast<uint32_t>(kBK * 2 * hp.Wb * hp.RB);
-  p.b_bytes = static_cast<uint32_t>(hp.tg * hp.bn * kBK * 2);
+  p.b_bytes = static_cast<uint32_t>(hp.tg * (hp.bn / hp.ctas) * kBK * 2);
   p.div_tiles_n.set(p.tiles_n);
   p.div_tpi.set(hp.tiles_per_img);
   p.div_wb.set(hp.Wb);
   CUtensorMap ma, mb;
   if (!encode_halo_box(&ma, x, d, Cp, hp.Wb, hp.RB) ||
-      !encode_halo_weights(&mb, wt, d.O, d.Kh * d.Kw, Cp, hp.bn, hp.tg))
+      !encode_halo_weights(&mb, wt, d.O, d.Kh * d.Kw, Cp, hp.bn / hp.ctas, hp.tg))
     return GL_ERR_CUDA;
-  return hp.bn == 128 ? launch_halo<128, 1>(ma, mb, out, p, st) : launch_halo<64, 2>(ma, mb, out, p, st);
+  if (hp.ctas == 2)
+    return hp.bn == 128 ? launch_halo<128, 1, 2>(ma, mb, out, p, st) : launch_halo<64, 1, 2>(ma, mb, out, p, st);
+  return hp.bn == 128 ? launch_halo<128, 1, 1>(ma, mb, out, p, st) : launch_halo<64, 2, 1>(ma, mb, out, p, st);
 }
 
 // A 1x1, stride-1, unpadded window over channels-last items is no window at all: the activations
