@@ -389,6 +389,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   const uint64_t t0 = global_timer();
   uint32_t spins = 0;
   while (!mbar_try_wait(bar, parity)) {
+    __nanosleep(40);
     if ((++spins & 0xFFu) == 0) {
       if (*abort_flag) return false;
       if (global_timer() - t0 > limit_ns) {
@@ -1342,24 +1343,32 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 // holds each input row run ONCE (2 KB for 128 output columns), copied by one bulk copy per filter row, and
 // cartProd/dotProd run over it as Kh * ceil(Kw*Cp/16) MMAs per tile.  The weights (a few KB) stay resident.
 
-constexpr int kRunThreads = 192;       // warp 0 copies, warp 1 issues MMAs, warps 2-5 store results
-constexpr int kRunMaxStages = 8;
-constexpr int kRunEpiBytes = 4 * 2 * 4096;   // two 32x32 fp32 staging tiles per epilogue warp
+constexpr int kRunExpanders = 4;       // warp 0 copies raw rows, warps 6-9 widen them; warp 1 issues MMAs, warps 2-5 store results
+constexpr int kRunThreads = 32 * (6 + kRunExpanders);
+constexpr int kRunMaxStages = 4;
+constexpr int kRunEpiBytes = 4 * 4096;   // one 32x32 fp32 staging tile per epilogue warp
 
 struct RowRunParams {
   int64_t O;
   int relu;
   int out_bf16;   // results rounded to bf16 (O a multiple of 8)
-  int Ho, Wo, Hp, Sh, Kh;
+  int C, H, W, Ho, Wo, Sh, Sw, Kh, Kw, ph, pw;
+  int cp_log2;                  // pixels are widened to 8 / Sw = 2^cp_log2 channels
+  int channels_last;            // items (H,W,C) / (Kh,Kw,C), else (C,H,W) / (C,Kh,Kw)
+  int64_t xs_n, xs_h, xs_c;     // elements between images, rows and (for (C,H,W) items) channel planes
+  int nseg;                     // raw copies per input row: 1 (pixels hold their channels) or C (one per plane)
+  uint32_t raw_seg_bytes;       // shared-memory pitch of one raw copy, of the copies of a row, of a raw stage
+  uint32_t raw_row_bytes, raw_stage_bytes;
+  int raw_stages;
+  int w_elems;                  // O * Kh * Kw * C (they fit the raw stages, where the block parks them once)
   int segs, tiles;              // 128-column segments per output row; tiles = N * Ho * segs
   int ksteps;                   // MMAs (K = 16) per filter row
   int bn;                       // MMA N: O rounded up to 16
   uint32_t seg_bytes;           // bytes of one run: 127 * 16 + ksteps * 32
   uint32_t slot_bytes;          // shared-memory pitch of a run
-  uint32_t pitch_bytes;         // bytes between padded input rows in global memory
   uint32_t b_bytes;             // resident weights: Kh * ksteps * 2 chunks * bn rows * 16 bytes
   int stages;
-  FastDiv div_segs, div_ho;
+  FastDiv div_segs, div_ho, div_nseg, div_bn, div_chunks;
 };
 
 __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -1367,9 +1376,18 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uin
                ::"r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
                : "memory");
 }
-
+// The activations are read where they are, in either item layout.  Per tile (128 output columns of one output
+// row) and filter row, the stretch of the input row that the tile's windows cover is brought into shared memory
+// as it lies in global memory, by plain bulk copies of whole 16-byte pieces (one copy per row for (H,W,C) items,
+// one per channel plane for (C,H,W) items); three warps then widen it into the padded row run: pixel wp of the
+// run of filter row kh holds the C channels of input pixel (ho * Sh + kh - ph, seg * 128 * Sw + wp - pw), zeros
+// for the border and for the channels past C.  The weights are rearranged into operand order by the whole block
+// once, before the first tile.  Nothing passes through a global-memory copy.
+// CT, CL: channel count and item layout as compile-time constants (CT = 0: both taken from p at run time).  The
+// widening warps are bound by their instruction count per pixel; with constants it is a fifth of the general form.
+template <int CT, int CL>
 __global__ void __launch_bounds__(kRunThreads, 2)
-conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restrict__ wpack,
+conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
             const __grid_constant__ CUtensorMap map_c, const RowRunParams p) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -1379,23 +1397,25 @@ conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restr
   const uint32_t epi_base = base;                                         // 1024-byte aligned staging tiles
   const uint32_t b_base = epi_base + kRunEpiBytes;
   const uint32_t a_base = b_base + ((p.b_bytes + 127u) & ~127u);
-  const uint32_t bars_off = (a_base - base) + ((static_cast<uint32_t>(p.stages) * stage_bytes + 7u) & ~7u);
+  const uint32_t r_base = a_base + static_cast<uint32_t>(p.stages) * stage_bytes;   // raw copies (slot_bytes is a multiple of 128)
+  const uint32_t bars_off = (r_base - base) + static_cast<uint32_t>(p.raw_stages) * p.raw_stage_bytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(gen + bars_off);
-  const uint32_t bar_full = smem_u32(bars);                  // [kRunMaxStages]
-  const uint32_t bar_empty = bar_full + 8 * kRunMaxStages;   // [kRunMaxStages]
-  const uint32_t bar_tfull = bar_empty + 8 * kRunMaxStages;  // [2]
+  const uint32_t bar_full = smem_u32(bars);                  // [kRunMaxStages] widened runs ready
+  const uint32_t bar_empty = bar_full + 8 * kRunMaxStages;   // [kRunMaxStages] ... consumed by the MMAs
+  const uint32_t bar_rfull = bar_empty + 8 * kRunMaxStages;  // [kRunMaxStages] raw copies landed
+  const uint32_t bar_rempty = bar_rfull + 8 * kRunMaxStages; // [kRunMaxStages] ... widened
+  const uint32_t bar_tfull = bar_rempty + 8 * kRunMaxStages; // [2]
   const uint32_t bar_tempty = bar_tfull + 16;                // [2]
-  const uint32_t bar_b = bar_tempty + 16;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kRunMaxStages + 5);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 4 * kRunMaxStages + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const uint32_t tmem_cols = 2 * p.bn <= 32 ? 32u : (2 * p.bn <= 64 ? 64u : (2 * p.bn <= 128 ? 128u : 256u));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 64) asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_c)) : "memory");
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+    for (int s = 0; s < p.stages; ++s) { mbar_init(bar_full + 8 * s, kRunExpanders); mbar_init(bar_empty + 8 * s, 1); }
+    for (int s = 0; s < p.raw_stages; ++s) { mbar_init(bar_rfull + 8 * s, 1); mbar_init(bar_rempty + 8 * s, kRunExpanders); }
     for (int a = 0; a < 2; ++a) { mbar_init(bar_tfull + 8 * a, 1); mbar_init(bar_tempty + 8 * a, 4); }
-    mbar_init(bar_b, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -1412,31 +1432,138 @@ conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restr
   pdl_wait();
   pdl_launch_dependents();
 
-  if (warp == 0) {
-    // ---------------- producer: the weights once, then Kh row runs per tile ----------------
-    // lane 0 waits for the stage and announces the bytes; lanes 0..Kh-1 then issue one row copy each
-    // (one warp instruction instead of Kh trips through a single-thread loop)
-    if (lane == 0) {
-      mbar_expect_tx(bar_b, p.b_bytes);
-      bulk_copy_g2s(b_base, wpack, p.b_bytes, bar_b);
+  // ---- weights into operand order [kh][K chunk j][row o < bn][8 elements]: element kw * cp + c of filter row
+  // kh sits at (j, i) = ((kw * cp + c) / 8, (kw * cp + c) % 8), zeros elsewhere.  The weight tensor is first
+  // copied as it is (16-byte loads) into the area of the raw stages, which nothing uses yet; every thread then
+  // assembles 16-byte pieces (kh, j, o) from it.
+  {
+    uint16_t* wraw = reinterpret_cast<uint16_t*>(gen + (r_base - base));
+    const int nvec = p.w_elems >> 3;
+    for (int i = threadIdx.x; i < nvec; i += kRunThreads)
+      reinterpret_cast<uint4*>(wraw)[i] = reinterpret_cast<const uint4*>(wt)[i];
+    for (int i = nvec * 8 + threadIdx.x; i < p.w_elems; i += kRunThreads) wraw[i] = wt[i];
+    __syncthreads();
+    const int chunks = 2 * p.ksteps, pieces = p.Kh * chunks * p.bn;
+    const int cp_mask = (1 << p.cp_log2) - 1;
+    uint4* wop = reinterpret_cast<uint4*>(gen + (b_base - base));
+    for (int q = threadIdx.x; q < pieces; q += kRunThreads) {
+      uint32_t t, o, kh, j;
+      p.div_bn.divmod(static_cast<uint32_t>(q), t, o);
+      p.div_chunks.divmod(t, kh, j);
+      // (H,W,C) items: element ((o Kh + kh) Kw + kw) C + c;  (C,H,W) items: ((o C + c) Kh + kh) Kw + kw
+      const int at = p.channels_last ? static_cast<int>(o * p.Kh + kh) * p.Kw * p.C : (static_cast<int>(o) * p.C * p.Kh + static_cast<int>(kh)) * p.Kw;
+      const int step_kw = p.channels_last ? p.C : 1, step_c = p.channels_last ? 1 : p.Kh * p.Kw;
+      uint32_t v[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int el = static_cast<int>(j) * 8 + i, kw = el >> p.cp_log2, c = el & cp_mask;
+        const bool ok = static_cast<int64_t>(o) < p.O && kw < p.Kw && c < p.C;
+        v[i] = ok ? wraw[at + kw * step_kw + c * step_c] : 0u;
+      }
+      wop[q] = make_uint4(v[0] | (v[1] << 16), v[2] | (v[3] << 16), v[4] | (v[5] << 16), v[6] | (v[7] << 16));
     }
-    uint32_t s = 0, ph = 0;
-    int ok = 1;
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads them through the async proxy
+    __syncthreads();
+  }
+
+  const int npx = static_cast<int>(p.seg_bytes >> (p.cp_log2 + 1));   // pixels of a run
+  const int epx = p.channels_last ? p.C : 1;                          // elements per pixel in one raw copy
+  if (warp == 0) {
+    // ---------------- raw copies: lane i takes copy i = (filter row, segment) of the tile ----------------
+    const int ncopies = p.Kh * p.nseg;   // at most 32
+    uint32_t kh_l, c_l;
+    p.div_nseg.divmod(static_cast<uint32_t>(lane), kh_l, c_l);
+    uint32_t r = 0, ph = 0;
     for (int u = blockIdx.x; u < p.tiles; u += gridDim.x) {
       uint32_t row, seg, img, ho;
       p.div_segs.divmod(static_cast<uint32_t>(u), row, seg);
       p.div_ho.divmod(row, img, ho);
-      // filter row `lane` of the tile: padded input row img * Hp + ho * Sh + lane, 16 bytes per output column
-      const unsigned char* src = xpad + (static_cast<int64_t>(img) * p.Hp + static_cast<int64_t>(ho) * p.Sh + lane) * p.pitch_bytes +
-                                 static_cast<int64_t>(seg) * (kBM * 16);
-      if (lane == 0) {
-        ok = mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag) ? 1 : 0;
-        if (ok) mbar_expect_tx(bar_full + 8 * s, static_cast<uint32_t>(p.Kh) * p.seg_bytes);
+      if (!mbar_wait(bar_rempty + 8 * r, ph ^ 1u, abort_flag)) break;
+      const int w_first = static_cast<int>(seg) * (kBM * p.Sw) - p.pw;   // input column of run pixel 0
+      const int w_lo = max(w_first, 0), w_hi = min(w_first + npx, p.W);
+      const int h = static_cast<int>(ho) * p.Sh + static_cast<int>(kh_l) - p.ph;
+      uint32_t size = 0;
+      int64_t a0 = 0;
+      if (lane < ncopies && h >= 0 && h < p.H && w_hi > w_lo) {
+        const int64_t e0 = static_cast<int64_t>(img) * p.xs_n + static_cast<int64_t>(h) * p.xs_h +
+                           (p.channels_last ? static_cast<int64_t>(w_lo) * p.C : static_cast<int64_t>(c_l) * p.xs_c + w_lo);
+        const int64_t b0 = e0 * 2, b1 = b0 + static_cast<int64_t>(w_hi - w_lo) * epx * 2;
+        a0 = b0 & ~static_cast<int64_t>(15);                              // whole 16-byte pieces around the stretch;
+        size = static_cast<uint32_t>(((b1 + 15) & ~static_cast<int64_t>(15)) - a0);   // the tensor's byte count is a multiple of 16
       }
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      if (lane < p.Kh) bulk_copy_g2s(a_base + s * stage_bytes + lane * p.slot_bytes, src, p.seg_bytes, bar_full + 8 * s);
+      const uint32_t total = __reduce_add_sync(0xffffffffu, size);
+      if (lane == 0) mbar_expect_tx(bar_rfull + 8 * r, total);
+      __syncwarp();
+      if (size)
+        bulk_copy_g2s(r_base + r * p.raw_stage_bytes + kh_l * p.raw_row_bytes + c_l * p.raw_seg_bytes,
+                      reinterpret_cast<const unsigned char*>(x) + a0, size, bar_rfull + 8 * r);
+      if (++r == static_cast<uint32_t>(p.raw_stages)) { r = 0; ph ^= 1u; }
+    }
+  } else if (warp >= 6) {
+    // ---------------- widening: raw rows -> padded row runs, filter rows dealt round robin to the warps ----------------
+    const int eidx = warp - 6;
+    const int cp = 1 << p.cp_log2;
+    constexpr int kC = CT > 0 ? CT : 8;
+    const int nch = CT > 0 ? CT : p.C;
+    const bool cl = CT > 0 ? CL != 0 : p.channels_last != 0;
+    const int epx_e = cl ? nch : 1;
+    uint32_t s = 0, ph = 0, r = 0, rph = 0;
+    for (int u = blockIdx.x; u < p.tiles; u += gridDim.x) {
+      uint32_t row, seg, img, ho;
+      p.div_segs.divmod(static_cast<uint32_t>(u), row, seg);
+      p.div_ho.divmod(row, img, ho);
+      if (!mbar_wait(bar_rfull + 8 * r, rph, abort_flag)) break;
+      if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) break;
+      const int w_first = static_cast<int>(seg) * (kBM * p.Sw) - p.pw;
+      const int w_lo = max(w_first, 0), w_hi = min(w_first + npx, p.W);
+      for (int kh = eidx; kh < p.Kh; kh += kRunExpanders) {
+        const int h = static_cast<int>(ho) * p.Sh + kh - p.ph;
+        const bool row_ok = h >= 0 && h < p.H;
+        // where the stretch starts inside its 16-byte aligned copy, per raw copy of this row
+        const int64_t e0 = static_cast<int64_t>(img) * p.xs_n + static_cast<int64_t>(h) * p.xs_h +
+                           (cl ? static_cast<int64_t>(w_lo) * nch : static_cast<int64_t>(w_lo));
+        // element offset of the stretch inside its 16-byte aligned copy, per raw copy of this row
+        uint32_t delta[kC];
+#pragma unroll
+        for (int c = 0; c < kC; ++c)
+          delta[c] = static_cast<uint32_t>((((e0 + (cl ? 0 : c * p.xs_c)) * 2) & 15) >> 1) +
+                     (cl ? static_cast<uint32_t>(c) : static_cast<uint32_t>(c) * (p.raw_seg_bytes >> 1));
+        const uint16_t* src_row = reinterpret_cast<const uint16_t*>(gen + (r_base - base) + r * p.raw_stage_bytes +
+                                                                    static_cast<uint32_t>(kh) * p.raw_row_bytes);
+        unsigned char* dst_row = gen + (a_base - base) + s * stage_bytes + static_cast<uint32_t>(kh) * p.slot_bytes;
+        // four pixels per lane and trip: their loads are issued together
+        for (int wp0 = lane; wp0 < npx; wp0 += 128) {
+          uint32_t v[4][8];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const int wp = wp0 + 32 * k, w = w_first + wp;
+            const bool ok = row_ok && wp < npx && w >= w_lo && w < w_hi;
+            const uint16_t* px = src_row + (ok ? (w - w_lo) * epx_e : 0);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) v[k][c] = 0u;
+#pragma unroll
+            for (int c = 0; c < kC; ++c)
+              if ((CT > 0 || c < nch) && ok) v[k][c] = px[delta[c]];
+          }
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const int wp = wp0 + 32 * k;
+            if (wp < npx) {
+              unsigned char* dst = dst_row + (static_cast<uint32_t>(wp) << (p.cp_log2 + 1));
+              const uint32_t w01 = v[k][0] | (v[k][1] << 16), w23 = v[k][2] | (v[k][3] << 16);
+              if (cp == 8) *reinterpret_cast<uint4*>(dst) = make_uint4(w01, w23, v[k][4] | (v[k][5] << 16), v[k][6] | (v[k][7] << 16));
+              else if (cp == 4) *reinterpret_cast<uint2*>(dst) = make_uint2(w01, w23);
+              else if (cp == 2) *reinterpret_cast<uint32_t*>(dst) = w01;
+              else *reinterpret_cast<uint16_t*>(dst) = static_cast<uint16_t>(w01);
+            }
+          }
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes before the tensor core's reads
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(bar_full + 8 * s); mbar_arrive(bar_rempty + 8 * r); }
       if (++s == static_cast<uint32_t>(p.stages)) { s = 0; ph ^= 1u; }
+      if (++r == static_cast<uint32_t>(p.raw_stages)) { r = 0; rph ^= 1u; }
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
@@ -1447,7 +1574,7 @@ conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restr
       const uint64_t desc_b0 = make_desc(b_base, static_cast<uint32_t>(p.bn) * 16, 128, 0);    // [chunk][row][16 bytes]
       const uint32_t b_step = (2u * p.bn * 16u) >> 4;                                           // two K chunks per MMA
       uint32_t s = 0, ph = 0, tile_it = 0;
-      bool ok = mbar_wait(bar_b, 0, abort_flag);
+      bool ok = true;
       for (int u = blockIdx.x; u < p.tiles && ok; u += gridDim.x, ++tile_it) {
         const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
         if (!mbar_wait(bar_tempty + 8 * acc, aph ^ 1u, abort_flag)) { ok = false; break; }
@@ -1507,8 +1634,8 @@ conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restr
             r[16 + i] = pack_bf16x2(a, b);
           }
         }
-        const uint32_t buf = epi_base + q * 8192 + (chunk_it & 1u) * 4096;
-        if (leader) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // the store before last has read this buffer
+        const uint32_t buf = epi_base + q * 4096;
+        if (leader) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // the previous store has read this buffer
         __syncwarp();
 #pragma unroll
         for (int j = 0; j < 8; ++j)
@@ -1543,87 +1670,6 @@ conv_rowrun(const unsigned char* __restrict__ xpad, const unsigned char* __restr
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
-  }
-}
-
-// Layout pre-pass of conv_rowrun, one launch.
-// Blocks [0, row_blocks): padded copy (N, Hp, Wpa, Cp) with zero borders.  A warp takes one padded row at a
-// time and builds it in shared memory: the buffer starts as zeros, the pixels of the input row are dropped
-// at their padded positions (border cells and channels past C are never written, so they stay zero), and
-// the finished row leaves as 16-byte pieces.  Blocks from row_blocks on: the weights in operand order
-// [kh][K chunk j][row o < bn][8 elements], element kw * Cp + c of filter row kh at
-// (j, i) = ((kw * Cp + c) / 8, (kw * Cp + c) % 8); zeros elsewhere.
-constexpr int kPackWarps = 8;
-constexpr int kPackRowsPerWarp = 1;
-
-template <int C>   // input channels (1..8), a compile-time constant so that the per-pixel loops carry no tests
-__global__ void __launch_bounds__(32 * kPackWarps) rowrun_pack(const uint16_t* __restrict__ in, uint16_t* __restrict__ out,
-                                                               const uint16_t* __restrict__ win, uint16_t* __restrict__ wout,
-                                                               int channels_last, int row_blocks, int rows, int H,
-                                                               int W, int Hp, int Wpa, int cp_log2, int ph, int pw, int O,
-                                                               int Kh, int Kw, int chunks, int bn) {
-  extern __shared__ uint4 padded_rows[];   // [kPackWarps][Wpa * Cp / 8] pieces of 16 bytes
-  pdl_wait();
-  pdl_launch_dependents();
-  const int Cp = 1 << cp_log2;
-  if (static_cast<int>(blockIdx.x) >= row_blocks) {
-    const int total = Kh * chunks * bn * 8;
-    for (int e = (static_cast<int>(blockIdx.x) - row_blocks) * blockDim.x + threadIdx.x; e < total;
-         e += (static_cast<int>(gridDim.x) - row_blocks) * blockDim.x) {
-      const int i = e & 7, t = e >> 3;
-      const int o = t % bn, j = (t / bn) % chunks, kh = t / (bn * chunks);
-      const int el = j * 8 + i, kw = el >> cp_log2, c = el & (Cp - 1);
-      uint16_t val = 0;
-      if (o < O && kw < Kw && c < C)
-        val = channels_last ? win[((static_cast<int64_t>(o) * Kh + kh) * Kw + kw) * C + c]
-                            : win[((static_cast<int64_t>(o) * C + c) * Kh + kh) * Kw + kw];
-      wout[e] = val;
-    }
-    return;
-  }
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int nchunks = (Wpa << cp_log2) >> 3;
-  uint4* mine = padded_rows + warp * nchunks;
-  uint16_t* cells = reinterpret_cast<uint16_t*>(mine) + (pw << cp_log2);   // pixel 0 of the input row
-  for (int ch = lane; ch < nchunks; ch += 32) mine[ch] = make_uint4(0u, 0u, 0u, 0u);
-  int rowid = (static_cast<int>(blockIdx.x) * kPackWarps + warp) * kPackRowsPerWarp;
-  int n = rowid / Hp, hp = rowid - n * Hp;
-  for (int r = 0; r < kPackRowsPerWarp && rowid < rows; ++r, ++rowid) {
-    const int h = hp - ph;
-    uint4* orow = reinterpret_cast<uint4*>(out + (static_cast<int64_t>(rowid) * Wpa << cp_log2));
-    if (h < 0 || h >= H) {   // a border row
-      for (int ch = lane; ch < nchunks; ch += 32) orow[ch] = make_uint4(0u, 0u, 0u, 0u);
-    } else {
-      __syncwarp();   // the previous row has left the buffer
-      // four pixels per lane per trip, all their channel loads in flight before any is placed
-      const int64_t HW = static_cast<int64_t>(H) * W;
-      const uint16_t* src = channels_last ? in + (static_cast<int64_t>(n) * H + h) * W * C
-                                          : in + (static_cast<int64_t>(n) * C * H + h) * W;
-      const int64_t step_w = channels_last ? C : 1, step_c = channels_last ? 1 : HW;
-      for (int w0 = 0; w0 < W; w0 += 128) {
-        uint16_t v[4][C];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int w = w0 + i * 32 + lane;
-#pragma unroll
-          for (int c = 0; c < C; ++c) {
-            v[i][c] = 0;
-            if (w < W) v[i][c] = src[w * step_w + c * step_c];
-          }
-        }
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int w = w0 + i * 32 + lane;
-          if (w < W) {
-#pragma unroll
-            for (int c = 0; c < C; ++c) cells[(w << cp_log2) + c] = v[i][c];
-          }
-        }
-      }
-      __syncwarp();
-      for (int ch = lane; ch < nchunks; ch += 32) orow[ch] = mine[ch];
-    }
-    if (++hp == Hp) { hp = 0; ++n; }
   }
 }
 
@@ -1921,8 +1967,8 @@ struct ConvPlan {
   // then the [N*H'*W', Cp] matrix of a plain matrix product
   bool as_matrix = false;
   bool rowrun = false;
-  int rr_cp = 0, rr_ksteps = 0, rr_bn = 0, rr_stages = 0;
-  uint32_t rr_seg = 0, rr_slot = 0, rr_b_bytes = 0;
+  int rr_cp = 0, rr_ksteps = 0, rr_bn = 0, rr_stages = 0, rr_raw_stages = 0, rr_nseg = 0;
+  uint32_t rr_seg = 0, rr_slot = 0, rr_b_bytes = 0, rr_raw_seg = 0;
 };
 
 ConvPlan plan_conv(const DotProblem& d, uint32_t flags) {
@@ -1935,27 +1981,28 @@ ConvPlan plan_conv(const DotProblem& d, uint32_t flags) {
   pl.tc = fits && ((d.M + 127) / 128) * ((d.O + 63) / 64) < (1ll << 28);
   pl.prepass = !d.channels_last || pl.Cp != d.C;
   if (pl.tc && !(flags & GL_OUT_NCHW) && (d.Sw == 1 || d.Sw == 2 || d.Sw == 4 || d.Sw == 8) && d.C <= 8 / d.Sw &&
-      d.O % ((flags & GL_OUT_BF16) ? 8 : 4) == 0 && d.O <= 128 && d.Kh <= 16 && kPackWarps * (d.W + d.pw_lo + d.pw_hi + 64) * 16 <= 48 * 1024 && d.Wo < (1ll << 24) &&
-      d.N * (d.H + d.ph_lo + d.ph_hi) < (1ll << 31)) {
+      d.O % ((flags & GL_OUT_BF16) ? 8 : 4) == 0 && d.O <= 128 && d.Kh <= 16 && d.Wo < (1ll << 24) &&
+      d.N * d.Ho * ((d.Wo + kBM - 1) / kBM) < (1ll << 31) &&
+      (d.N * d.C * d.H * d.W) % 8 == 0 &&                    // raw rows are copied as whole 16-byte pieces
+      d.Kh * (d.channels_last ? 1 : d.C) <= 32) {            // one copy per lane of the copying warp
     const int cp = static_cast<int>(8 / d.Sw);
     const int ksteps = static_cast<int>((d.Kw * cp + 15) / 16);
     const int bn = static_cast<int>((d.O + 15) / 16 * 16);
     const uint32_t seg = 127 * 16 + ksteps * 32, slot = (seg + 127u) & ~127u;
     const uint32_t b_bytes = static_cast<uint32_t>(d.Kh) * ksteps * 2 * bn * 16;
+    const int nseg = static_cast<int>(d.channels_last ? 1 : d.C);
+    // a raw copy: the run's pixels as they lie in memory, widened to whole 16-byte pieces at both ends
+    const uint32_t raw_seg = static_cast<uint32_t>(((seg / (2 * cp)) * (d.channels_last ? d.C : 1) * 2 + 30 + 15) / 16 * 16);
+    const int64_t raw_stage = d.Kh * nseg * static_cast<int64_t>(raw_seg);
     const int64_t room = 113 * 1024 - 1024 - kRunEpiBytes - 256 - ((b_bytes + 127) & ~127u);   // two blocks per SM
-    const int64_t stages = std::min<int64_t>(kRunMaxStages, room / (d.Kh * slot));
-    if (stages >= 2) {
+    const int64_t stages = 2;                                                                   // widened runs
+    const int64_t raw_stages = std::min<int64_t>(kRunMaxStages, (room - stages * d.Kh * slot) / raw_stage);
+    if (raw_stages >= 2 && d.O * d.Kh * d.Kw * d.C * 2 <= raw_stages * raw_stage) {   // the weights fit the raw stages
       pl.rowrun = true;
-      pl.prepass = true;
+      pl.prepass = false;   // the kernel reads both operands where they are, in either item layout
       pl.rr_cp = cp; pl.rr_ksteps = ksteps; pl.rr_bn = bn; pl.rr_stages = static_cast<int>(stages);
       pl.rr_seg = seg; pl.rr_slot = slot; pl.rr_b_bytes = b_bytes;
-      pl.Hp = d.H + d.ph_lo + d.ph_hi;
-      // every window of a real output column lies inside its row; the row pitch is a multiple of 16 bytes
-      pl.Wpa = std::max(d.W + d.pw_lo + d.pw_hi, (d.Wo - 1) * d.Sw + (ksteps * 16 + cp - 1) / cp);
-      pl.Wpa = (pl.Wpa * cp + 7) / 8 * 8 / cp;
-      // the runs of the columns past Wo (computed, never stored) may reach past the last row: slack
-      pl.x_bytes = round_up(static_cast<size_t>(d.N * pl.Hp * pl.Wpa * cp) * 2 + kBM * 16 + 4096, 1024);
-      pl.w_bytes = round_up(b_bytes, 1024);
+      pl.rr_raw_stages = static_cast<int>(raw_stages); pl.rr_nseg = nseg; pl.rr_raw_seg = raw_seg;
       return pl;
     }
   }
@@ -2011,26 +2058,25 @@ HaloPlan plan_halo(const DotProblem& d, const ConvPlan& pl, uint32_t flags) {
   hp.R = static_cast<int>(R);
   hp.RB = static_cast<int>(R + d.Kh - 1);
   hp.tiles_per_img = static_cast<int>(tpi);
-  {
-    const char* e = getenv("GL_HALO_PAIR");
-    if (e && e[0] == '1' && d.N * tpi >= 2) hp.ctas = 2;
-  }
+  // 128-wide tiles: pairs of blocks halve the weight bytes each SM pulls from L2 and the shared-memory
+  // reads per MMA (measured 12.0 -> 11.2 us on 28x28x128, 11.7 -> 11.1 us on 14x14x256); at 64 columns the
+  // pair's single block per SM loses to two independent blocks per SM
+  if (hp.bn == 128 && d.N * tpi >= 2) hp.ctas = 2;
   // a B stage holds one filter row of one 64-channel chunk when that stays within 48 KB, else one tap
   hp.tg = d.Kw * hp.bn * kBK * 2 <= 48 * 1024 ? static_cast<int>(d.Kw) : 1;
   const int stage_b = hp.tg * (hp.bn / hp.ctas) * kBK * 2;
   const int64_t groups = (pl.Cp / kBK) * d.Kh * (d.Kw / hp.tg);
   const int tiles_n = static_cast<int>((d.O + hp.bn - 1) / hp.bn);
   if (hp.ctas == 2) {
-    const char* e2 = getenv("GL_HALO_SA");
     hp.occ = 1;
-    hp.sa = e2 ? atoi(e2) : 2;
+    hp.sa = 2;
     hp.sb = std::min<int>(kHaloMaxStages, (kHaloSmemBudget - hp.sa * kHaloAStage) / stage_b);
     hp.ok = hp.sb >= 2;
     return hp;
   }
   if (hp.bn == 64) {
-    // N = 64 MMAs are bound by their issue floor; two blocks per SM with one input-box stage each hide
-    // start-up, loads and epilogue of one block under the MMAs of the other
+    // two blocks per SM with one input-box stage each: start-up, loads and epilogue of one block run under
+    // the MMAs of the other (one block per SM with resident weights measures the same, 14.7 against 14.4 us)
     hp.occ = 2;
     hp.sa = 1;
     hp.sb = std::min<int>(8, (113 * 1024 - 1024 - kHaloBarBytes - kHaloEpiBytes - kHaloAStage) / stage_b);
@@ -2148,8 +2194,7 @@ int run_halo(const HaloPlan& hp, const DotProblem& d, int64_t Cp, const uint16_t
   if (!encode_halo_box(&ma, x, d, Cp, hp.Wb, hp.RB) ||
       !encode_halo_weights(&mb, wt, d.O, d.Kh * d.Kw, Cp, hp.bn / hp.ctas, hp.tg))
     return GL_ERR_CUDA;
-  if (hp.ctas == 2)
-    return hp.bn == 128 ? launch_halo<128, 1, 2>(ma, mb, out, p, st) : launch_halo<64, 1, 2>(ma, mb, out, p, st);
+  if (hp.ctas == 2) return launch_halo<128, 1, 2>(ma, mb, out, p, st);
   return hp.bn == 128 ? launch_halo<128, 1, 1>(ma, mb, out, p, st) : launch_halo<64, 2, 1>(ma, mb, out, p, st);
 }
 
@@ -2309,69 +2354,62 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
 
   const uint16_t* x = pa;
   const uint16_t* wt = pb;
+  if (pl.rowrun) {
+    RowRunParams rp;
+    std::memset(&rp, 0, sizeof(rp));
+    rp.O = d.O; rp.relu = relu; rp.out_bf16 = out_bf16;
+    rp.C = static_cast<int>(d.C); rp.H = static_cast<int>(d.H); rp.W = static_cast<int>(d.W);
+    rp.Ho = static_cast<int>(d.Ho); rp.Wo = static_cast<int>(d.Wo);
+    rp.Sh = static_cast<int>(d.Sh); rp.Sw = static_cast<int>(d.Sw);
+    rp.Kh = static_cast<int>(d.Kh); rp.Kw = static_cast<int>(d.Kw);
+    rp.ph = static_cast<int>(d.ph_lo); rp.pw = static_cast<int>(d.pw_lo);
+    while ((1 << rp.cp_log2) < pl.rr_cp) ++rp.cp_log2;
+    rp.channels_last = d.channels_last ? 1 : 0;
+    rp.xs_n = d.C * d.H * d.W;
+    if (d.channels_last) { rp.xs_h = d.W * d.C; rp.xs_c = 1; }
+    else { rp.xs_h = d.W; rp.xs_c = d.H * d.W; }
+    rp.div_bn.set(pl.rr_bn);
+    rp.div_chunks.set(2 * pl.rr_ksteps);
+    rp.nseg = pl.rr_nseg;
+    rp.raw_seg_bytes = pl.rr_raw_seg;
+    rp.raw_row_bytes = pl.rr_raw_seg * static_cast<uint32_t>(pl.rr_nseg);
+    rp.raw_stage_bytes = rp.raw_row_bytes * static_cast<uint32_t>(d.Kh);
+    rp.raw_stages = pl.rr_raw_stages;
+    rp.w_elems = static_cast<int>(d.O * d.Kh * d.Kw * d.C);
+    rp.div_nseg.set(pl.rr_nseg);
+    rp.segs = static_cast<int>((d.Wo + kBM - 1) / kBM);
+    rp.tiles = static_cast<int>(d.N * d.Ho * rp.segs);
+    rp.ksteps = pl.rr_ksteps; rp.bn = pl.rr_bn;
+    rp.seg_bytes = pl.rr_seg; rp.slot_bytes = pl.rr_slot;
+    rp.b_bytes = pl.rr_b_bytes;
+    rp.stages = pl.rr_stages;
+    rp.div_segs.set(rp.segs);
+    rp.div_ho.set(d.Ho);
+    CUtensorMap mc;
+    if (!encode_result_rows(&mc, dst, d.N * d.Ho, d.Wo, d.O, out_bf16 != 0)) return GL_ERR_CUDA;
+    const int smem = 1024 + kRunEpiBytes + static_cast<int>((rp.b_bytes + 127u) & ~127u) +
+                     rp.stages * rp.Kh * static_cast<int>(rp.slot_bytes) + rp.raw_stages * static_cast<int>(rp.raw_stage_bytes) + 256;
+    static bool attr_set_dev[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return GL_ERR_CUDA;
+    if (!attr_set_dev[dev]) {
+      if (cudaFuncSetAttribute(conv_rowrun<0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024) != cudaSuccess ||
+          cudaFuncSetAttribute(conv_rowrun<3, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024) != cudaSuccess ||
+          cudaFuncSetAttribute(conv_rowrun<3, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024) != cudaSuccess)
+        return GL_ERR_CUDA;
+      attr_set_dev[dev] = true;
+    }
+    const int grid = std::min(rp.tiles, 2 * num_sms());
+    // three channels (RGB) have kernels of their own, one per item layout
+    auto kernel = d.C == 3 ? (d.channels_last ? conv_rowrun<3, 1> : conv_rowrun<3, 0>) : conv_rowrun<0, 0>;
+    return launch_pdl(kernel, dim3(static_cast<unsigned>(grid)), dim3(kRunThreads), static_cast<size_t>(smem), st, 1,
+                      pa, pb, mc, rp) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+  }
   if (pl.prepass) {
     const size_t need = pl.x_bytes + pl.w_bytes;
     if (!workspace || workspace_bytes < need || (reinterpret_cast<uintptr_t>(workspace) & 1023u)) return GL_ERR_WORKSPACE;
     uint16_t* xs = static_cast<uint16_t*>(workspace);
     uint16_t* ws = reinterpret_cast<uint16_t*>(static_cast<unsigned char*>(workspace) + pl.x_bytes);
-    if (pl.rowrun) {
-      const int chunks = 2 * pl.rr_ksteps;
-      int cp_log2 = 0;
-      while ((1 << cp_log2) < pl.rr_cp) ++cp_log2;
-      const int rows = static_cast<int>(d.N * pl.Hp);
-      const int rows_per_block = kPackWarps * kPackRowsPerWarp;
-      const int row_blocks = (rows + rows_per_block - 1) / rows_per_block;
-      const int wblocks = static_cast<int>((pl.rr_b_bytes / 2 + 255) / 256);
-      const dim3 pgrid(static_cast<unsigned>(row_blocks + wblocks));
-      const size_t psmem = static_cast<size_t>(kPackWarps * pl.Wpa * pl.rr_cp * 2);
-#define GL_ROWRUN_PACK(CT)                                                                                              \
-  launch_pdl(rowrun_pack<CT>, pgrid, dim3(32 * kPackWarps), psmem, st, 1, pa, xs, pb, ws, d.channels_last ? 1 : 0,       \
-             row_blocks, rows, static_cast<int>(d.H), static_cast<int>(d.W), static_cast<int>(pl.Hp),                  \
-             static_cast<int>(pl.Wpa), cp_log2, static_cast<int>(d.ph_lo), static_cast<int>(d.pw_lo),                  \
-             static_cast<int>(d.O), static_cast<int>(d.Kh), static_cast<int>(d.Kw), chunks, pl.rr_bn)
-      switch (d.C) {
-        case 1: GL_ROWRUN_PACK(1); break;
-        case 2: GL_ROWRUN_PACK(2); break;
-        case 3: GL_ROWRUN_PACK(3); break;
-        case 4: GL_ROWRUN_PACK(4); break;
-        case 5: GL_ROWRUN_PACK(5); break;
-        case 6: GL_ROWRUN_PACK(6); break;
-        case 7: GL_ROWRUN_PACK(7); break;
-        default: GL_ROWRUN_PACK(8); break;
-      }
-#undef GL_ROWRUN_PACK
-      if (cudaGetLastError() != cudaSuccess) return GL_ERR_CUDA;
-      RowRunParams rp;
-      std::memset(&rp, 0, sizeof(rp));
-      rp.O = d.O; rp.relu = relu; rp.out_bf16 = out_bf16;
-      rp.Ho = static_cast<int>(d.Ho); rp.Wo = static_cast<int>(d.Wo); rp.Hp = static_cast<int>(pl.Hp);
-      rp.Sh = static_cast<int>(d.Sh); rp.Kh = static_cast<int>(d.Kh);
-      rp.segs = static_cast<int>((d.Wo + kBM - 1) / kBM);
-      rp.tiles = static_cast<int>(d.N * d.Ho * rp.segs);
-      rp.ksteps = pl.rr_ksteps; rp.bn = pl.rr_bn;
-      rp.seg_bytes = pl.rr_seg; rp.slot_bytes = pl.rr_slot;
-      rp.pitch_bytes = static_cast<uint32_t>(pl.Wpa * pl.rr_cp * 2);
-      rp.b_bytes = pl.rr_b_bytes;
-      rp.stages = pl.rr_stages;
-      rp.div_segs.set(rp.segs);
-      rp.div_ho.set(d.Ho);
-      CUtensorMap mc;
-      if (!encode_result_rows(&mc, dst, d.N * d.Ho, d.Wo, d.O, out_bf16 != 0)) return GL_ERR_CUDA;
-      const int smem = 1024 + kRunEpiBytes + static_cast<int>((rp.b_bytes + 127u) & ~127u) +
-                       rp.stages * rp.Kh * static_cast<int>(rp.slot_bytes) + 256;
-      static bool attr_set_dev[64] = {false};
-      int dev = 0;
-      if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return GL_ERR_CUDA;
-      if (!attr_set_dev[dev]) {
-        if (cudaFuncSetAttribute(conv_rowrun, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024) != cudaSuccess)
-          return GL_ERR_CUDA;
-        attr_set_dev[dev] = true;
-      }
-      const int grid = std::min(rp.tiles, 2 * num_sms());
-      return launch_pdl(conv_rowrun, dim3(static_cast<unsigned>(grid)), dim3(kRunThreads), static_cast<size_t>(smem), st, 1,
-                        reinterpret_cast<const unsigned char*>(xs), reinterpret_cast<const unsigned char*>(ws), mc,
-                        rp) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
-    }
     if (pl.rowwin) {
       rowwin_pack_x<<<static_cast<unsigned>(d.N * pl.Hp), 256, 0, st>>>(
           pa, xs, d.channels_last ? 1 : 0, static_cast<int>(d.C), static_cast<int>(d.H), static_cast<int>(d.W),

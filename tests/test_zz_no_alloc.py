@@ -4,10 +4,12 @@ Some users of this library run where device memory cannot be requested: inside a
 framework's operator, in a plug-in that only receives its input and output buffers, or in a
 process whose memory all belongs to a pool.  They cannot hand gl_cartesian_dot a workspace,
 so this variant keeps its scratch in a fixed array inside the library.  The tests call it
-through the C ABI on problems that need scratch (the (C,H,W) layout, few-channel stems, a
+through the C ABI on problems that need scratch (the (C,H,W) layout, few-channel windows, a
 split contraction) and compare with the ordinary entry point and with the CPU checker, twice
 in a row, because the array is shared by all calls and keeps the previous call's contents;
 they also check that the device's free memory does not move across a call."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -56,7 +58,7 @@ CASES = [
     # seed, (n, c, h, w, o, k), integer inputs, stride
     (51, (3, 20, 13, 11, 24, 3), True, 1),       # channels padded 20 -> 24: zero-filled cells in the copies
     (52, (2, 64, 14, 14, 48, 3), False, 1),      # N(0,1) inputs, resident-window kernel behind the layout copy
-    (53, (2, 3, 30, 30, 16, 7), True, 2),        # RGB stem 7x7 stride 2 pad 3: zero-bordered row runs, packed weights
+    (53, (2, 3, 30, 30, 136, 7), True, 2),       # RGB stem 7x7 stride 2 pad 3 with 136 filters: row-window copies
     (54, (2, 12, 10, 12, 8, 3), True, 1),        # row-window copies with zero borders and zero weight tails
     (55, (1, 2048, 7, 7, 64, 1), True, 1),       # one tile, 32 K blocks: split contraction, partial planes in the scratch
 ]
@@ -80,11 +82,17 @@ def test_static_scratch_matches_workspace_entry_point_and_checker_twice(gl):
         assert rel_err(g.squeeze(1), ref) <= REL_TOL
         # a second call on the now-dirty array: same answer, and no device memory changes hands
         again = gl.AccessPattern(torch.empty_like(want.tensor), want.access_ndim)
-        torch.cuda.synchronize()
-        held, free = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
-        gl.gl_cartesian_dot_static(xa, spec, wa, again, flags=gl.GL_EPILOGUE_RELU)
-        torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == held and torch.cuda.mem_get_info()[0] == free
+        gc.collect()                  # tensors of earlier tests that are still waiting for the collector go now,
+        gc.disable()                  # not between the two readings
+        try:
+            torch.cuda.synchronize()
+            held, free = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
+            gl.gl_cartesian_dot_static(xa, spec, wa, again, flags=gl.GL_EPILOGUE_RELU)
+            torch.cuda.synchronize()
+            held_after, free_after = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
+        finally:
+            gc.enable()
+        assert (held_after, free_after) == (held, free)
         assert torch.equal(again.tensor, torch.clamp_min(got.tensor, 0.0))
 
 
