@@ -10,8 +10,11 @@
  *
  * Conventions for every call
  *   - Return value: GL_OK or a GL_ERR_* code; gl_strerror() names it.
- *   - All arguments are validated before anything is enqueued; a call that
- *     returns an error has launched nothing and written nothing.
+ *   - All arguments are validated, and every descriptor a call needs is prepared,
+ *     before anything is enqueued: a call that returns any error other than a
+ *     failed kernel launch has launched nothing and written nothing.  (A launch
+ *     that the runtime itself refuses, GL_ERR_CUDA, may follow an earlier launch
+ *     of the same call, which has then written the workspace but not `out`.)
  *   - gl_shape_* calls are host-only: they read shapes, never `data`.
  *   - Device calls enqueue kernels on `stream` (a cudaStream_t passed as
  *     void*, NULL = the default stream).  They never synchronise and never
@@ -196,7 +199,11 @@ GL_API int gl_compute_reduce_sum(const gl_ap* in, gl_ap* out, void* stream);
  * Everything else runs on a slower general kernel.  The sum over the window is
  * taken in an unspecified order.  `workspace` must hold at least
  * gl_cartesian_dot_workspace() bytes (it may be NULL when that is 0) and must be
- * 1024-byte aligned; its contents are scratch.  The kernels are launched with programmatic
+ * 1024-byte aligned; its contents are scratch.  Few-channel convolutions (at most
+ * 8 / Sw channels, the RGB stem) and channels-last items with a channel count
+ * that is a multiple of 8 need none: the kernels read both operands where they
+ * are.  Encoded tensor maps are kept per argument list, so a repeated call on the
+ * same buffers skips the driver's encoding.  The kernels are launched with programmatic
  * stream serialisation: their set-up may run while the preceding kernel of the stream
  * drains, and they wait for its completion before their first access to memory. */
 GL_API int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w_or_null, const gl_ap* a1, gl_ap* out,
@@ -219,9 +226,11 @@ GL_API size_t gl_cartesian_dot_workspace(const gl_ap* a0, const gl_windows* w_or
  * cudaMalloc, cudaFree or other allocating routine.
  *
  *   - Same arguments, results and error codes as gl_cartesian_dot without the workspace
- *     pair.  If gl_cartesian_dot_workspace() for these arguments exceeds
- *     GL_STATIC_SCRATCH_BYTES the call returns GL_ERR_WORKSPACE and launches nothing
- *     (for scale: the (C,H,W) activations of a 32x64x56x56 convolution need 12.3 MiB).
+ *     pair.  If the layout copies of these arguments exceed GL_STATIC_SCRATCH_BYTES
+ *     the call returns GL_ERR_WORKSPACE and launches nothing (for scale: the (C,H,W)
+ *     activations of a 32x64x56x56 convolution need 12.3 MiB).  A contraction that
+ *     gl_cartesian_dot would split, and whose partial planes do not fit beside the
+ *     copies, runs unsplit instead.
  *   - The first call on each device looks up the array's device address (that device
  *     must be current); make that first call before any stream capture begins.
  *   - All calls share the one array and it keeps whatever the last call left in it.
@@ -234,7 +243,11 @@ GL_API int gl_cartesian_dot_static(const gl_ap* a0, const gl_windows* w_or_null,
 
 /* compute reduceMax (windows? in) (operator table, Fig. 2c max pooling): the largest
  * value of every item; with w given the windows are formed on the fly and never
- * stored.  GL_F32.  Inputs must be NaN-free. */
+ * stored.  GL_F32 in any form.  GL_BF16 (results of GL_OUT_BF16 convolutions) in two forms:
+ * 2D windows over ((..),(H,W)) items, and channels-last items ((N),(H,W,C)) with window
+ * (Kh,Kw,1), stride (Sh,Sw,1) and C a multiple of 8; other bf16 forms return
+ * GL_ERR_UNSUPPORTED.  The largest of a set of values is one of them, so nothing is rounded.
+ * Inputs must be NaN-free. */
 GL_API int gl_compute_reduce_max(const gl_ap* in, const gl_windows* w_or_null, gl_ap* out, void* stream);
 
 /* compute relu (not in the paper's operator table): out = in > 0 ? in : +0, item

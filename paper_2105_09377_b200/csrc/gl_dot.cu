@@ -19,7 +19,10 @@
 #include <algorithm>
 #include <cstdlib>
 #include <cstring>
+#include <functional>
 #include <mutex>
+#include <string>
+#include <unordered_map>
 
 #include "gl_internal.h"
 #include "gl_launch.cuh"
@@ -552,23 +555,6 @@ constexpr int kBK = 64;          // bf16 elements per K block = one 128-byte swi
 constexpr int kTcThreads = 224;  // warp 0 TMA (A), warp 1 MMA + TMEM, warps 2-5 epilogue, warp 6 TMA (B)
 
 enum AMode { kDense = 0, kIm2col = 1, kIm2colGranule = 2, kRowWin = 3 };
-
-// Division of a 31-bit number by a fixed divisor as multiply-high + shift: the loops below run
-// in single threads, where an integer division is a ~150-cycle dependent chain.
-// With p = ceil(log2 d) and m = ceil(2^(31+p) / d):  n / d = umulhi(n, m) >> (p - 1)  for n < 2^31.
-struct FastDiv {
-  uint32_t d, mul, shift;
-  __host__ void set(int64_t divisor) {
-    d = static_cast<uint32_t>(divisor);
-    uint32_t p = 0;
-    while ((1ull << p) < d) ++p;
-    if (p == 0) { mul = 0; shift = 0; return; }
-    mul = static_cast<uint32_t>(((1ull << (31 + p)) + d - 1) / d);
-    shift = p - 1;
-  }
-  __device__ __forceinline__ uint32_t div(uint32_t n) const { return d == 1 ? n : (__umulhi(n, mul) >> shift); }
-  __device__ __forceinline__ void divmod(uint32_t n, uint32_t& q, uint32_t& r) const { q = div(n); r = n - q * d; }
-};
 
 struct TcParams {
   int64_t M, O, K;        // K as laid out in B (for conv: Kh*Kw*Cp)
@@ -1722,6 +1708,78 @@ const DriverApi& driver_api() {
   return api;
 }
 
+// Encoded tensor maps, kept per argument list (base address, extents, strides, box, modes).  A program that
+// calls the library on the same buffers again - every layer of a network on every step - skips the driver's
+// encoding, which costs more host time than the rest of a call.  The map depends on nothing but its arguments,
+// so a recycled address with the same geometry yields the same, still valid, map.
+class TensorMapCache {
+ public:
+  template <typename Encode>
+  bool get(const std::string& key, CUtensorMap* out, Encode&& encode) {
+    {
+      std::lock_guard<std::mutex> lock(mu_);
+      auto it = maps_.find(key);
+      if (it != maps_.end()) { *out = it->second; return true; }
+    }
+    if (!encode(out)) return false;
+    std::lock_guard<std::mutex> lock(mu_);
+    if (maps_.size() >= kMaxEntries) maps_.clear();
+    maps_.emplace(key, *out);
+    return true;
+  }
+
+ private:
+  static constexpr size_t kMaxEntries = 4096;
+  std::mutex mu_;
+  std::unordered_map<std::string, CUtensorMap> maps_;
+};
+
+TensorMapCache& map_cache() {
+  static TensorMapCache cache;
+  return cache;
+}
+
+template <typename T>
+void key_add(std::string* key, const T* v, size_t n) { key->append(reinterpret_cast<const char*>(v), n * sizeof(T)); }
+
+bool encode_tiled_cached(CUtensorMap* m, CUtensorMapDataType dt, cuuint32_t rank, const void* base, const cuuint64_t* dims,
+                         const cuuint64_t* strides, const cuuint32_t* box, const cuuint32_t* estr, CUtensorMapSwizzle swz,
+                         CUtensorMapL2promotion l2) {
+  std::string key;
+  key.reserve(160);
+  const uint32_t head[4] = {0u, static_cast<uint32_t>(dt), rank, static_cast<uint32_t>(swz) | (static_cast<uint32_t>(l2) << 8)};
+  key_add(&key, head, 4);
+  key_add(&key, &base, 1);
+  key_add(&key, dims, rank);
+  key_add(&key, strides, rank - 1);
+  key_add(&key, box, rank);
+  key_add(&key, estr, rank);
+  return map_cache().get(key, m, [&](CUtensorMap* out) {
+    return driver_api().tiled(out, dt, rank, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                              l2, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  });
+}
+
+bool encode_im2col_cached(CUtensorMap* m, const void* base, const cuuint64_t* dims, const cuuint64_t* strides, const int* lower,
+                          const int* upper, cuuint32_t channels, cuuint32_t pixels, const cuuint32_t* estr,
+                          CUtensorMapSwizzle swz) {
+  std::string key;
+  key.reserve(160);
+  const uint32_t head[4] = {1u, channels, pixels, static_cast<uint32_t>(swz)};
+  key_add(&key, head, 4);
+  key_add(&key, &base, 1);
+  key_add(&key, dims, 4);
+  key_add(&key, strides, 3);
+  key_add(&key, lower, 2);
+  key_add(&key, upper, 2);
+  key_add(&key, estr, 4);
+  return map_cache().get(key, m, [&](CUtensorMap* out) {
+    return driver_api().im2col(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, lower, upper,
+                               channels, pixels, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  });
+}
+
 int num_sms() {
   static int sms[64] = {0};   // per device
   int dev = 0;
@@ -1738,9 +1796,7 @@ bool encode_kmajor_sw128(CUtensorMap* m, const void* base, int64_t rows, int64_t
   const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * 2};
   const cuuint32_t box[2] = {kBK, static_cast<cuuint32_t>(box_rows)};
   const cuuint32_t estr[2] = {1, 1};
-  return driver_api().tiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_tiled_cached(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
 }
 
 // [rows, K] bf16 viewed as {8 elements, rows, K/8 granules}: one box {8, box_rows, 8}
@@ -1750,9 +1806,7 @@ bool encode_kmajor_granules(CUtensorMap* m, const void* base, int64_t rows, int6
   const cuuint64_t strides[2] = {static_cast<cuuint64_t>(K) * 2, 16};
   const cuuint32_t box[3] = {8, static_cast<cuuint32_t>(box_rows), 8};
   const cuuint32_t estr[3] = {1, 1, 1};
-  return driver_api().tiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_tiled_cached(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
 }
 
 // Channels-last activations (N,H,W,Cp) as an im2col tensor map: 128 window
@@ -1765,10 +1819,8 @@ bool encode_im2col(CUtensorMap* m, const void* base, const DotProblem& d, int64_
   const int lower[2] = {static_cast<int>(-d.pw_lo), static_cast<int>(-d.ph_lo)};
   const int upper[2] = {static_cast<int>(d.pw_hi - (d.Kw - 1)), static_cast<int>(d.ph_hi - (d.Kh - 1))};
   const cuuint32_t estr[4] = {1, static_cast<cuuint32_t>(d.Sw), static_cast<cuuint32_t>(d.Sh), 1};
-  return driver_api().im2col(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, lower,
-                             upper, static_cast<cuuint32_t>(channels), kBM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                             swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
-                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_im2col_cached(m, base, dims, strides, lower, upper, static_cast<cuuint32_t>(channels), kBM, estr,
+                              swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE);
 }
 
 // Result planes [planes, M, O]: boxes of 32 rows x 128 bytes (32 fp32 or 64 bf16 columns), 128-byte swizzle
@@ -1779,9 +1831,7 @@ bool encode_result(CUtensorMap* m, float* base, int64_t M, int64_t O, int64_t pl
   const cuuint64_t strides[2] = {static_cast<cuuint64_t>(O) * es, static_cast<cuuint64_t>(M * O) * es};
   const cuuint32_t box[3] = {bf16 ? 64u : 32u, 32, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
-  return driver_api().tiled(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_tiled_cached(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE);
 }
 
 // fp32 result of a row-window convolution viewed as (N*Ho, Wo, O): 32x32 boxes inside one output row.
@@ -1791,9 +1841,7 @@ bool encode_result_rows(CUtensorMap* m, float* base, int64_t rows, int64_t Wo, i
   const cuuint64_t strides[2] = {static_cast<cuuint64_t>(O) * es, static_cast<cuuint64_t>(Wo * O) * es};
   const cuuint32_t box[3] = {bf16 ? 64u : 32u, 32, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
-  return driver_api().tiled(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_tiled_cached(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE);
 }
 
 // Row-window activations (N*Hp, Wpa, Cp): dimension 1 walks output columns with a stride of
@@ -1803,13 +1851,17 @@ bool encode_rowwin(CUtensorMap* m, const void* base, int64_t rows, int64_t Wo, i
   const cuuint64_t strides[2] = {static_cast<cuuint64_t>(Sw * Cp) * 2, static_cast<cuuint64_t>(Wpa * Cp) * 2};
   const cuuint32_t box[3] = {64, kBM, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
-  return driver_api().tiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_tiled_cached(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
 }
 
+// The layout copies of a call (if it has any) are enqueued by this callable, which the launch functions run
+// right before their own launch: everything that can fail without a launch - tensor-map encoding, function
+// attributes, occupancy queries - has then been done, so a call refused for such a reason has enqueued nothing.
+using PreLaunch = std::function<int()>;
+inline int run_pre(const PreLaunch& pre) { return pre ? pre() : GL_OK; }
+
 template <int BN, int MODE, int G, int OCC, int CTAS = 1>
-int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams p, cudaStream_t st) {
+int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams p, cudaStream_t st, const PreLaunch& pre) {
   using Cfg = TcCfg<BN, G, OCC, CTAS>;
   static bool attr_set_dev[64] = {false};   // per device; benign race: the attribute call is idempotent
   static int max_pairs_dev[64] = {0};       // CTAS == 2: pairs that can be resident at once
@@ -1862,6 +1914,7 @@ int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams
     mc = ma;   // unused by the kernel; any valid map
   }
   const int tiles = p.tiles_m * p.tiles_n * p.ksplit;
+  if (const int rc = run_pre(pre)) return rc;
   if (CTAS == 2) {
     const int pairs = std::min(tiles, std::min(max_pairs_dev[dev], num_sms() / 2));
     if (launch_pdl(dot_tc<BN, MODE, G, OCC, CTAS>, dim3(static_cast<unsigned>(2 * pairs)), dim3(kTcThreads),
@@ -1882,22 +1935,22 @@ bool use_pair(int mode, int bn, const TcParams& p) {
 
 template <int MODE>
 int launch_tc_bn(int bn, const CUtensorMap& ma, const CUtensorMap& mb, float* out, const TcParams& p,
-                 cudaStream_t st) {
+                 cudaStream_t st, const PreLaunch& pre) {
   switch (bn) {
     case 256:
       if (use_pair(MODE, bn, p)) {
         TcParams pp = p;
         pp.tiles_m = (p.tiles_m + 1) / 2;
-        return launch_tc<256, (MODE == kDense || MODE == kIm2col) ? MODE : kDense, 1, 1, 2>(ma, mb, out, pp, st);
+        return launch_tc<256, (MODE == kDense || MODE == kIm2col) ? MODE : kDense, 1, 1, 2>(ma, mb, out, pp, st, pre);
       }
-      return launch_tc<256, MODE, 1, 1>(ma, mb, out, p, st);
+      return launch_tc<256, MODE, 1, 1>(ma, mb, out, p, st, pre);
     // narrower tiles are bound by the MMA-issuing thread (about 50 cycles per MMA, 250 per commit):
     // 128 wide: two K blocks per stage halve the commits; 64 wide: two blocks per SM interleave
     // their issue threads (measured on the 3x3 and 1x1 convolution shapes)
-    case 128: return launch_tc<128, MODE, 2, 1>(ma, mb, out, p, st);
+    case 128: return launch_tc<128, MODE, 2, 1>(ma, mb, out, p, st, pre);
     default:
-      if (MODE == kIm2colGranule) return launch_tc<64, MODE, 1, 1>(ma, mb, out, p, st);
-      return launch_tc<64, MODE, 1, 2>(ma, mb, out, p, st);
+      if (MODE == kIm2colGranule) return launch_tc<64, MODE, 1, 1>(ma, mb, out, p, st, pre);
+      return launch_tc<64, MODE, 1, 2>(ma, mb, out, p, st, pre);
   }
 }
 
@@ -2106,9 +2159,7 @@ bool encode_halo_box(CUtensorMap* m, const void* base, const DotProblem& d, int6
                                  static_cast<cuuint64_t>(d.H * d.W * Cp) * 2};
   const cuuint32_t box[4] = {kBK, static_cast<cuuint32_t>(Wb), static_cast<cuuint32_t>(RB), 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
-  return driver_api().tiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_tiled_cached(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
 }
 
 // Weights (O, Kh, Kw, Cp) viewed as (64 channels, O, chunk, tap): one box = BN rows x 64 channels of
@@ -2119,13 +2170,12 @@ bool encode_halo_weights(CUtensorMap* m, const void* base, int64_t O, int64_t ta
   const cuuint64_t strides[3] = {static_cast<cuuint64_t>(taps * Cp) * 2, kBK * 2, static_cast<cuuint64_t>(Cp) * 2};
   const cuuint32_t box[4] = {kBK, static_cast<cuuint32_t>(bn), 1, static_cast<cuuint32_t>(tg)};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
-  return driver_api().tiled(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
-                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_tiled_cached(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
 }
 
 template <int BN, int OCC, int CTAS>
-int launch_halo(const CUtensorMap& ma, const CUtensorMap& mb, float* out, const HaloParams& p, cudaStream_t st) {
+int launch_halo(const CUtensorMap& ma, const CUtensorMap& mb, float* out, const HaloParams& p, cudaStream_t st,
+                const PreLaunch& pre) {
   const int smem = p.sa_stages * kHaloAStage + p.sb_stages * static_cast<int>(p.b_bytes) + kHaloEpiBytes + kHaloBarBytes + 1024;
   static bool attr_set_dev[64] = {false};
   static int max_pairs_dev[64] = {0};       // CTAS == 2: pairs that can be resident at once
@@ -2158,6 +2208,7 @@ int launch_halo(const CUtensorMap& ma, const CUtensorMap& mb, float* out, const 
     attr_set_dev[dev] = true;
   }
   const int tiles = p.tiles_m * p.tiles_n;
+  if (const int rc = run_pre(pre)) return rc;
   if (CTAS == 2) {
     const int pairs = std::min(tiles, std::min(max_pairs_dev[dev], OCC * (num_sms() / 2)));
     return launch_pdl(conv_halo<BN, OCC, CTAS>, dim3(static_cast<unsigned>(2 * pairs)), dim3(kTcThreads),
@@ -2169,7 +2220,7 @@ int launch_halo(const CUtensorMap& ma, const CUtensorMap& mb, float* out, const 
 }
 
 int run_halo(const HaloPlan& hp, const DotProblem& d, int64_t Cp, const uint16_t* x, const uint16_t* wt, float* out,
-             int relu, int out_bf16, cudaStream_t st) {
+             int relu, int out_bf16, cudaStream_t st, const PreLaunch& pre) {
   HaloParams p;
   std::memset(&p, 0, sizeof(p));
   p.O = d.O; p.relu = relu; p.out_bf16 = out_bf16;
@@ -2194,8 +2245,8 @@ int run_halo(const HaloPlan& hp, const DotProblem& d, int64_t Cp, const uint16_t
   if (!encode_halo_box(&ma, x, d, Cp, hp.Wb, hp.RB) ||
       !encode_halo_weights(&mb, wt, d.O, d.Kh * d.Kw, Cp, hp.bn / hp.ctas, hp.tg))
     return GL_ERR_CUDA;
-  if (hp.ctas == 2) return launch_halo<128, 1, 2>(ma, mb, out, p, st);
-  return hp.bn == 128 ? launch_halo<128, 1, 1>(ma, mb, out, p, st) : launch_halo<64, 2, 1>(ma, mb, out, p, st);
+  if (hp.ctas == 2) return launch_halo<128, 1, 2>(ma, mb, out, p, st, pre);
+  return hp.bn == 128 ? launch_halo<128, 1, 1>(ma, mb, out, p, st, pre) : launch_halo<64, 2, 1>(ma, mb, out, p, st, pre);
 }
 
 // A 1x1, stride-1, unpadded window over channels-last items is no window at all: the activations
@@ -2242,25 +2293,36 @@ void fill_general(const gl_ap* a0, const gl_windows* w, const DotProblem& d, Gen
   g->item = s;
 }
 
+
+// Scratch of a call in two parts: the layout copies, without which it cannot run, and the partial planes of a
+// split contraction, without which it runs unsplit.
+void workspace_parts(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, uint32_t flags, size_t* required,
+                     size_t* optional) {
+  *required = *optional = 0;
+  DotProblem d;
+  if (classify_dot(a0, w, a1, &d) != GL_OK) return;
+  if (flags & GL_DOT_GENERAL_KERNEL) return;
+  if (conv_is_plain_matrix(d, flags)) d.conv = false;
+  if (!d.conv) {
+    if (dense_tc_ok(d)) *optional = plan_tiles(d.M, d.O, (d.K + kBK - 1) / kBK, true).partial_bytes;
+    return;
+  }
+  const ConvPlan pl = plan_conv(d, flags);
+  if (!pl.tc) return;
+  *required = pl.prepass ? pl.x_bytes + pl.w_bytes : 0;
+  // the resident-window and row-run kernels never split
+  if (!pl.rowwin && !pl.rowrun && pl.Cp >= kBK && !(flags & GL_OUT_NCHW) && !plan_halo(d, pl, flags).ok)
+    *optional = plan_tiles(d.M, d.O, d.Kh * d.Kw * ((pl.Cp + kBK - 1) / kBK), true).partial_bytes;
+}
+
 }  // namespace
 
 extern "C" {
 
 size_t gl_cartesian_dot_workspace(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, uint32_t flags) {
-  DotProblem d;
-  if (classify_dot(a0, w, a1, &d) != GL_OK) return 0;
-  if (flags & GL_DOT_GENERAL_KERNEL) return 0;
-  if (conv_is_plain_matrix(d, flags)) d.conv = false;
-  if (!d.conv) {
-    if (!dense_tc_ok(d)) return 0;
-    return plan_tiles(d.M, d.O, (d.K + kBK - 1) / kBK, true).partial_bytes;
-  }
-  const ConvPlan pl = plan_conv(d, flags);
-  if (!pl.tc) return 0;
-  size_t need = pl.prepass ? pl.x_bytes + pl.w_bytes : 0;
-  if (!pl.rowwin && pl.Cp >= kBK && !(flags & GL_OUT_NCHW))
-    need += plan_tiles(d.M, d.O, d.Kh * d.Kw * ((pl.Cp + kBK - 1) / kBK), true).partial_bytes;
-  return need;
+  size_t required = 0, optional = 0;
+  workspace_parts(a0, w, a1, flags, &required, &optional);
+  return required + optional;
 }
 
 int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_ap* out, uint32_t flags,
@@ -2349,11 +2411,12 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     if (!encode_kmajor_sw128(&ma, pa, d.M, d.K, kBM) ||
         !encode_kmajor_sw128(&mb, pb, d.O, d.K, use_pair(kDense, bn, p) ? bn / 2 : bn))
       return GL_ERR_CUDA;
-    return finish(launch_tc_bn<kDense>(bn, ma, mb, dst, p, st));
+    return finish(launch_tc_bn<kDense>(bn, ma, mb, dst, p, st, PreLaunch()));
   }
 
   const uint16_t* x = pa;
   const uint16_t* wt = pb;
+  PreLaunch pre;   // the layout copies, enqueued by the launch function once nothing else can fail
   if (pl.rowrun) {
     RowRunParams rp;
     std::memset(&rp, 0, sizeof(rp));
@@ -2411,13 +2474,15 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     uint16_t* xs = static_cast<uint16_t*>(workspace);
     uint16_t* ws = reinterpret_cast<uint16_t*>(static_cast<unsigned char*>(workspace) + pl.x_bytes);
     if (pl.rowwin) {
-      rowwin_pack_x<<<static_cast<unsigned>(d.N * pl.Hp), 256, 0, st>>>(
-          pa, xs, d.channels_last ? 1 : 0, static_cast<int>(d.C), static_cast<int>(d.H), static_cast<int>(d.W),
-          static_cast<int>(pl.Hp), static_cast<int>(pl.Wpa), static_cast<int>(pl.Cp), static_cast<int>(d.ph_lo),
-          static_cast<int>(d.pw_lo));
-      rowwin_pack_w<<<static_cast<unsigned>(std::min<int64_t>((d.O * d.Kh * 64 + 255) / 256, 1 << 20)), 256, 0, st>>>(
-          pb, ws, d.channels_last ? 1 : 0, d.O, d.C, d.Kh, d.Kw, static_cast<int>(pl.Cp));
-      if (cudaGetLastError() != cudaSuccess) return GL_ERR_CUDA;
+      pre = [=]() -> int {
+        rowwin_pack_x<<<static_cast<unsigned>(d.N * pl.Hp), 256, 0, st>>>(
+            pa, xs, d.channels_last ? 1 : 0, static_cast<int>(d.C), static_cast<int>(d.H), static_cast<int>(d.W),
+            static_cast<int>(pl.Hp), static_cast<int>(pl.Wpa), static_cast<int>(pl.Cp), static_cast<int>(d.ph_lo),
+            static_cast<int>(d.pw_lo));
+        rowwin_pack_w<<<static_cast<unsigned>(std::min<int64_t>((d.O * d.Kh * 64 + 255) / 256, 1 << 20)), 256, 0, st>>>(
+            pb, ws, d.channels_last ? 1 : 0, d.O, d.C, d.Kh, d.Kw, static_cast<int>(pl.Cp));
+        return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+      };
       p.K = d.Kh * kBK;
       p.kblocks = static_cast<int>(d.Kh);
       p.Cp = static_cast<int>(pl.Cp);
@@ -2429,16 +2494,19 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
       p.tiles_m = static_cast<int>(d.N * d.Ho * p.segs);
       if (encode_rowwin(&ma, xs, d.N * pl.Hp, d.Wo, pl.Wpa, pl.Cp, d.Sw) &&
           encode_kmajor_sw128(&mb, ws, d.O, p.K, bn))
-        return launch_tc_bn<kRowWin>(bn, ma, mb, dst, p, st);
+        return launch_tc_bn<kRowWin>(bn, ma, mb, dst, p, st, pre);
       return GL_ERR_CUDA;
     }
     const int64_t HW = d.H * d.W, T = d.Kh * d.Kw;
     if (d.channels_last) {
       // (N,H,W,C) with C not a multiple of 8: re-pitch the channel dim (a (N*HW, C) -> (N*HW, Cp) copy)
-      weights_to_channels_last<<<static_cast<unsigned>(std::min<int64_t>((d.N * HW * pl.Cp + 255) / 256, 1 << 20)), 256, 0,
-                                 st>>>(pa, xs, d.N * HW, d.C, 1, pl.Cp);
-      weights_to_channels_last<<<static_cast<unsigned>(std::min<int64_t>((d.O * T * pl.Cp + 255) / 256, 1 << 20)), 256, 0,
-                                 st>>>(pb, ws, d.O * T, d.C, 1, pl.Cp);
+      pre = [=]() -> int {
+        weights_to_channels_last<<<static_cast<unsigned>(std::min<int64_t>((d.N * HW * pl.Cp + 255) / 256, 1 << 20)), 256, 0,
+                                   st>>>(pa, xs, d.N * HW, d.C, 1, pl.Cp);
+        weights_to_channels_last<<<static_cast<unsigned>(std::min<int64_t>((d.O * T * pl.Cp + 255) / 256, 1 << 20)), 256, 0,
+                                   st>>>(pb, ws, d.O * T, d.C, 1, pl.Cp);
+        return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+      };
     } else {
       PrepassParams pp;
       std::memset(&pp, 0, sizeof(pp));
@@ -2464,21 +2532,25 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
         pp.by_Ws = make_fastdiv(pp.Ws);
         if (!copy_w) ws = const_cast<uint16_t*>(pb);
         const size_t smem = std::max<size_t>(64 * 66 * 2, static_cast<size_t>(wwarps) * 64 * T * 2);
-        if (launch_pdl(nchw_prepass, dim3(static_cast<unsigned>(x_blocks + w_blocks)), dim3(256), smem, st, 1, pa, xs, pb,
-                       ws, pp) != cudaSuccess)
-          return GL_ERR_CUDA;
+        uint16_t* const ws_dst = ws;
+        pre = [=]() -> int {
+          return launch_pdl(nchw_prepass, dim3(static_cast<unsigned>(x_blocks + w_blocks)), dim3(256), smem, st, 1, pa, xs, pb,
+                            ws_dst, pp) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+        };
       } else if (pl.as_matrix) {
         return GL_ERR_UNSUPPORTED;
       } else {
         if (d.N > 65535 || (d.C + 31) / 32 > 65535) return GL_ERR_UNSUPPORTED;
         const dim3 grid(static_cast<unsigned>((HW + 31) / 32), static_cast<unsigned>((pl.Cp + 31) / 32),
                         static_cast<unsigned>(d.N));
-        nchw_to_nhwc_pad<<<grid, 256, 0, st>>>(pa, xs, d.C, HW, pl.Cp);
-        weights_to_channels_last<<<static_cast<unsigned>(std::min<int64_t>((d.O * T * pl.Cp + 255) / 256, 1 << 20)), 256,
-                                   0, st>>>(pb, ws, d.O, d.C, T, pl.Cp);
+        pre = [=]() -> int {
+          nchw_to_nhwc_pad<<<grid, 256, 0, st>>>(pa, xs, d.C, HW, pl.Cp);
+          weights_to_channels_last<<<static_cast<unsigned>(std::min<int64_t>((d.O * T * pl.Cp + 255) / 256, 1 << 20)), 256,
+                                     0, st>>>(pb, ws, d.O, d.C, T, pl.Cp);
+          return cudaGetLastError() == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+        };
       }
     }
-    if (cudaGetLastError() != cudaSuccess) return GL_ERR_CUDA;
     x = xs;
     wt = ws;
   }
@@ -2489,9 +2561,9 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     if (!encode_kmajor_sw128(&ma, x, d.M, Cp, kBM) ||
         !encode_kmajor_sw128(&mb, wt, d.O, Cp, use_pair(kDense, bn, p) ? bn / 2 : bn))
       return GL_ERR_CUDA;
-    return finish(launch_tc_bn<kDense>(bn, ma, mb, dst, p, st));
+    return finish(launch_tc_bn<kDense>(bn, ma, mb, dst, p, st, pre));
   }
-  if (hp.ok) return run_halo(hp, d, Cp, x, wt, dst, relu, out_bf16, st);
+  if (hp.ok) return run_halo(hp, d, Cp, x, wt, dst, relu, out_bf16, st, pre);
   p.K = taps * Cp;
   p.Cp = static_cast<int>(Cp);
   p.Kh = static_cast<int>(d.Kh); p.Kw = static_cast<int>(d.Kw);
@@ -2504,12 +2576,12 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     if (!encode_im2col(&ma, x, d, Cp, kBK, true) ||
         !encode_kmajor_sw128(&mb, wt, d.O, p.K, use_pair(kIm2col, bn, p) ? bn / 2 : bn))
       return GL_ERR_CUDA;
-    return finish(launch_tc_bn<kIm2col>(bn, ma, mb, dst, p, st));
+    return finish(launch_tc_bn<kIm2col>(bn, ma, mb, dst, p, st, pre));
   }
   p.cchunks = static_cast<int>(Cp / 8);
   p.kblocks = static_cast<int>((taps * p.cchunks + 7) / 8);
   if (!encode_im2col(&ma, x, d, Cp, 8, false) || !encode_kmajor_granules(&mb, wt, d.O, p.K, bn)) return GL_ERR_CUDA;
-  return launch_tc_bn<kIm2colGranule>(bn, ma, mb, dst, p, st);
+  return launch_tc_bn<kIm2colGranule>(bn, ma, mb, dst, p, st, pre);
 }
 
 int gl_selftest_bounded_wait(uint32_t limit_ms, void* stream) {
@@ -2578,11 +2650,18 @@ extern "C" {
 int gl_cartesian_dot_static(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_ap* out, uint32_t flags,
                             void* stream) {
   // validate first, so that an over-sized request is told apart from a malformed one
-  DotProblem d;
-  int rc = classify_dot(a0, w, a1, &d);
+  int rc = check_data(a0);
   if (rc) return rc;
-  const size_t need = gl_cartesian_dot_workspace(a0, w, a1, flags);
-  if (need > GL_STATIC_SCRATCH_BYTES) return GL_ERR_WORKSPACE;   // beyond the built-in scratch
+  rc = check_data(a1);
+  if (rc) return rc;
+  if (a0->dtype != GL_BF16 || a1->dtype != GL_BF16) return GL_ERR_DTYPE;
+  DotProblem d;
+  rc = classify_dot(a0, w, a1, &d);
+  if (rc) return rc;
+  // only the layout copies must fit: a contraction whose partial planes do not fit beside them runs unsplit
+  size_t required = 0, optional = 0;
+  workspace_parts(a0, w, a1, flags, &required, &optional);
+  if (required > GL_STATIC_SCRATCH_BYTES) return GL_ERR_WORKSPACE;   // beyond the built-in scratch
   void* base = nullptr;
   rc = static_scratch_address(&base);
   if (rc) return rc;

@@ -16,20 +16,26 @@ namespace gl {
 
 // Division of n < 2^31 by a divisor fixed on the host: p = ceil(log2 d), mul = ceil(2^(31+p) / d),
 // n / d = umulhi(n, mul) >> (p - 1); mul = 0 stands for d = 1.  An integer division on the device costs
-// some twenty-five instructions (over a hundred for 64-bit operands); kernels whose blocks move a few KB
-// each (im2col_rows, nchw_prepass) need several per thread.
+// some twenty-five instructions (over a hundred for 64-bit operands), and in the single-thread and
+// single-warp loops of the tensor-core kernels it is a dependent chain of about 150 cycles.
 struct FastDiv {
-  uint32_t mul, shift;
+  uint32_t d, mul, shift;
+  __host__ void set(int64_t divisor) {
+    d = static_cast<uint32_t>(divisor);
+    uint32_t pw2 = 0;
+    while ((1ull << pw2) < static_cast<uint64_t>(divisor)) ++pw2;
+    mul = pw2 ? static_cast<uint32_t>(((1ull << (31 + pw2)) + divisor - 1) / divisor) : 0u;
+    shift = pw2 ? pw2 - 1 : 0u;
+  }
+  __device__ __forceinline__ uint32_t div(uint32_t n) const { return mul ? (__umulhi(n, mul) >> shift) : n; }
+  __device__ __forceinline__ void divmod(uint32_t n, uint32_t& q, uint32_t& r) const { q = div(n); r = n - q * d; }
 };
 inline FastDiv make_fastdiv(int64_t d) {
-  uint32_t pw2 = 0;
-  while ((1ull << pw2) < static_cast<uint64_t>(d)) ++pw2;
   FastDiv fd;
-  fd.mul = pw2 ? static_cast<uint32_t>(((1ull << (31 + pw2)) + d - 1) / d) : 0u;
-  fd.shift = pw2 ? pw2 - 1 : 0u;
+  fd.set(d);
   return fd;
 }
-__device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& fd) { return fd.mul ? __umulhi(n, fd.mul) >> fd.shift : n; }
+__device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& fd) { return fd.div(n); }
 
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

@@ -706,6 +706,92 @@ __global__ void __launch_bounds__(kThreads) window_max_2d(const float* __restric
   }
 }
 
+// The same for 2-byte (bf16) planes: values are compared as floats (every bf16 value is a float, and the
+// largest of them is one of them, so nothing is rounded).
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t b) { return __uint_as_float(b << 16); }
+
+__global__ void __launch_bounds__(kThreads) window_max_2d_bf16(const uint16_t* __restrict__ in, uint16_t* __restrict__ out,
+                                                                int64_t planes, int H, int W, int Kh, int Kw, int Sh, int Sw,
+                                                                int ph, int pw, int Ho, int Wo, float fill) {
+  pdl_wait();
+  pdl_launch_dependents();
+  const int64_t total = planes * Ho * Wo;
+  for (int64_t c = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; c < total; c += (int64_t)gridDim.x * blockDim.x) {
+    const int y = static_cast<int>(c % Wo);
+    const int x = static_cast<int>((c / Wo) % Ho);
+    const uint16_t* plane = in + (c / ((int64_t)Wo * Ho)) * H * W;
+    float best = -INFINITY;
+    for (int dx = 0; dx < Kh; ++dx) {
+      const int h = x * Sh + dx - ph;
+      for (int dy = 0; dy < Kw; ++dy) {
+        const int w = y * Sw + dy - pw;
+        const bool inside = h >= 0 && h < H && w >= 0 && w < W;
+        best = fmaxf(best, inside ? bf16_bits_to_float(plane[(int64_t)h * W + w]) : fill);
+      }
+    }
+    out[c] = static_cast<uint16_t>(__float_as_uint(best) >> 16);
+  }
+}
+
+// Channels-last items: compute reduceMax (windows (access act 1) (Kh,Kw,1) (Sh,Sw,1)) on ((N),(H,W,C)), the max
+// pooling of Fig. 2c with the channel as the innermost dimension.  A thread owns one output pixel and one
+// 16-byte piece of its channels (4 floats or 8 bf16 values): every load is a full piece, consecutive threads
+// read consecutive pieces.  Border cells count as `fill`.
+struct PoolHwc {
+  int H, W, Kh, Kw, Sh, Sw, ph, pw, Ho, Wo, cv;   // cv: 16-byte pieces per pixel
+  int64_t total;                                  // N * Ho * Wo * cv
+  FastDiv by_cv, by_Wo, by_Ho;
+};
+
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads) window_max_hwc(const uint4* __restrict__ in, uint4* __restrict__ out, const PoolHwc p,
+                                                            float fill) {
+  pdl_wait();
+  pdl_launch_dependents();
+  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < p.total; e += (int64_t)gridDim.x * blockDim.x) {
+    uint32_t pix, v, row, wo, n, ho;
+    p.by_cv.divmod(static_cast<uint32_t>(e), pix, v);
+    p.by_Wo.divmod(pix, row, wo);
+    p.by_Ho.divmod(row, n, ho);
+    float best[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) best[i] = -INFINITY;
+    bool border = false;
+    for (int dy = 0; dy < p.Kh; ++dy) {
+      const int h = static_cast<int>(ho) * p.Sh + dy - p.ph;
+      for (int dx = 0; dx < p.Kw; ++dx) {
+        const int w = static_cast<int>(wo) * p.Sw + dx - p.pw;
+        if (h < 0 || h >= p.H || w < 0 || w >= p.W) { border = true; continue; }
+        const uint4 q = in[((static_cast<int64_t>(n) * p.H + h) * p.W + w) * p.cv + v];
+        const uint32_t qq[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          if (BF16) {
+            best[2 * i] = fmaxf(best[2 * i], bf16_bits_to_float(qq[i] & 0xFFFFu));
+            best[2 * i + 1] = fmaxf(best[2 * i + 1], __uint_as_float(qq[i] & 0xFFFF0000u));
+          } else {
+            best[i] = fmaxf(best[i], __uint_as_float(qq[i]));
+          }
+        }
+      }
+    }
+    if (border) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) best[i] = fmaxf(best[i], fill);
+    }
+    uint4 r;
+    if (BF16) {
+      r.x = (__float_as_uint(best[0]) >> 16) | (__float_as_uint(best[1]) & 0xFFFF0000u);
+      r.y = (__float_as_uint(best[2]) >> 16) | (__float_as_uint(best[3]) & 0xFFFF0000u);
+      r.z = (__float_as_uint(best[4]) >> 16) | (__float_as_uint(best[5]) & 0xFFFF0000u);
+      r.w = (__float_as_uint(best[6]) >> 16) | (__float_as_uint(best[7]) & 0xFFFF0000u);
+    } else {
+      r = make_uint4(__float_as_uint(best[0]), __float_as_uint(best[1]), __float_as_uint(best[2]), __float_as_uint(best[3]));
+    }
+    out[e] = r;
+  }
+}
+
 // 2D windows + reduceMax, tiled: one block owns TH output rows of one plane.  It
 // stages the (TH-1)*Sh+Kh input rows it needs (border cells hold the fill value)
 // with 128-bit loads, then every thread reduces whole windows out of shared
@@ -1133,7 +1219,7 @@ int gl_compute_reduce_max(const gl_ap* in, const gl_windows* w, gl_ap* out, void
   int rc = check_data(in);
   if (rc) return rc;
   if (!out) return GL_ERR_NULL;
-  if (in->dtype != GL_F32) return GL_ERR_DTYPE;
+  if (in->dtype != GL_F32 && in->dtype != GL_BF16) return GL_ERR_DTYPE;
   gl_ap want = *in;
   rc = gl_shape_reduce_max(in, w, &want);
   if (rc) return rc;
@@ -1144,6 +1230,52 @@ int gl_compute_reduce_max(const gl_ap* in, const gl_windows* w, gl_ap* out, void
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const float* src = static_cast<const float*>(in->data);
   float* dst = static_cast<float*>(out->data);
+  const bool bf16 = in->dtype == GL_BF16;
+  if (w) {
+    // channels-last items (H,W,C) with window (Kh,Kw,1), stride (Sh,Sw,1), no pad on C: 16-byte channel pieces
+    const int nc = in->access_ndim;
+    const int64_t per_piece = bf16 ? 8 : 4;
+    if (w->n == 3 && w->wshape[2] == 1 && w->stride[2] == 1 && w->pad_lo[2] == 0 && w->pad_hi[2] == 0 &&
+        in->shape[nc + 2] % per_piece == 0 && in->shape[nc] < (1 << 20) && in->shape[nc + 1] < (1 << 20)) {
+      gl_ap A = *in;
+      gl_shape_windows(in, w, &A);
+      PoolHwc t;
+      t.H = (int)in->shape[nc]; t.W = (int)in->shape[nc + 1];
+      t.Kh = (int)w->wshape[0]; t.Kw = (int)w->wshape[1];
+      t.Sh = (int)w->stride[0]; t.Sw = (int)w->stride[1];
+      t.ph = (int)w->pad_lo[0]; t.pw = (int)w->pad_lo[1];
+      t.Ho = (int)A.shape[nc]; t.Wo = (int)A.shape[nc + 1];
+      t.cv = (int)(in->shape[nc + 2] / per_piece);
+      t.total = prod(in->shape, 0, nc) * t.Ho * t.Wo * t.cv;
+      if (t.total < (1ll << 31)) {
+        t.by_cv = make_fastdiv(t.cv);
+        t.by_Wo = make_fastdiv(t.Wo);
+        t.by_Ho = make_fastdiv(t.Ho);
+        const float fill = w->pad_kind == GL_PAD_NEG_INF ? -INFINITY : 0.0f;
+        const dim3 grid(grid_for(t.total, kThreads));
+        const cudaError_t err =
+            bf16 ? launch_pdl(window_max_hwc<true>, grid, dim3(kThreads), 0, st, 1, static_cast<const uint4*>(in->data),
+                              static_cast<uint4*>(out->data), t, fill)
+                 : launch_pdl(window_max_hwc<false>, grid, dim3(kThreads), 0, st, 1, static_cast<const uint4*>(in->data),
+                              static_cast<uint4*>(out->data), t, fill);
+        return err == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+      }
+    }
+  }
+  if (bf16) {
+    // 2-byte planes ((..),(H,W)): the plain kernel; other bf16 forms have no kernel
+    const int nb = in->access_ndim;
+    if (!w || w->n != 2 || in->shape[nb] >= (1 << 30) || in->shape[nb + 1] >= (1 << 30)) return GL_ERR_UNSUPPORTED;
+    gl_ap A = *in;
+    gl_shape_windows(in, w, &A);
+    const float fill = w->pad_kind == GL_PAD_NEG_INF ? -INFINITY : 0.0f;
+    const int64_t nwin = numel(want);
+    return launch_pdl(window_max_2d_bf16, dim3(grid_for(nwin, kThreads)), dim3(kThreads), 0, st, 1,
+                      static_cast<const uint16_t*>(in->data), static_cast<uint16_t*>(out->data), prod(in->shape, 0, nb),
+                      (int)in->shape[nb], (int)in->shape[nb + 1], (int)w->wshape[0], (int)w->wshape[1], (int)w->stride[0],
+                      (int)w->stride[1], (int)w->pad_lo[0], (int)w->pad_lo[1], (int)A.shape[nb], (int)A.shape[nb + 1],
+                      fill) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+  }
   if (!w) {
     const int64_t items = prod(in->shape, 0, in->access_ndim), item = prod(in->shape, in->access_ndim, in->ndim);
     item_max<<<grid_for(items, kThreads / 32), kThreads, 0, st>>>(src, dst, items, item);

@@ -97,6 +97,67 @@ def build_call(cfg, layout: str, device, batch=None, flags=0):
     return gl.prepare_compute_reduce_max(gl.AccessPattern(x, 2), spec, out), 0.0, cfg.algorithmic_bytes
 
 
+def build_chain(cfg, layout: str, device, seed=None):
+    """The program of `synth.ChainCase` as a list of prepared calls plus the access pattern of its result.
+
+    layout "nhwc": items (H,W,C), layer results stored as bf16 rows [pixels, channels] (GL_OUT_BF16) which are the
+    next layer's items as they stand.  layout "nchw": the paper's (C,H,W) items, every convolution followed by the
+    squeeze + transpose of Fig. 2a (GL_OUT_NCHW).  The dense weights are laid out to match the flatten order of the
+    layout, so both layouts compute the same numbers."""
+    x, w1, w2, wd = cfg.inputs(synth.config_seed(5) if seed is None else seed)
+    (h1, wd1), (h2, wd2), (h3, wd3) = cfg.dims()
+    n, c1, c2, k2 = cfg.n, cfg.c1, cfg.c2, cfg.pool2
+    relu_bf16 = gl.GL_EPILOGUE_RELU | gl.GL_OUT_BF16
+    steps = []
+
+    def conv(xa, spec, wa, out_shape, flags):
+        out = gl.AccessPattern(torch.empty(out_shape, dtype=torch.bfloat16, device=device), len(out_shape))
+        need = gl.gl_cartesian_dot_workspace(xa, spec, wa, flags)
+        ws = torch.empty(need + 1024, dtype=torch.uint8, device=device) if need else None
+        steps.append(gl.prepare_cartesian_dot(xa, spec, wa, out, flags, ws))
+        return out
+
+    def pool(a, spec, out_shape, na):
+        out = gl.AccessPattern(torch.empty(out_shape, dtype=torch.bfloat16, device=device), na)
+        steps.append(gl.prepare_compute_reduce_max(a, spec, out))
+        return out
+
+    if layout == "nhwc":
+        t = lambda a: np.ascontiguousarray(a.transpose(0, 2, 3, 1))
+        xa = gl.AccessPattern(_bf16(t(x), device), 1)
+        y1 = conv(xa, gl.windows_spec((7, 7, 3), (2, 2, 1), (3, 3, 0), (3, 3, 0)), gl.AccessPattern(_bf16(t(w1), device), 1),
+                  (n, h1, wd1, 1, c1), relu_bf16)
+        p1 = pool(gl.AccessPattern(y1.tensor.view(n, h1, wd1, c1), 1),
+                  gl.windows_spec((3, 3, 1), (2, 2, 1), (1, 1, 0), (1, 1, 0), gl.GL_PAD_NEG_INF), (n, h2, wd2, c1), 4)
+        y2 = conv(gl.AccessPattern(p1.tensor, 1), gl.windows_spec((3, 3, c1), (1, 1, 1), (1, 1, 0), (1, 1, 0)),
+                  gl.AccessPattern(_bf16(t(w2), device), 1), (n, h2, wd2, 1, c2), relu_bf16)
+        p2 = pool(gl.AccessPattern(y2.tensor.view(n, h2, wd2, c2), 1), gl.windows_spec((k2, k2, 1), (k2, k2, 1)),
+                  (n, h3, wd3, c2), 4)
+        feat = gl.AccessPattern(p2.tensor.view(n, h3 * wd3 * c2), 1)                 # flatten: metadata
+        wdense = gl.AccessPattern(_bf16(t(wd).reshape(cfg.units, -1), device), 1)
+    else:
+        xa = gl.AccessPattern(_bf16(x, device), 1)
+        nchw = relu_bf16 | gl.GL_OUT_NCHW
+        y1 = conv(xa, gl.windows_spec((3, 7, 7), (1, 2, 2), (0, 3, 3), (0, 3, 3)), gl.AccessPattern(_bf16(w1, device), 1),
+                  (n, c1, h1, wd1), nchw)
+        p1 = pool(gl.AccessPattern(y1.tensor, 2), gl.windows_spec((3, 3), (2, 2), (1, 1), (1, 1), gl.GL_PAD_NEG_INF),
+                  (n, c1, h2, wd2), 4)
+        y2 = conv(gl.AccessPattern(p1.tensor, 1), gl.windows_spec((c1, 3, 3), (1, 1, 1), (0, 1, 1), (0, 1, 1)),
+                  gl.AccessPattern(_bf16(w2, device), 1), (n, c2, h2, wd2), nchw)
+        p2 = pool(gl.AccessPattern(y2.tensor, 2), gl.windows_spec((k2, k2), (k2, k2)), (n, c2, h3, wd3), 4)
+        feat = gl.AccessPattern(p2.tensor.view(n, c2 * h3 * wd3), 1)
+        wdense = gl.AccessPattern(_bf16(wd.reshape(cfg.units, -1), device), 1)
+    logits = gl.AccessPattern(torch.empty((n, cfg.units), dtype=torch.float32, device=device), 2)
+    need = gl.gl_cartesian_dot_workspace(feat, None, wdense, 0)
+    ws = torch.empty(need + 1024, dtype=torch.uint8, device=device) if need else None
+    steps.append(gl.prepare_cartesian_dot(feat, None, wdense, logits, 0, ws))
+
+    def run(stream=None):
+        for step in steps:
+            step(stream)
+    return run, logits, len(steps)
+
+
 def main():
     table = workloads()
     ap = argparse.ArgumentParser()

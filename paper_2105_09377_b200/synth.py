@@ -214,5 +214,60 @@ MEM_PAD = MemCase("pad_w1_32x64x56x56", "pad", (32, 64, 56, 56), pad=1)
 MEM_MAXPOOL = MemCase("maxpool3x3s2p1_32x64x112x112", "maxpool", (32, 64, 112, 112), (3, 3), 2, 1)
 
 
+@dataclass(frozen=True)
+class ChainCase:
+    """The kernels of Fig. 2 composed into one program at the scale of a ResNet stem:
+    conv 7x7 stride 2 pad 3 (3 -> c1) + relu, max pool 3x3 stride 2 pad 1, conv 3x3 pad 1 (c1 -> c2) + relu,
+    max pool `pool2` x `pool2` with that stride, flatten per image, dense layer to `units` outputs.
+    Layer results are stored as bf16 (the next layer's operand type); the dense layer's result is fp32."""
+    name: str
+    n: int
+    h: int
+    w: int
+    c1: int
+    c2: int
+    pool2: int
+    units: int
+    integer: bool = False
+
+    def dims(self):
+        h1, w1 = (self.h + 6 - 7) // 2 + 1, (self.w + 6 - 7) // 2 + 1          # conv 7x7 s2 p3
+        h2, w2 = (h1 + 2 - 3) // 2 + 1, (w1 + 2 - 3) // 2 + 1                  # pool 3x3 s2 p1
+        h3, w3 = (h2 - self.pool2) // self.pool2 + 1, (w2 - self.pool2) // self.pool2 + 1
+        return (h1, w1), (h2, w2), (h3, w3)
+
+    @property
+    def features(self):
+        return self.c2 * self.dims()[2][0] * self.dims()[2][1]
+
+    @property
+    def flops(self):
+        (h1, w1), (h2, w2), _ = self.dims()
+        return 2.0 * self.n * (h1 * w1 * self.c1 * 147 + h2 * w2 * self.c2 * 9 * self.c1 + self.units * self.features)
+
+    @property
+    def algorithmic_bytes(self):
+        """Every layer reads its operands once and writes its result once (bf16 between layers, fp32 at the end)."""
+        (h1, w1), (h2, w2), (h3, w3) = self.dims()
+        acts = (self.h * self.w * 3, h1 * w1 * self.c1, h2 * w2 * self.c1, h2 * w2 * self.c2, h3 * w3 * self.c2)
+        moved = acts[0] + 2 * sum(acts[1:])                       # each intermediate written once and read once
+        weights = self.c1 * 147 + self.c2 * 9 * self.c1 + self.units * self.features
+        return 2 * (self.n * moved + weights) + 4 * self.n * self.units
+
+    def inputs(self, seed: int):
+        """(image NCHW, conv1 weights, conv2 weights, dense weights [units, (c2, h3, w3)]) as float32 arrays of
+        bf16 values.  The integer variant draws from {-1, 0, 1}: every layer's sums are then exact in fp32."""
+        (h3, w3) = self.dims()[2]
+        shapes = ((self.n, 3, self.h, self.w), (self.c1, 3, 7, 7), (self.c2, self.c1, 3, 3), (self.units, self.c2, h3, w3))
+        if self.integer:
+            return tuple(uniform_int(seed, i + 1, shp, -1, 1) for i, shp in enumerate(shapes))
+        fan = (1.0, 147.0, 9.0 * self.c1, float(self.features))
+        return tuple(bf16_round(normal(seed, i + 1, shp, 1.0 if i == 0 else math.sqrt(2.0 / fan[i])))
+                     for i, shp in enumerate(shapes))
+
+
+CHAIN_STEM = ChainCase("chain_stem_32x224x224", 32, 224, 224, 64, 64, 8, 1000)
+
+
 def config_seed(config_index: int) -> int:
     return BASE_SEED + config_index

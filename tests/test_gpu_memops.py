@@ -162,6 +162,48 @@ def test_windows_reduce_max(gl, shape, na, wshape, stride, lo, hi):
     _same_bits(out.tensor, ref.data.astype(np.float32))
 
 
+POOL_HWC_CASES = [
+    # n, h, w, c, (kh, kw), (sh, sw), (ph, pw)
+    (2, 9, 8, 8, (3, 3), (2, 2), (1, 1)),
+    (3, 12, 10, 16, (2, 3), (1, 2), (0, 1)),
+    (1, 16, 16, 64, (8, 8), (8, 8), (0, 0)),
+    (2, 7, 5, 24, (3, 3), (1, 1), (1, 1)),
+]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("n,h,w,c,k,s,pd", POOL_HWC_CASES)
+def test_channels_last_max_pool(gl, n, h, w, c, k, s, pd, dtype):
+    # ((N),(H,W,C)) items, window (Kh,Kw,1): the pooling of Fig. 2c with channels innermost, against the
+    # brute-force pooling of the (C,H,W) view
+    x = synth.uniform(12, 1, (n, h, w, c), -1.0, 1.0) - 2.0
+    if dtype == "bf16":
+        x = synth.bf16_round(x)
+    ref = brute.maxpool(np.ascontiguousarray(x.transpose(0, 3, 1, 2)), k, s, ((pd[0], pd[0]), (pd[1], pd[1]))).transpose(0, 2, 3, 1)
+    dev = to_bf16_device(x) if dtype == "bf16" else to_f32_device(x)
+    spec = gl.windows_spec((k[0], k[1], 1), (s[0], s[1], 1), (pd[0], pd[1], 0), (pd[0], pd[1], 0), gl.GL_PAD_NEG_INF)
+    out = gl.gl_compute_reduce_max(gl.AccessPattern(dev, 1), spec)
+    assert out.shape == ((n,) + ref.shape[1:], ())
+    assert np.array_equal(out.tensor.float().cpu().numpy(), ref)
+    # the interpreter's windows + reduceMax on the same items
+    a = gi.access(x, 1)
+    for i, l in enumerate(pd):
+        if l:
+            a = gi.pad(a, 1 + i, l, l, "neg_inf")
+    prog = gi.compute("reduceMax", gi.windows(a, (k[0], k[1], 1), (s[0], s[1], 1)))
+    assert np.array_equal(prog.data.astype(np.float32), ref)
+
+
+@pytest.mark.parametrize("shape,k,s,pd", [((2, 3, 9, 8), (3, 3), (2, 2), (1, 1)), ((1, 5, 16, 24), (8, 8), (8, 8), (0, 0)),
+                                          ((3, 2, 7, 11), (2, 3), (1, 2), (0, 1))])
+def test_bf16_plane_max_pool(gl, shape, k, s, pd):
+    x = synth.bf16_round(synth.uniform(13, 1, shape, -1.0, 1.0) - 2.0)
+    ref = brute.maxpool(x, k, s, ((pd[0], pd[0]), (pd[1], pd[1])))
+    out = gl.gl_compute_reduce_max(gl.AccessPattern(to_bf16_device(x), 2), gl.windows_spec(k, s, pd, pd, gl.GL_PAD_NEG_INF))
+    assert tuple(out.tensor.shape) == ref.shape and out.tensor.dtype == torch.bfloat16
+    assert np.array_equal(out.tensor.float().cpu().numpy(), ref)
+
+
 def test_reduce_max_whole_items(gl):
     x = synth.uniform(11, 1, (7, 5, 33), -1.0, 1.0)
     ref = gi.compute("reduceMax", gi.access(x, 1))
