@@ -10,7 +10,11 @@ work of all ranks over the slowest rank's time.
 
 `--impl reference` times the CPU checker (oracle/) on a bounded sample of the
 same workload instead.  `--detail` (default at one GPU) adds per-workload
-timings of the convolution sweeps and the memory-bound access operators.
+timings of the convolution sweeps, the composed stem-scale chain and the
+memory-bound access operators, as compact rows at the end of the line:
+[workload, layout, us per call, TFLOP/s, GB/s (algorithmic), fraction of the
+binding roofline].  `--gpus N` without a launcher (no WORLD_SIZE in the
+environment) starts the N replica processes itself.
 """
 from __future__ import annotations
 
@@ -43,6 +47,21 @@ def load_peaks():
 # --------------------------------------------------------------------------
 # multi-process plumbing (replicas; no data-path collective)
 # --------------------------------------------------------------------------
+
+def spawn_replicas(n: int, argv) -> int:
+    """`--gpus N` run plainly: start N replica processes (one per GPU, rendezvous on 127.0.0.1) and wait for them.
+    Rank 0 prints the JSON line."""
+    import socket
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    procs = []
+    for rank in range(n):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + list(argv), env=env))
+    return max(p.wait() for p in procs)
+
 
 def dist_env():
     return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
@@ -231,12 +250,51 @@ def time_graph(calls, iters: int, device):
     return statistics.median(times), min(times)
 
 
+def host_us_per_call(call, iters: int = 300) -> float:
+    """Host time of one plain library call (argument checks, planning, tensor maps, launch), with the device kept
+    idle enough that the launch queue never fills: the cost a caller pays without CUDA graphs."""
+    import torch
+    for _ in range(20):
+        call()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(iters):
+        call()
+        if i % 50 == 49:
+            torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    torch.cuda.synchronize()
+    return dt / iters * 1e6
+
+
 def detail_workloads(device, peaks):
     """Per-workload timings of the other configurations (not the headline value)."""
     import torch
     from paper_2105_09377_b200 import run_workload as rw
     from paper_2105_09377_b200 import synth
     out = []
+
+    def chain_entry(layout):
+        cfg = synth.CHAIN_STEM
+        nsets = 3
+        runs = [rw.build_chain(cfg, layout, device)[0] for _ in range(nsets)]
+        med, best = time_graph(runs, 20, device)
+        # roofline time of the chain: the sum of its layers' binding-roofline times
+        (h1, w1), (h2, w2), (h3, w3) = cfg.dims()
+        n = cfg.n
+        layers = [  # (flops, bytes)
+            (2.0 * n * h1 * w1 * cfg.c1 * 147, 2 * n * (cfg.h * cfg.w * 3 + h1 * w1 * cfg.c1)),
+            (0.0, 2 * n * cfg.c1 * (h1 * w1 + h2 * w2)),
+            (2.0 * n * h2 * w2 * cfg.c2 * 9 * cfg.c1, 2 * n * h2 * w2 * (cfg.c1 + cfg.c2)),
+            (0.0, 2 * n * cfg.c2 * (h2 * w2 + h3 * w3)),
+            (2.0 * n * cfg.units * cfg.features, 2 * (n + cfg.units) * cfg.features + 4 * n * cfg.units),
+        ]
+        t_roof = sum(max(f / (peaks["bf16_tflops"] * 1e12), b / (peaks["hbm_gbs"] * 1e9)) for f, b in layers)
+        out.append({"workload": cfg.name, "layout": layout + ", 5 calls", "us": med * 1e6, "us_best": best * 1e6,
+                    "tflops": cfg.flops / med / 1e12, "gbs": cfg.algorithmic_bytes / med / 1e9,
+                    "frac_binding_roof": t_roof / med, "buffer_sets": nsets})
+        del runs
+        torch.cuda.empty_cache()
 
     def entry(cfg, layout, bf16_out=False):
         from paper_2105_09377_b200 import binding as gl
@@ -266,9 +324,29 @@ def detail_workloads(device, peaks):
     entry(synth.CONV_SWEEP_3X3[0], "rewritten")   # the materialised im2col form of Section 5.3, for comparison
     for cfg in (synth.CONV_SWEEP_3X3[0], synth.CONV_STRIDED_1X1[0], synth.CONV_STRIDED_1X1[1]):
         entry(cfg, "nhwc", bf16_out=True)         # the two bandwidth-bound shapes with bf16 results
+    for layout in ("nhwc", "nchw"):
+        chain_entry(layout)                       # Fig. 2a + relu + Fig. 2c + Fig. 2b composed, per item layout
     for cfg in (synth.MEM_IM2COL, synth.MEM_TRANSPOSE, synth.MEM_MAXPOOL, synth.MEM_RELU, synth.MEM_PAD):
         entry(cfg, "")
+    # host cost of a plain call (no CUDA graph) on a small convolution: planning, tensor maps (cached per
+    # argument list after the first call) and the launch
+    from paper_2105_09377_b200 import binding as gl
+    small = synth.ConvCase("conv3x3_14x14x256_n1", 1, 256, 14, 14, 256, 3, 3, 1, 1)
+    call, _, _ = rw.build_call(small, "nhwc", device)
+    out.append({"workload": "host_us_per_plain_call", "layout": "conv3x3 14x14x256, one image, channels-last",
+                "us": host_us_per_call(call)})
     return out
+
+
+def compact_rows(detail):
+    """[workload, layout, us, TFLOP/s or None, GB/s or None, fraction of the binding roofline or of the copy rate]"""
+    def r(v, nd):
+        return None if v is None else round(v, nd)
+    rows = []
+    for e in detail:
+        frac = e.get("frac_binding_roof", e.get("frac_hbm_peak"))
+        rows.append([e["workload"], e.get("layout", ""), r(e["us"], 2), r(e.get("tflops"), 1), r(e.get("gbs"), 0), r(frac, 3)])
+    return rows
 
 
 def run_gpu(args):
@@ -374,18 +452,49 @@ def run_gpu(args):
     barrier()
     e2e_seconds = max_over_ranks(e0.elapsed_time(e1) * 1e-3, device)
 
+    # a second, long leg (outside the headline's timed region): about a second of back-to-back launches, the
+    # regime of the sustained tensor peak (power cap active, clocks below their maximum)
+    sustained = None
+    if world == 1 and args.sustained_seconds > 0:
+        per = max(seconds / args.steps, 1e-6)
+        n_long = int(max(200, min(50000, args.sustained_seconds / per)))
+        sampler2 = ClockSampler(local_rank)
+        sampler2.start()
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(n_long):
+            calls[i % nsets]()
+        e1.record()
+        torch.cuda.synchronize()
+        clk2 = sampler2.stop()
+        s_long = e0.elapsed_time(e1) * 1e-3
+        ach = case.flops * n_long / s_long / 1e12
+        sustained = {"achieved": ach, "peak": peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]), "unit": "TFLOP/s",
+                     "frac": ach / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]), "launches": n_long,
+                     "seconds": s_long, "sm_mhz": clk2.get("sm_mhz"), "reasons": clk2.get("reasons")}
+
     if rank != 0:
         return 0
 
     value = aggregate_value(case.flops * args.steps, world, seconds_max) / 1e12
     kernel_s = seconds / args.steps
     achieved = case.flops / kernel_s / 1e12
-    traffic = None
+    # DRAM bytes per launch from the committed ncu capture of this kernel; the file names the kernel source it was
+    # taken on (a hash of csrc/gl_dot.cu), and the figure is dropped once the kernel has changed since
+    traffic, traffic_source = None, None
     tpath = os.path.join(ROOT, "profiles", "dense_4096_dram_bytes_per_launch.txt")
     if os.path.exists(tpath):
         try:
-            traffic = float(open(tpath).read().split()[0])
-        except (ValueError, IndexError):
+            fields = open(tpath).read().split()
+            import hashlib
+            src = os.path.join(ROOT, "paper_2105_09377_b200", "csrc", "gl_dot.cu")
+            now = hashlib.sha256(open(src, "rb").read()).hexdigest()[:16]
+            if len(fields) >= 2 and fields[1] == now:
+                traffic = float(fields[0])
+                traffic_source = "profiles/dense_4096_dram_bytes_per_launch.txt (ncu, kernel source %s)" % now
+            else:
+                traffic_source = "none: the kernel source changed since the committed ncu capture"
+        except (ValueError, IndexError, OSError):
             traffic = None
     long_region = seconds > 1.0
     peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]) if long_region else peaks["bf16_tflops"]
@@ -397,12 +506,12 @@ def run_gpu(args):
                    "output": "fp32", "epilogue": "relu fused", "parallelism": "replicas x%d" % world,
                    "l2": "rotating over %d buffer sets (%.0f MB) > L2" % (nsets, nsets * bytes_per_set / 1e6)},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                     "frac": achieved / peak, "traffic": traffic,
+                     "frac": achieved / peak, "traffic": traffic, "traffic_source": traffic_source,
                      "peak_source": "%s (%s)" % (peaks_kind, "sustained: timed region > 1 s" if long_region else "burst"),
                      "frac_of_burst": achieved / peaks["bf16_tflops"],
                      "frac_of_sustained": achieved / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
                      "frac_of_nominal_2250": achieved / 2250.0, "kernel": "dot_tc (dense)",
-                     "kernel_us": kernel_s * 1e6},
+                     "kernel_us": kernel_s * 1e6, "sustained": sustained},
         "e2e": {"value": aggregate_value(case.flops * e2e_steps, world, e2e_seconds) / 1e12, "unit": "TFLOP/s",
                 "h2d_bytes_per_step": a_pin.numel() * 2 + b_pin.numel() * 2, "d2h_bytes_per_step": o_pin[0].numel() * 4,
                 "pipelining": "2 buffer sets; copy-in, kernel and copy-out on 3 streams",
@@ -412,7 +521,8 @@ def run_gpu(args):
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline_dense(args.cpu_seconds)
     if world == 1 and args.detail:
-        line["detail"] = detail_workloads(device, peaks)
+        line["detail_columns"] = ["workload", "layout", "us", "TFLOP/s", "GB/s (algorithmic)", "fraction of binding roofline"]
+        line["detail"] = compact_rows(detail_workloads(device, peaks))
     print(json.dumps(line))
     return 0
 
@@ -427,9 +537,13 @@ def main():
     ap.add_argument("--no-detail", dest="detail", action="store_false")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--sustained-seconds", type=float, default=1.0,
+                    help="length of the second, sustained-regime leg (0: skip it)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return spawn_replicas(args.gpus, sys.argv[1:])
     return run_gpu(args)
 
 

@@ -36,3 +36,18 @@ def test_single_process_helpers():
     assert bench.aggregate_value(8.0, 4, 2.0) == 16.0
     peaks, kind = bench.load_peaks()
     assert peaks["hbm_gbs"] > 1000 and kind in ("measured", "fallback")
+
+
+def test_gpus_flag_without_a_launcher_starts_the_replicas():
+    # `bench.py --gpus N` run plainly starts N ranks itself; here through the reference arm, which needs no GPU:
+    # rank 0 prints the one JSON line, the other rank exits quietly
+    import json
+    import subprocess
+    code = ("import sys; sys.path.insert(0, %r); import bench; "
+            "sys.exit(bench.spawn_replicas(2, ['--impl', 'reference', '--steps', '1', '--warmup', '0', '--gpus', '2']))" % ROOT)
+    done = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=300)
+    assert done.returncode == 0, done.stderr
+    lines = [ln for ln in done.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
