@@ -739,39 +739,50 @@ __global__ void __launch_bounds__(kThreads) window_max_2d_bf16(const uint16_t* _
 // read consecutive pieces.  Border cells count as `fill`.
 struct PoolHwc {
   int H, W, Kh, Kw, Sh, Sw, ph, pw, Ho, Wo, cv;   // cv: 16-byte pieces per pixel
-  int64_t total;                                  // N * Ho * Wo * cv
-  FastDiv by_cv, by_Wo, by_Ho;
+  int split_log2;                                 // 2^split_log2 neighbouring lanes share one output piece
+  int64_t total;                                  // N * Ho * Wo * cv << split_log2
+  FastDiv by_cv, by_Wo, by_Ho, by_Kw;
 };
 
+// Large windows over few outputs (a pooling layer that ends a network) would leave most of the machine idle with
+// one thread per output piece, so 2^split_log2 neighbouring lanes share a piece: lane j takes the window cells
+// j, j + 2^split_log2, ... and the lanes' maxima are combined by shuffles.
 template <bool BF16>
 __global__ void __launch_bounds__(kThreads) window_max_hwc(const uint4* __restrict__ in, uint4* __restrict__ out, const PoolHwc p,
                                                             float fill) {
   pdl_wait();
   pdl_launch_dependents();
-  for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < p.total; e += (int64_t)gridDim.x * blockDim.x) {
+  const int split = 1 << p.split_log2, taps = p.Kh * p.Kw;
+  // all threads of a warp take part in the shuffles: the loop bound is rounded up to whole blocks
+  const int64_t total_r = (p.total + blockDim.x - 1) / blockDim.x * blockDim.x;
+  for (int64_t e0 = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e0 < total_r; e0 += (int64_t)gridDim.x * blockDim.x) {
+    const bool live = e0 < p.total;
+    const uint32_t e = static_cast<uint32_t>(live ? e0 : 0) >> p.split_log2, part = static_cast<uint32_t>(e0) & (split - 1);
     uint32_t pix, v, row, wo, n, ho;
-    p.by_cv.divmod(static_cast<uint32_t>(e), pix, v);
+    p.by_cv.divmod(e, pix, v);
     p.by_Wo.divmod(pix, row, wo);
     p.by_Ho.divmod(row, n, ho);
     float best[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) best[i] = -INFINITY;
     bool border = false;
-    for (int dy = 0; dy < p.Kh; ++dy) {
-      const int h = static_cast<int>(ho) * p.Sh + dy - p.ph;
-      for (int dx = 0; dx < p.Kw; ++dx) {
-        const int w = static_cast<int>(wo) * p.Sw + dx - p.pw;
-        if (h < 0 || h >= p.H || w < 0 || w >= p.W) { border = true; continue; }
-        const uint4 q = in[((static_cast<int64_t>(n) * p.H + h) * p.W + w) * p.cv + v];
-        const uint32_t qq[4] = {q.x, q.y, q.z, q.w};
+    const uint4* img = in + static_cast<int64_t>(n) * p.H * p.W * p.cv + v;
+#pragma unroll 4
+    for (int t = part; t < taps; t += split) {
+      uint32_t dy, dx;
+      p.by_Kw.divmod(static_cast<uint32_t>(t), dy, dx);
+      const int h = static_cast<int>(ho) * p.Sh + static_cast<int>(dy) - p.ph;
+      const int w = static_cast<int>(wo) * p.Sw + static_cast<int>(dx) - p.pw;
+      if (h < 0 || h >= p.H || w < 0 || w >= p.W) { border = true; continue; }
+      const uint4 q = img[(static_cast<int64_t>(h) * p.W + w) * p.cv];
+      const uint32_t qq[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          if (BF16) {
-            best[2 * i] = fmaxf(best[2 * i], bf16_bits_to_float(qq[i] & 0xFFFFu));
-            best[2 * i + 1] = fmaxf(best[2 * i + 1], __uint_as_float(qq[i] & 0xFFFF0000u));
-          } else {
-            best[i] = fmaxf(best[i], __uint_as_float(qq[i]));
-          }
+      for (int i = 0; i < 4; ++i) {
+        if (BF16) {
+          best[2 * i] = fmaxf(best[2 * i], bf16_bits_to_float(qq[i] & 0xFFFFu));
+          best[2 * i + 1] = fmaxf(best[2 * i + 1], __uint_as_float(qq[i] & 0xFFFF0000u));
+        } else {
+          best[i] = fmaxf(best[i], __uint_as_float(qq[i]));
         }
       }
     }
@@ -779,16 +790,22 @@ __global__ void __launch_bounds__(kThreads) window_max_hwc(const uint4* __restri
 #pragma unroll
       for (int i = 0; i < 8; ++i) best[i] = fmaxf(best[i], fill);
     }
-    uint4 r;
-    if (BF16) {
-      r.x = (__float_as_uint(best[0]) >> 16) | (__float_as_uint(best[1]) & 0xFFFF0000u);
-      r.y = (__float_as_uint(best[2]) >> 16) | (__float_as_uint(best[3]) & 0xFFFF0000u);
-      r.z = (__float_as_uint(best[4]) >> 16) | (__float_as_uint(best[5]) & 0xFFFF0000u);
-      r.w = (__float_as_uint(best[6]) >> 16) | (__float_as_uint(best[7]) & 0xFFFF0000u);
-    } else {
-      r = make_uint4(__float_as_uint(best[0]), __float_as_uint(best[1]), __float_as_uint(best[2]), __float_as_uint(best[3]));
+    for (int d = 1; d < split; d <<= 1) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) best[i] = fmaxf(best[i], __shfl_xor_sync(0xffffffffu, best[i], d));
     }
-    out[e] = r;
+    if (live && part == 0) {
+      uint4 r;
+      if (BF16) {
+        r.x = (__float_as_uint(best[0]) >> 16) | (__float_as_uint(best[1]) & 0xFFFF0000u);
+        r.y = (__float_as_uint(best[2]) >> 16) | (__float_as_uint(best[3]) & 0xFFFF0000u);
+        r.z = (__float_as_uint(best[4]) >> 16) | (__float_as_uint(best[5]) & 0xFFFF0000u);
+        r.w = (__float_as_uint(best[6]) >> 16) | (__float_as_uint(best[7]) & 0xFFFF0000u);
+      } else {
+        r = make_uint4(__float_as_uint(best[0]), __float_as_uint(best[1]), __float_as_uint(best[2]), __float_as_uint(best[3]));
+      }
+      out[e] = r;
+    }
   }
 }
 
@@ -804,16 +821,25 @@ struct PoolTile {
   int vec;       // rows are 16-byte multiples: float4 loads
 };
 
-__global__ void __launch_bounds__(kThreads) window_max_2d_tiled(const float* __restrict__ in, float* __restrict__ out,
+// T: float, or uint16_t for bf16 planes (staged and compared as floats; the largest value is one of the inputs, so
+// storing its upper 16 bits rounds nothing).  `vec` rows are read as 16-byte pieces: 4 floats or 8 bf16 values.
+__device__ __forceinline__ float pool_load(const float* p) { return *p; }
+__device__ __forceinline__ float pool_load(const uint16_t* p) { return bf16_bits_to_float(*p); }
+__device__ __forceinline__ void pool_store(float* p, float v) { *p = v; }
+__device__ __forceinline__ void pool_store(uint16_t* p, float v) { *p = static_cast<uint16_t>(__float_as_uint(v) >> 16); }
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads) window_max_2d_tiled(const T* __restrict__ in, T* __restrict__ out,
                                                                  const PoolTile p, float fill) {
   extern __shared__ __align__(16) float pool_stage[];
+  constexpr int kPer = 16 / static_cast<int>(sizeof(T));   // elements per 16-byte piece
   const int64_t plane = blockIdx.x / p.tiles;
   const int tile = blockIdx.x % p.tiles;
   const int y0 = tile * p.TH;
   const int th = min(p.TH, p.Ho - y0);
   const int rows = (th - 1) * p.Sh + p.Kh;
   const int h0 = y0 * p.Sh - p.ph;
-  const float* src = in + plane * p.H * p.W;
+  const T* src = in + plane * p.H * p.W;
   // left and right border columns, then the rows themselves
   const int right = p.Wp - p.pw - p.W;
   for (int e = threadIdx.x; e < rows * (p.pw + right); e += blockDim.x) {
@@ -821,32 +847,60 @@ __global__ void __launch_bounds__(kThreads) window_max_2d_tiled(const float* __r
     pool_stage[r * p.Wp + (j < p.pw ? j : p.W + j)] = fill;
   }
   if (p.vec) {
-    const int w4 = p.W >> 2;
-    for (int e = threadIdx.x; e < rows * w4; e += blockDim.x) {
-      const int r = e / w4, x = (e - r * w4) << 2;
+    const int wv = p.W / kPer;
+    for (int e = threadIdx.x; e < rows * wv; e += blockDim.x) {
+      const int r = e / wv, x = (e - r * wv) * kPer;
       const int h = h0 + r;
-      float4 v = make_float4(fill, fill, fill, fill);
-      if (h >= 0 && h < p.H) v = *reinterpret_cast<const float4*>(src + (int64_t)h * p.W + x);
       float* d = pool_stage + r * p.Wp + p.pw + x;
-      d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+      if (h >= 0 && h < p.H) {
+        const uint4 q = *reinterpret_cast<const uint4*>(src + (int64_t)h * p.W + x);
+        const uint32_t qq[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          if (kPer == 4) d[i] = __uint_as_float(qq[i]);
+          else { d[2 * i] = bf16_bits_to_float(qq[i] & 0xFFFFu); d[2 * i + 1] = __uint_as_float(qq[i] & 0xFFFF0000u); }
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) d[i] = fill;
+      }
     }
   } else {
     for (int e = threadIdx.x; e < rows * p.W; e += blockDim.x) {
       const int r = e / p.W, x = e - r * p.W;
       const int h = h0 + r;
-      pool_stage[r * p.Wp + p.pw + x] = (h >= 0 && h < p.H) ? src[(int64_t)h * p.W + x] : fill;
+      pool_stage[r * p.Wp + p.pw + x] = (h >= 0 && h < p.H) ? pool_load(src + (int64_t)h * p.W + x) : fill;
     }
   }
   __syncthreads();
-  float* dst = out + (plane * p.Ho + y0) * p.Wo;
+  T* dst = out + (plane * p.Ho + y0) * p.Wo;
   for (int e = threadIdx.x; e < th * p.Wo; e += blockDim.x) {
     const int y = e / p.Wo, x = e - y * p.Wo;
     const float* win = pool_stage + (y * p.Sh) * p.Wp + x * p.Sw;
     float best = -INFINITY;
     for (int dy = 0; dy < p.Kh; ++dy)
       for (int dx = 0; dx < p.Kw; ++dx) best = fmaxf(best, win[dy * p.Wp + dx]);
-    dst[e] = best;
+    pool_store(dst + e, best);
   }
+}
+
+// Tiling of window_max_2d_tiled: as many output rows per block as fit 24 KB of staged floats.
+inline bool plan_pool_tile(const gl_ap* in, const gl_windows* w, const gl_ap& A, int na, int per_piece, PoolTile* t) {
+  t->H = (int)in->shape[na]; t->W = (int)in->shape[na + 1];
+  t->Kh = (int)w->wshape[0]; t->Kw = (int)w->wshape[1];
+  t->Sh = (int)w->stride[0]; t->Sw = (int)w->stride[1];
+  t->ph = (int)w->pad_lo[0]; t->pw = (int)w->pad_lo[1];
+  t->Ho = (int)A.shape[na]; t->Wo = (int)A.shape[na + 1];
+  // staged columns: left border, the row, and whatever the last window reaches beyond it
+  t->Wp = std::max(t->pw + t->W, (t->Wo - 1) * t->Sw + t->Kw);
+  t->vec = (t->W % per_piece == 0) ? 1 : 0;
+  const int budget = 24 * 1024 / 4;   // floats of shared memory per block
+  const int max_rows = budget / t->Wp;
+  if (max_rows < t->Kh) return false;
+  t->TH = std::min(t->Ho, (max_rows - t->Kh) / t->Sh + 1);
+  t->tiles = (t->Ho + t->TH - 1) / t->TH;
+  t->TH = (t->Ho + t->tiles - 1) / t->tiles;   // even out the tiles
+  return prod(in->shape, 0, na) * t->tiles <= 0x7FFFFFFF;
 }
 
 // Fig. 2c with a 3x3 window, stride 2 and one border cell on the low side (the pooling layer of
@@ -1246,8 +1300,14 @@ int gl_compute_reduce_max(const gl_ap* in, const gl_windows* w, gl_ap* out, void
       t.ph = (int)w->pad_lo[0]; t.pw = (int)w->pad_lo[1];
       t.Ho = (int)A.shape[nc]; t.Wo = (int)A.shape[nc + 1];
       t.cv = (int)(in->shape[nc + 2] / per_piece);
-      t.total = prod(in->shape, 0, nc) * t.Ho * t.Wo * t.cv;
+      const int64_t pieces = prod(in->shape, 0, nc) * t.Ho * t.Wo * t.cv;
+      // few outputs with large windows: up to 32 lanes per output piece, while that leaves every lane four cells
+      // and the machine is not yet full
+      t.split_log2 = 0;
+      while (t.split_log2 < 5 && (t.Kh * t.Kw >> (t.split_log2 + 1)) >= 4 && (pieces << t.split_log2) < 148 * 2048 * 2) ++t.split_log2;
+      t.total = pieces << t.split_log2;
       if (t.total < (1ll << 31)) {
+        t.by_Kw = make_fastdiv(t.Kw);
         t.by_cv = make_fastdiv(t.cv);
         t.by_Wo = make_fastdiv(t.Wo);
         t.by_Ho = make_fastdiv(t.Ho);
@@ -1263,13 +1323,24 @@ int gl_compute_reduce_max(const gl_ap* in, const gl_windows* w, gl_ap* out, void
     }
   }
   if (bf16) {
-    // 2-byte planes ((..),(H,W)): the plain kernel; other bf16 forms have no kernel
+    // 2-byte planes ((..),(H,W)): the tiled kernel, else the plain one; other bf16 forms have no kernel
     const int nb = in->access_ndim;
     if (!w || w->n != 2 || in->shape[nb] >= (1 << 30) || in->shape[nb + 1] >= (1 << 30)) return GL_ERR_UNSUPPORTED;
     gl_ap A = *in;
     gl_shape_windows(in, w, &A);
     const float fill = w->pad_kind == GL_PAD_NEG_INF ? -INFINITY : 0.0f;
     const int64_t nwin = numel(want);
+    if (in->shape[nb] < (1 << 20) && in->shape[nb + 1] < (1 << 20) && w->wshape[0] < 1024 && w->wshape[1] < 1024 &&
+        w->stride[0] < 1024 && w->stride[1] < 1024) {
+      PoolTile t;
+      if (plan_pool_tile(in, w, A, nb, 8, &t)) {
+        const int rows = (t.TH - 1) * t.Sh + t.Kh;
+        window_max_2d_tiled<uint16_t><<<static_cast<unsigned>(prod(in->shape, 0, nb) * t.tiles), kThreads,
+                                        static_cast<size_t>(rows) * t.Wp * 4, st>>>(
+            static_cast<const uint16_t*>(in->data), static_cast<uint16_t*>(out->data), t, fill);
+        return launch_status();
+      }
+    }
     return launch_pdl(window_max_2d_bf16, dim3(grid_for(nwin, kThreads)), dim3(kThreads), 0, st, 1,
                       static_cast<const uint16_t*>(in->data), static_cast<uint16_t*>(out->data), prod(in->shape, 0, nb),
                       (int)in->shape[nb], (int)in->shape[nb + 1], (int)w->wshape[0], (int)w->wshape[1], (int)w->stride[0],
@@ -1307,28 +1378,11 @@ int gl_compute_reduce_max(const gl_ap* in, const gl_windows* w, gl_ap* out, void
   if (w->n == 2 && in->shape[na] < (1 << 20) && in->shape[na + 1] < (1 << 20) && w->wshape[0] < 1024 &&
       w->wshape[1] < 1024 && w->stride[0] < 1024 && w->stride[1] < 1024) {
     PoolTile t;
-    t.H = (int)in->shape[na]; t.W = (int)in->shape[na + 1];
-    t.Kh = (int)w->wshape[0]; t.Kw = (int)w->wshape[1];
-    t.Sh = (int)w->stride[0]; t.Sw = (int)w->stride[1];
-    t.ph = (int)w->pad_lo[0]; t.pw = (int)w->pad_lo[1];
-    t.Ho = (int)A.shape[na]; t.Wo = (int)A.shape[na + 1];
-    // staged columns: left border, the row, and whatever the last window reaches beyond it
-    t.Wp = std::max(t.pw + t.W, (t.Wo - 1) * t.Sw + t.Kw);
-    t.vec = (t.W % 4 == 0) ? 1 : 0;
-    const int budget = 24 * 1024 / 4;   // floats of shared memory per block
-    const int max_rows = budget / t.Wp;
-    const int64_t planes = prod(in->shape, 0, na);
-    if (max_rows >= t.Kh) {
-      t.TH = std::min(t.Ho, (max_rows - t.Kh) / t.Sh + 1);
-      t.tiles = (t.Ho + t.TH - 1) / t.TH;
-      t.TH = (t.Ho + t.tiles - 1) / t.tiles;   // even out the tiles
+    if (plan_pool_tile(in, w, A, na, 4, &t)) {
       const int rows = (t.TH - 1) * t.Sh + t.Kh;
-      const int64_t blocks = planes * t.tiles;
-      if (blocks <= 0x7FFFFFFF) {
-        window_max_2d_tiled<<<static_cast<unsigned>(blocks), kThreads, static_cast<size_t>(rows) * t.Wp * 4, st>>>(
-            src, dst, t, fill);
-        return launch_status();
-      }
+      window_max_2d_tiled<float><<<static_cast<unsigned>(prod(in->shape, 0, na) * t.tiles), kThreads,
+                                   static_cast<size_t>(rows) * t.Wp * 4, st>>>(src, dst, t, fill);
+      return launch_status();
     }
   }
   if (w->n == 2 && in->shape[na] < (1 << 30) && in->shape[na + 1] < (1 << 30)) {
