@@ -1348,6 +1348,12 @@ struct RowRunParams {
   int raw_stages;
   int w_elems;                  // O * Kh * Kw * C (they fit the raw stages, where the block parks them once)
   int segs, tiles;              // 128-column segments per output row; tiles = N * Ho * segs
+  // A block owns a strip of `strip` consecutive output rows of one image and segment.  Consecutive tiles share
+  // Kh - Sh input rows, so the widened runs live in a ring of `ring` slots (input row hp of the strip at slot
+  // (hp - first row) mod ring) and only the rows a tile adds - all Kh for the strip's first tile, min(Kh, Sh)
+  // afterwards - are copied and widened.
+  int strip, strips_per_img, ring;
+  FastDiv div_spi, div_ring;
   int ksteps;                   // MMAs (K = 16) per filter row
   int bn;                       // MMA N: O rounded up to 16
   uint32_t seg_bytes;           // bytes of one run: 127 * 16 + ksteps * 32
@@ -1367,8 +1373,10 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uin
 // as it lies in global memory, by plain bulk copies of whole 16-byte pieces (one copy per row for (H,W,C) items,
 // one per channel plane for (C,H,W) items); three warps then widen it into the padded row run: pixel wp of the
 // run of filter row kh holds the C channels of input pixel (ho * Sh + kh - ph, seg * 128 * Sw + wp - pw), zeros
-// for the border and for the channels past C.  The weights are rearranged into operand order by the whole block
-// once, before the first tile.  Nothing passes through a global-memory copy.
+// for the border and for the channels past C.  A block walks down a strip of output rows, so every input row of the
+// strip is copied and widened once and then serves the Kh / Sh tiles whose windows reach it.  The weights are
+// rearranged into operand order by the whole block once, before the first tile.  Nothing passes through a
+// global-memory copy.
 // CT, CL: channel count and item layout as compile-time constants (CT = 0: both taken from p at run time).  The
 // widening warps are bound by their instruction count per pixel; with constants it is a fifth of the general form.
 template <int CT, int CL>
@@ -1379,11 +1387,10 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   unsigned char* gen = smem_raw + (base - raw);
-  const uint32_t stage_bytes = static_cast<uint32_t>(p.Kh) * p.slot_bytes;
   const uint32_t epi_base = base;                                         // 1024-byte aligned staging tiles
   const uint32_t b_base = epi_base + kRunEpiBytes;
   const uint32_t a_base = b_base + ((p.b_bytes + 127u) & ~127u);
-  const uint32_t r_base = a_base + static_cast<uint32_t>(p.stages) * stage_bytes;   // raw copies (slot_bytes is a multiple of 128)
+  const uint32_t r_base = a_base + static_cast<uint32_t>(p.ring) * p.slot_bytes;   // raw copies (slot_bytes is a multiple of 128)
   const uint32_t bars_off = (r_base - base) + static_cast<uint32_t>(p.raw_stages) * p.raw_stage_bytes;
   uint64_t* bars = reinterpret_cast<uint64_t*>(gen + bars_off);
   const uint32_t bar_full = smem_u32(bars);                  // [kRunMaxStages] widened runs ready
@@ -1454,23 +1461,28 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
 
   const int npx = static_cast<int>(p.seg_bytes >> (p.cp_log2 + 1));   // pixels of a run
   const int epx = p.channels_last ? p.C : 1;                          // elements per pixel in one raw copy
+  // this block's strip: image, segment, first output row, number of tiles
+  uint32_t strip_id, img_seg, img, seg;
+  p.div_spi.divmod(blockIdx.x, img_seg, strip_id);
+  p.div_segs.divmod(img_seg, img, seg);
+  const int ho0 = static_cast<int>(strip_id) * p.strip;
+  const int ntiles = min(p.strip, p.Ho - ho0);
+  const int hp0 = ho0 * p.Sh;                       // first padded input row of the strip (row h = hp - ph)
+  const int nnew_later = min(p.Kh, p.Sh);           // rows a tile adds (the first tile adds all Kh)
+  const int w_first = static_cast<int>(seg) * (kBM * p.Sw) - p.pw;   // input column of run pixel 0
+  const int w_lo = max(w_first, 0), w_hi = min(w_first + npx, p.W);
   if (warp == 0) {
-    // ---------------- raw copies: lane i takes copy i = (filter row, segment) of the tile ----------------
-    const int ncopies = p.Kh * p.nseg;   // at most 32
-    uint32_t kh_l, c_l;
-    p.div_nseg.divmod(static_cast<uint32_t>(lane), kh_l, c_l);
+    // ---------------- raw copies: lane i takes copy i = (new row, raw segment) of the tile ----------------
+    uint32_t j_l, c_l;
+    p.div_nseg.divmod(static_cast<uint32_t>(lane), j_l, c_l);
     uint32_t r = 0, ph = 0;
-    for (int u = blockIdx.x; u < p.tiles; u += gridDim.x) {
-      uint32_t row, seg, img, ho;
-      p.div_segs.divmod(static_cast<uint32_t>(u), row, seg);
-      p.div_ho.divmod(row, img, ho);
+    for (int t = 0; t < ntiles; ++t) {
       if (!mbar_wait(bar_rempty + 8 * r, ph ^ 1u, abort_flag)) break;
-      const int w_first = static_cast<int>(seg) * (kBM * p.Sw) - p.pw;   // input column of run pixel 0
-      const int w_lo = max(w_first, 0), w_hi = min(w_first + npx, p.W);
-      const int h = static_cast<int>(ho) * p.Sh + static_cast<int>(kh_l) - p.ph;
+      const int nnew = t == 0 ? p.Kh : nnew_later;
+      const int h = hp0 + t * p.Sh + p.Kh - nnew + static_cast<int>(j_l) - p.ph;
       uint32_t size = 0;
       int64_t a0 = 0;
-      if (lane < ncopies && h >= 0 && h < p.H && w_hi > w_lo) {
+      if (static_cast<int>(j_l) < nnew && h >= 0 && h < p.H && w_hi > w_lo) {
         const int64_t e0 = static_cast<int64_t>(img) * p.xs_n + static_cast<int64_t>(h) * p.xs_h +
                            (p.channels_last ? static_cast<int64_t>(w_lo) * p.C : static_cast<int64_t>(c_l) * p.xs_c + w_lo);
         const int64_t b0 = e0 * 2, b1 = b0 + static_cast<int64_t>(w_hi - w_lo) * epx * 2;
@@ -1481,29 +1493,29 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
       if (lane == 0) mbar_expect_tx(bar_rfull + 8 * r, total);
       __syncwarp();
       if (size)
-        bulk_copy_g2s(r_base + r * p.raw_stage_bytes + kh_l * p.raw_row_bytes + c_l * p.raw_seg_bytes,
+        bulk_copy_g2s(r_base + r * p.raw_stage_bytes + j_l * p.raw_row_bytes + c_l * p.raw_seg_bytes,
                       reinterpret_cast<const unsigned char*>(x) + a0, size, bar_rfull + 8 * r);
       if (++r == static_cast<uint32_t>(p.raw_stages)) { r = 0; ph ^= 1u; }
     }
   } else if (warp >= 6) {
-    // ---------------- widening: raw rows -> padded row runs, filter rows dealt round robin to the warps ----------------
+    // ---------------- widening: raw rows -> padded row runs; the halves of the new rows dealt round robin to the warps ----------------
     const int eidx = warp - 6;
     const int cp = 1 << p.cp_log2;
     constexpr int kC = CT > 0 ? CT : 8;
     const int nch = CT > 0 ? CT : p.C;
     const bool cl = CT > 0 ? CL != 0 : p.channels_last != 0;
     const int epx_e = cl ? nch : 1;
+    const int npx_half = ((npx >> 1) + 31) & ~31;
     uint32_t s = 0, ph = 0, r = 0, rph = 0;
-    for (int u = blockIdx.x; u < p.tiles; u += gridDim.x) {
-      uint32_t row, seg, img, ho;
-      p.div_segs.divmod(static_cast<uint32_t>(u), row, seg);
-      p.div_ho.divmod(row, img, ho);
+    for (int t = 0; t < ntiles; ++t) {
       if (!mbar_wait(bar_rfull + 8 * r, rph, abort_flag)) break;
       if (!mbar_wait(bar_empty + 8 * s, ph ^ 1u, abort_flag)) break;
-      const int w_first = static_cast<int>(seg) * (kBM * p.Sw) - p.pw;
-      const int w_lo = max(w_first, 0), w_hi = min(w_first + npx, p.W);
-      for (int kh = eidx; kh < p.Kh; kh += kRunExpanders) {
-        const int h = static_cast<int>(ho) * p.Sh + kh - p.ph;
+      const int nnew = t == 0 ? p.Kh : nnew_later;
+      const int hp_first = hp0 + t * p.Sh + p.Kh - nnew;
+      for (int item = eidx; item < 2 * nnew; item += kRunExpanders) {
+        const int j = item >> 1, half = item & 1;
+        const int wp_begin = half ? npx_half : 0, wp_end = half ? npx : min(npx, npx_half);
+        const int h = hp_first + j - p.ph;
         const bool row_ok = h >= 0 && h < p.H;
         // where the stretch starts inside its 16-byte aligned copy, per raw copy of this row
         const int64_t e0 = static_cast<int64_t>(img) * p.xs_n + static_cast<int64_t>(h) * p.xs_h +
@@ -1514,16 +1526,18 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
         for (int c = 0; c < kC; ++c)
           delta[c] = static_cast<uint32_t>((((e0 + (cl ? 0 : c * p.xs_c)) * 2) & 15) >> 1) +
                      (cl ? static_cast<uint32_t>(c) : static_cast<uint32_t>(c) * (p.raw_seg_bytes >> 1));
+        uint32_t slot, lap;
+        p.div_ring.divmod(static_cast<uint32_t>(hp_first + j - hp0), lap, slot);
         const uint16_t* src_row = reinterpret_cast<const uint16_t*>(gen + (r_base - base) + r * p.raw_stage_bytes +
-                                                                    static_cast<uint32_t>(kh) * p.raw_row_bytes);
-        unsigned char* dst_row = gen + (a_base - base) + s * stage_bytes + static_cast<uint32_t>(kh) * p.slot_bytes;
+                                                                    static_cast<uint32_t>(j) * p.raw_row_bytes);
+        unsigned char* dst_row = gen + (a_base - base) + slot * p.slot_bytes;
         // four pixels per lane and trip: their loads are issued together
-        for (int wp0 = lane; wp0 < npx; wp0 += 128) {
+        for (int wp0 = wp_begin + lane; wp0 < wp_end; wp0 += 128) {
           uint32_t v[4][8];
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
             const int wp = wp0 + 32 * k, w = w_first + wp;
-            const bool ok = row_ok && wp < npx && w >= w_lo && w < w_hi;
+            const bool ok = row_ok && wp < wp_end && w >= w_lo && w < w_hi;
             const uint16_t* px = src_row + (ok ? (w - w_lo) * epx_e : 0);
 #pragma unroll
             for (int c = 0; c < 8; ++c) v[k][c] = 0u;
@@ -1534,7 +1548,7 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
             const int wp = wp0 + 32 * k;
-            if (wp < npx) {
+            if (wp < wp_end) {
               unsigned char* dst = dst_row + (static_cast<uint32_t>(wp) << (p.cp_log2 + 1));
               const uint32_t w01 = v[k][0] | (v[k][1] << 16), w23 = v[k][2] | (v[k][3] << 16);
               if (cp == 8) *reinterpret_cast<uint4*>(dst) = make_uint4(w01, w23, v[k][4] | (v[k][5] << 16), v[k][6] | (v[k][7] << 16));
@@ -1561,16 +1575,19 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
       const uint32_t b_step = (2u * p.bn * 16u) >> 4;                                           // two K chunks per MMA
       uint32_t s = 0, ph = 0, tile_it = 0;
       bool ok = true;
-      for (int u = blockIdx.x; u < p.tiles && ok; u += gridDim.x, ++tile_it) {
+      uint32_t slot = 0;   // ring slot of the tile's first input row: (t * Sh) mod ring
+      const uint32_t slot_step = static_cast<uint32_t>(p.Sh) % static_cast<uint32_t>(p.ring);
+      for (int t = 0; t < ntiles && ok; ++t, ++tile_it) {
         const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
         if (!mbar_wait(bar_tempty + 8 * acc, aph ^ 1u, abort_flag)) { ok = false; break; }
         if (!mbar_wait(bar_full + 8 * s, ph, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * p.bn;
-        uint64_t da_row = desc_a0 + ((s * stage_bytes) >> 4), db = desc_b0;
-        uint32_t accumulate = 0;
-        for (int kh = 0; kh < p.Kh; ++kh, da_row += p.slot_bytes >> 4) {
-          uint64_t da = da_row;
+        uint64_t db = desc_b0;
+        uint32_t accumulate = 0, sl = slot;
+        for (int kh = 0; kh < p.Kh; ++kh) {
+          uint64_t da = desc_a0 + ((sl * p.slot_bytes) >> 4);
+          if (++sl == static_cast<uint32_t>(p.ring)) sl = 0;
           for (int k = 0; k < p.ksteps; ++k, da += 2, db += b_step) {
             if (leader) tc_mma_bf16(d_tmem, da, db, idesc, accumulate);
             accumulate = 1u;
@@ -1581,6 +1598,8 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
           tc_commit(bar_tfull + 8 * acc);
         }
         if (++s == static_cast<uint32_t>(p.stages)) { s = 0; ph ^= 1u; }
+        slot += slot_step;
+        if (slot >= static_cast<uint32_t>(p.ring)) slot -= p.ring;
       }
     }
   } else {
@@ -1589,10 +1608,9 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
     const bool leader = elect_one();   // issues this warp's TMA stores (always the same lane: it owns the bulk groups)
     uint32_t tile_it = 0, chunk_it = 0;
     bool ok = true;
-    for (int u = blockIdx.x; u < p.tiles && ok; u += gridDim.x, ++tile_it) {
+    for (int t = 0; t < ntiles && ok; ++t, ++tile_it) {
       const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
-      uint32_t row, seg;
-      p.div_segs.divmod(static_cast<uint32_t>(u), row, seg);
+      const uint32_t row = img * static_cast<uint32_t>(p.Ho) + static_cast<uint32_t>(ho0 + t);   // output row of the (N*Ho, Wo, O) view
       if (!mbar_wait(bar_tfull + 8 * acc, aph, abort_flag)) { ok = false; break; }
       tc_fence_after();
       const int cstep = p.out_bf16 ? 64 : 32;   // a staged row is 128 bytes: 32 fp32 or 64 bf16 columns
@@ -2048,8 +2066,9 @@ ConvPlan plan_conv(const DotProblem& d, uint32_t flags) {
     const uint32_t raw_seg = static_cast<uint32_t>(((seg / (2 * cp)) * (d.channels_last ? d.C : 1) * 2 + 30 + 15) / 16 * 16);
     const int64_t raw_stage = d.Kh * nseg * static_cast<int64_t>(raw_seg);
     const int64_t room = 113 * 1024 - 1024 - kRunEpiBytes - 256 - ((b_bytes + 127) & ~127u);   // two blocks per SM
-    const int64_t stages = 2;                                                                   // widened runs
-    const int64_t raw_stages = std::min<int64_t>(kRunMaxStages, (room - stages * d.Kh * slot) / raw_stage);
+    const int64_t stages = 3;                                                                   // tiles in flight
+    const int64_t ring = d.Kh + (stages - 1) * d.Sh;                                            // widened runs kept
+    const int64_t raw_stages = std::min<int64_t>(kRunMaxStages, (room - ring * slot) / raw_stage);
     if (raw_stages >= 2 && d.O * d.Kh * d.Kw * d.C * 2 <= raw_stages * raw_stage) {   // the weights fit the raw stages
       pl.rowrun = true;
       pl.prepass = false;   // the kernel reads both operands where they are, in either item layout
@@ -2446,12 +2465,18 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     rp.seg_bytes = pl.rr_seg; rp.slot_bytes = pl.rr_slot;
     rp.b_bytes = pl.rr_b_bytes;
     rp.stages = pl.rr_stages;
+    rp.ring = static_cast<int>(d.Kh + (pl.rr_stages - 1) * d.Sh);
+    // strips: about one per block slot (two blocks per SM)
+    rp.strip = static_cast<int>(std::max<int64_t>(1, (static_cast<int64_t>(rp.tiles) + 2 * num_sms() - 1) / (2 * num_sms())));
+    rp.strips_per_img = static_cast<int>((d.Ho + rp.strip - 1) / rp.strip);
+    rp.div_spi.set(rp.strips_per_img);
+    rp.div_ring.set(rp.ring);
     rp.div_segs.set(rp.segs);
     rp.div_ho.set(d.Ho);
     CUtensorMap mc;
     if (!encode_result_rows(&mc, dst, d.N * d.Ho, d.Wo, d.O, out_bf16 != 0)) return GL_ERR_CUDA;
     const int smem = 1024 + kRunEpiBytes + static_cast<int>((rp.b_bytes + 127u) & ~127u) +
-                     rp.stages * rp.Kh * static_cast<int>(rp.slot_bytes) + rp.raw_stages * static_cast<int>(rp.raw_stage_bytes) + 256;
+                     rp.ring * static_cast<int>(rp.slot_bytes) + rp.raw_stages * static_cast<int>(rp.raw_stage_bytes) + 256;
     static bool attr_set_dev[64] = {false};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return GL_ERR_CUDA;
@@ -2462,7 +2487,8 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
         return GL_ERR_CUDA;
       attr_set_dev[dev] = true;
     }
-    const int grid = std::min(rp.tiles, 2 * num_sms());
+    const int64_t grid = d.N * rp.segs * rp.strips_per_img;   // one strip per block
+    if (grid >= (1ll << 31)) return GL_ERR_UNSUPPORTED;
     // three channels (RGB) have kernels of their own, one per item layout
     auto kernel = d.C == 3 ? (d.channels_last ? conv_rowrun<3, 1> : conv_rowrun<3, 0>) : conv_rowrun<0, 0>;
     return launch_pdl(kernel, dim3(static_cast<unsigned>(grid)), dim3(kRunThreads), static_cast<size_t>(smem), st, 1,
