@@ -1346,7 +1346,7 @@ struct RowRunParams {
   uint32_t raw_seg_bytes;       // shared-memory pitch of one raw copy, of the copies of a row, of a raw stage
   uint32_t raw_row_bytes, raw_stage_bytes;
   int raw_stages;
-  int w_elems;                  // O * Kh * Kw * C (they fit the raw stages, where the block parks them once)
+  int w_elems;                  // O * Kh * Kw * C (they fit the ring of row runs, where the block parks them once)
   int segs, tiles;              // 128-column segments per output row; tiles = N * Ho * segs
   // A block owns a strip of `strip` consecutive output rows of one image and segment.  Consecutive tiles share
   // Kh - Sh input rows, so the widened runs live in a ring of `ring` slots (input row hp of the strip at slot
@@ -1360,7 +1360,7 @@ struct RowRunParams {
   uint32_t slot_bytes;          // shared-memory pitch of a run
   uint32_t b_bytes;             // resident weights: Kh * ksteps * 2 chunks * bn rows * 16 bytes
   int stages;
-  FastDiv div_segs, div_ho, div_nseg, div_bn, div_chunks;
+  FastDiv div_segs, div_ho, div_nseg, div_bn;
 };
 
 __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -1425,40 +1425,6 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
   pdl_wait();
   pdl_launch_dependents();
 
-  // ---- weights into operand order [kh][K chunk j][row o < bn][8 elements]: element kw * cp + c of filter row
-  // kh sits at (j, i) = ((kw * cp + c) / 8, (kw * cp + c) % 8), zeros elsewhere.  The weight tensor is first
-  // copied as it is (16-byte loads) into the area of the raw stages, which nothing uses yet; every thread then
-  // assembles 16-byte pieces (kh, j, o) from it.
-  {
-    uint16_t* wraw = reinterpret_cast<uint16_t*>(gen + (r_base - base));
-    const int nvec = p.w_elems >> 3;
-    for (int i = threadIdx.x; i < nvec; i += kRunThreads)
-      reinterpret_cast<uint4*>(wraw)[i] = reinterpret_cast<const uint4*>(wt)[i];
-    for (int i = nvec * 8 + threadIdx.x; i < p.w_elems; i += kRunThreads) wraw[i] = wt[i];
-    __syncthreads();
-    const int chunks = 2 * p.ksteps, pieces = p.Kh * chunks * p.bn;
-    const int cp_mask = (1 << p.cp_log2) - 1;
-    uint4* wop = reinterpret_cast<uint4*>(gen + (b_base - base));
-    for (int q = threadIdx.x; q < pieces; q += kRunThreads) {
-      uint32_t t, o, kh, j;
-      p.div_bn.divmod(static_cast<uint32_t>(q), t, o);
-      p.div_chunks.divmod(t, kh, j);
-      // (H,W,C) items: element ((o Kh + kh) Kw + kw) C + c;  (C,H,W) items: ((o C + c) Kh + kh) Kw + kw
-      const int at = p.channels_last ? static_cast<int>(o * p.Kh + kh) * p.Kw * p.C : (static_cast<int>(o) * p.C * p.Kh + static_cast<int>(kh)) * p.Kw;
-      const int step_kw = p.channels_last ? p.C : 1, step_c = p.channels_last ? 1 : p.Kh * p.Kw;
-      uint32_t v[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int el = static_cast<int>(j) * 8 + i, kw = el >> p.cp_log2, c = el & cp_mask;
-        const bool ok = static_cast<int64_t>(o) < p.O && kw < p.Kw && c < p.C;
-        v[i] = ok ? wraw[at + kw * step_kw + c * step_c] : 0u;
-      }
-      wop[q] = make_uint4(v[0] | (v[1] << 16), v[2] | (v[3] << 16), v[4] | (v[5] << 16), v[6] | (v[7] << 16));
-    }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads them through the async proxy
-    __syncthreads();
-  }
-
   const int npx = static_cast<int>(p.seg_bytes >> (p.cp_log2 + 1));   // pixels of a run
   const int epx = p.channels_last ? p.C : 1;                          // elements per pixel in one raw copy
   // this block's strip: image, segment, first output row, number of tiles
@@ -1471,30 +1437,74 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
   const int nnew_later = min(p.Kh, p.Sh);           // rows a tile adds (the first tile adds all Kh)
   const int w_first = static_cast<int>(seg) * (kBM * p.Sw) - p.pw;   // input column of run pixel 0
   const int w_lo = max(w_first, 0), w_hi = min(w_first + npx, p.W);
-  if (warp == 0) {
-    // ---------------- raw copies: lane i takes copy i = (new row, raw segment) of the tile ----------------
+  // raw copies of tile t into raw stage r: lane i takes copy i = (new row, raw segment); called by warp 0
+  auto copy_tile = [&](int t, uint32_t r) {
     uint32_t j_l, c_l;
     p.div_nseg.divmod(static_cast<uint32_t>(lane), j_l, c_l);
-    uint32_t r = 0, ph = 0;
-    for (int t = 0; t < ntiles; ++t) {
-      if (!mbar_wait(bar_rempty + 8 * r, ph ^ 1u, abort_flag)) break;
-      const int nnew = t == 0 ? p.Kh : nnew_later;
-      const int h = hp0 + t * p.Sh + p.Kh - nnew + static_cast<int>(j_l) - p.ph;
-      uint32_t size = 0;
-      int64_t a0 = 0;
-      if (static_cast<int>(j_l) < nnew && h >= 0 && h < p.H && w_hi > w_lo) {
-        const int64_t e0 = static_cast<int64_t>(img) * p.xs_n + static_cast<int64_t>(h) * p.xs_h +
-                           (p.channels_last ? static_cast<int64_t>(w_lo) * p.C : static_cast<int64_t>(c_l) * p.xs_c + w_lo);
-        const int64_t b0 = e0 * 2, b1 = b0 + static_cast<int64_t>(w_hi - w_lo) * epx * 2;
-        a0 = b0 & ~static_cast<int64_t>(15);                              // whole 16-byte pieces around the stretch;
-        size = static_cast<uint32_t>(((b1 + 15) & ~static_cast<int64_t>(15)) - a0);   // the tensor's byte count is a multiple of 16
+    const int nnew = t == 0 ? p.Kh : nnew_later;
+    const int h = hp0 + t * p.Sh + p.Kh - nnew + static_cast<int>(j_l) - p.ph;
+    uint32_t size = 0;
+    int64_t a0 = 0;
+    if (static_cast<int>(j_l) < nnew && h >= 0 && h < p.H && w_hi > w_lo) {
+      const int64_t e0 = static_cast<int64_t>(img) * p.xs_n + static_cast<int64_t>(h) * p.xs_h +
+                         (p.channels_last ? static_cast<int64_t>(w_lo) * p.C : static_cast<int64_t>(c_l) * p.xs_c + w_lo);
+      const int64_t b0 = e0 * 2, b1 = b0 + static_cast<int64_t>(w_hi - w_lo) * epx * 2;
+      a0 = b0 & ~static_cast<int64_t>(15);                              // whole 16-byte pieces around the stretch;
+      size = static_cast<uint32_t>(((b1 + 15) & ~static_cast<int64_t>(15)) - a0);   // the tensor's byte count is a multiple of 16
+    }
+    const uint32_t total = __reduce_add_sync(0xffffffffu, size);
+    if (lane == 0) mbar_expect_tx(bar_rfull + 8 * r, total);
+    __syncwarp();
+    if (size)
+      bulk_copy_g2s(r_base + r * p.raw_stage_bytes + j_l * p.raw_row_bytes + c_l * p.raw_seg_bytes,
+                    reinterpret_cast<const unsigned char*>(x) + a0, size, bar_rfull + 8 * r);
+  };
+  if (warp == 0 && ntiles > 0) copy_tile(0, 0);   // in flight while the block arranges the weights
+
+  // ---- weights into operand order [kh][K chunk j][row o < bn][8 elements]: element kw * cp + c of filter row
+  // kh sits at (j, i) = ((kw * cp + c) / 8, (kw * cp + c) % 8), zeros elsewhere.  The weight tensor is first
+  // copied as it is (16-byte loads) into the ring of row runs, which nothing uses yet; every thread then
+  // assembles 16-byte pieces (kh, j, o) from it.
+  {
+    uint16_t* wraw = reinterpret_cast<uint16_t*>(gen + (a_base - base));
+    const int nvec = p.w_elems >> 3;
+    for (int i = threadIdx.x; i < nvec; i += kRunThreads)
+      reinterpret_cast<uint4*>(wraw)[i] = reinterpret_cast<const uint4*>(wt)[i];
+    for (int i = nvec * 8 + threadIdx.x; i < p.w_elems; i += kRunThreads) wraw[i] = wt[i];
+    __syncthreads();
+    // a thread takes one (filter row, output channel) pair and writes its row of K: `chunks` pieces of 16 bytes
+    const int chunks = 2 * p.ksteps, pairs = p.Kh * p.bn;
+    const int cp_mask = (1 << p.cp_log2) - 1;
+    uint4* wop = reinterpret_cast<uint4*>(gen + (b_base - base));
+    // (H,W,C) items: element ((o Kh + kh) Kw + kw) C + c;  (C,H,W) items: ((o C + c) Kh + kh) Kw + kw
+    const int step_kw = p.channels_last ? p.C : 1, step_c = p.channels_last ? 1 : p.Kh * p.Kw;
+    for (int q = threadIdx.x; q < pairs; q += kRunThreads) {
+      uint32_t kh, o;
+      p.div_bn.divmod(static_cast<uint32_t>(q), kh, o);
+      const bool row_ok = static_cast<int64_t>(o) < p.O;
+      const int at = p.channels_last ? static_cast<int>(o * p.Kh + kh) * p.Kw * p.C
+                                     : (static_cast<int>(o) * p.C * p.Kh + static_cast<int>(kh)) * p.Kw;
+      for (int j = 0; j < chunks; ++j) {
+        uint32_t v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int el = j * 8 + i, kw = el >> p.cp_log2, c = el & cp_mask;
+          v[i] = (row_ok && kw < p.Kw && c < p.C) ? wraw[at + kw * step_kw + c * step_c] : 0u;
+        }
+        wop[(static_cast<int>(kh) * chunks + j) * p.bn + static_cast<int>(o)] =
+            make_uint4(v[0] | (v[1] << 16), v[2] | (v[3] << 16), v[4] | (v[5] << 16), v[6] | (v[7] << 16));
       }
-      const uint32_t total = __reduce_add_sync(0xffffffffu, size);
-      if (lane == 0) mbar_expect_tx(bar_rfull + 8 * r, total);
-      __syncwarp();
-      if (size)
-        bulk_copy_g2s(r_base + r * p.raw_stage_bytes + j_l * p.raw_row_bytes + c_l * p.raw_seg_bytes,
-                      reinterpret_cast<const unsigned char*>(x) + a0, size, bar_rfull + 8 * r);
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads them through the async proxy
+    __syncthreads();
+  }
+
+  if (warp == 0) {
+    // ---------------- raw copies: the first tile's went out before the weights were arranged ----------------
+    uint32_t r = 1 % static_cast<uint32_t>(p.raw_stages), ph = p.raw_stages == 1 ? 1u : 0u;
+    for (int t = 1; t < ntiles; ++t) {
+      if (!mbar_wait(bar_rempty + 8 * r, ph ^ 1u, abort_flag)) break;
+      copy_tile(t, r);
       if (++r == static_cast<uint32_t>(p.raw_stages)) { r = 0; ph ^= 1u; }
     }
   } else if (warp >= 6) {
@@ -2069,7 +2079,7 @@ ConvPlan plan_conv(const DotProblem& d, uint32_t flags) {
     const int64_t stages = 3;                                                                   // tiles in flight
     const int64_t ring = d.Kh + (stages - 1) * d.Sh;                                            // widened runs kept
     const int64_t raw_stages = std::min<int64_t>(kRunMaxStages, (room - ring * slot) / raw_stage);
-    if (raw_stages >= 2 && d.O * d.Kh * d.Kw * d.C * 2 <= raw_stages * raw_stage) {   // the weights fit the raw stages
+    if (raw_stages >= 2 && d.O * d.Kh * d.Kw * d.C * 2 <= ring * slot) {   // the weights fit the ring, where the block parks them once
       pl.rowrun = true;
       pl.prepass = false;   // the kernel reads both operands where they are, in either item layout
       pl.rr_cp = cp; pl.rr_ksteps = ksteps; pl.rr_bn = bn; pl.rr_stages = static_cast<int>(stages);
@@ -2451,7 +2461,6 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     if (d.channels_last) { rp.xs_h = d.W * d.C; rp.xs_c = 1; }
     else { rp.xs_h = d.W; rp.xs_c = d.H * d.W; }
     rp.div_bn.set(pl.rr_bn);
-    rp.div_chunks.set(2 * pl.rr_ksteps);
     rp.nseg = pl.rr_nseg;
     rp.raw_seg_bytes = pl.rr_raw_seg;
     rp.raw_row_bytes = pl.rr_raw_seg * static_cast<uint32_t>(pl.rr_nseg);
