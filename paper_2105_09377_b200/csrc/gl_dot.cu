@@ -1477,19 +1477,21 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
     const int cp_mask = (1 << p.cp_log2) - 1;
     uint4* wop = reinterpret_cast<uint4*>(gen + (b_base - base));
     // (H,W,C) items: element ((o Kh + kh) Kw + kw) C + c;  (C,H,W) items: ((o C + c) Kh + kh) Kw + kw
-    const int step_kw = p.channels_last ? p.C : 1, step_c = p.channels_last ? 1 : p.Kh * p.Kw;
+    // (with CT > 0 the channel count and the layout are constants and most of the index arithmetic folds)
+    const int wC = CT > 0 ? CT : p.C;
+    const bool wcl = CT > 0 ? CL != 0 : p.channels_last != 0;
+    const int step_kw = wcl ? wC : 1, step_c = wcl ? 1 : p.Kh * p.Kw;
     for (int q = threadIdx.x; q < pairs; q += kRunThreads) {
       uint32_t kh, o;
       p.div_bn.divmod(static_cast<uint32_t>(q), kh, o);
       const bool row_ok = static_cast<int64_t>(o) < p.O;
-      const int at = p.channels_last ? static_cast<int>(o * p.Kh + kh) * p.Kw * p.C
-                                     : (static_cast<int>(o) * p.C * p.Kh + static_cast<int>(kh)) * p.Kw;
+      const int at = wcl ? static_cast<int>(o * p.Kh + kh) * p.Kw * wC : (static_cast<int>(o) * wC * p.Kh + static_cast<int>(kh)) * p.Kw;
       for (int j = 0; j < chunks; ++j) {
         uint32_t v[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
           const int el = j * 8 + i, kw = el >> p.cp_log2, c = el & cp_mask;
-          v[i] = (row_ok && kw < p.Kw && c < p.C) ? wraw[at + kw * step_kw + c * step_c] : 0u;
+          v[i] = (row_ok && kw < p.Kw && c < wC) ? wraw[at + kw * step_kw + c * step_c] : 0u;
         }
         wop[(static_cast<int>(kh) * chunks + j) * p.bn + static_cast<int>(o)] =
             make_uint4(v[0] | (v[1] << 16), v[2] | (v[3] << 16), v[4] | (v[5] << 16), v[6] | (v[7] << 16));
