@@ -428,6 +428,23 @@ __device__ __forceinline__ void tma_load_im2col(uint32_t dst, const CUtensorMap*
       : "memory");
 }
 
+// Prefetches into L2 with the coordinates of a later load.  A kernel launched with programmatic stream
+// serialisation issues them BEFORE it waits for its predecessor: a prefetch consumes nothing, and L2 is where all
+// SMs' writes meet, so a line the predecessor still writes afterwards is simply updated there.  The operands of
+// the first tiles then come from L2 instead of from DRAM once the wait is over.
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int x, int y) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap* map, int c, int w, int h, int n) {
+  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c), "r"(w), "r"(h), "r"(n) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_im2col(const CUtensorMap* map, int c, int w, int h, int n, uint16_t kw, uint16_t kh) {
+  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.im2col [%0, {%1, %2, %3, %4}], {%5, %6};"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(c), "r"(w), "r"(h), "r"(n), "h"(kw), "h"(kh) : "memory");
+}
+
 // ---- two-block clusters (CTA pairs): one tcgen05.mma spans the tensor cores and the shared
 // memory of both blocks of a pair; barriers that both blocks feed live in the pair's first block.
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -573,6 +590,8 @@ struct TcParams {
   // With ksplit > 1 the kernel writes partial [s][M][O] planes and a second kernel adds them up.
   int ksplit, kper;
   FastDiv div_ksplit;
+  int prefetch;           // operands may be prefetched into L2 before the dependency wait (not when the call's own
+                          // layout copies, the predecessor in the stream, are what writes them)
   // kRowWin only: one tile = (up to) 128 outputs of one output row
   int Hp, segs;           // padded input rows per image; 128-wide segments per output row
   FastDiv div_segs, div_ho;
@@ -652,11 +671,43 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
   else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  const int num_tiles = p.tiles_m * p.tiles_n * p.ksplit;   // work units (p.tiles_m counts 128*CTAS-row tiles)
+  const int unit0 = static_cast<int>(blockIdx.x) / CTAS, unit_step = static_cast<int>(gridDim.x) / CTAS;
+  // while the predecessor drains: the operands of this block's first unit (at most 4 K blocks of it) on their
+  // way into L2
+  if (p.prefetch && (MODE == kDense || MODE == kIm2col) && (warp == 0 || warp == 6) && unit0 < num_tiles) {
+    if (elect_one()) {
+      uint32_t t, ks, tm, tn;
+      p.div_ksplit.divmod(static_cast<uint32_t>(unit0), t, ks);
+      p.div_tiles_n.divmod(t, tm, tn);
+      const int kb_begin = static_cast<int>(ks) * p.kper, kb_end = min(min(p.kblocks, kb_begin + p.kper), kb_begin + 4);
+      const int m0 = (static_cast<int>(tm) * CTAS + static_cast<int>(rank)) * kBM;
+      const int n0 = static_cast<int>(tn) * BN + static_cast<int>(rank) * (BN / CTAS);
+      if (MODE == kDense) {
+        for (int kb = kb_begin; kb < kb_end; ++kb) {
+          if (warp == 0) tma_prefetch_2d(&map_a, kb * kBK, m0);
+          else tma_prefetch_2d(&map_b, kb * kBK, n0);
+        }
+      } else {
+        uint32_t im, rem, ho, wo;
+        p.div_howo.divmod(static_cast<uint32_t>(m0), im, rem);
+        p.div_wo.divmod(rem, ho, wo);
+        const int tap0 = kb_begin / p.cchunks;
+        int cc = kb_begin - tap0 * p.cchunks, kh = tap0 / p.Kw, kw = tap0 - kh * p.Kw;
+        for (int kb = kb_begin; kb < kb_end; ++kb) {
+          if (warp == 0)
+            tma_prefetch_im2col(&map_a, cc * kBK, static_cast<int>(wo) * p.Sw - p.pw, static_cast<int>(ho) * p.Sh - p.ph,
+                                static_cast<int>(im), static_cast<uint16_t>(kw), static_cast<uint16_t>(kh));
+          else
+            tma_prefetch_2d(&map_b, (kh * p.Kw + kw) * p.Cp + cc * kBK, n0);
+          if (++cc == p.cchunks) { cc = 0; if (++kw == p.Kw) { kw = 0; ++kh; } }
+        }
+      }
+    }
+  }
   pdl_wait();
   pdl_launch_dependents();
 
-  const int num_tiles = p.tiles_m * p.tiles_n * p.ksplit;   // work units (p.tiles_m counts 128*CTAS-row tiles)
-  const int unit0 = static_cast<int>(blockIdx.x) / CTAS, unit_step = static_cast<int>(gridDim.x) / CTAS;
 
   if (warp == 0 || warp == 6) {
     // ---------------- TMA producers: warp 0 stages A, warp 6 stages B ----------------
@@ -1003,6 +1054,7 @@ struct HaloParams {
   int tg, groups_per_chunk;                 // a B stage holds tg consecutive taps (a filter row, or one tap) of one chunk
   int ph, pw;
   int sa_stages, sb_stages, b_resident;     // b_resident: every B stage is loaded once per block and kept
+  int prefetch;                             // operands may be prefetched into L2 before the dependency wait
   uint32_t a_bytes, b_bytes;                // bytes of one input box (64 channels); of one B stage
   FastDiv div_tiles_n, div_tpi, div_wb;     // tiles per image; padded width
 };
@@ -1090,11 +1142,33 @@ conv_halo(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  pdl_wait();
-  pdl_launch_dependents();
   // work units: p.tiles_m counts tiles of CTAS M tiles; this block takes M tile tm * CTAS + rank
   const int num_tiles = p.tiles_m * p.tiles_n;
   const int unit0 = static_cast<int>(blockIdx.x) / CTAS, unit_step = static_cast<int>(gridDim.x) / CTAS;
+  // while the predecessor drains: this block's input boxes, and one weight box per block, on their way into L2
+  if (!p.prefetch) {
+  } else if (warp == 0) {
+    if (elect_one()) {
+      for (int u = unit0; u < num_tiles; u += unit_step) {
+        uint32_t tm, tn, img, ti;
+        p.div_tiles_n.divmod(static_cast<uint32_t>(u), tm, tn);
+        p.div_tpi.divmod(tm * CTAS + rank, img, ti);
+        for (int cc = 0; cc < p.cchunks; ++cc)
+          tma_prefetch_4d(&map_a, cc * kBK, -p.pw, static_cast<int>(ti) * p.R - p.ph, static_cast<int>(img));
+      }
+    }
+  } else if (warp == 6) {
+    if (elect_one()) {
+      const int groups = p.cchunks * p.groups_per_chunk;
+      for (int b = static_cast<int>(blockIdx.x); b < groups * p.tiles_n; b += static_cast<int>(gridDim.x)) {
+        const int tn = b / groups, gi = b - tn * groups, cc = gi / p.groups_per_chunk, g = gi - cc * p.groups_per_chunk;
+        for (int half = 0; half < CTAS; ++half)
+          tma_prefetch_4d(&map_b, 0, tn * BN + half * (BN / CTAS), cc, g * p.tg);
+      }
+    }
+  }
+  pdl_wait();
+  pdl_launch_dependents();
 
   if (warp == 0) {
     // ---------------- A producer: one input box per (tile, 64-channel chunk) ----------------
@@ -1926,6 +2000,7 @@ int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams
     attr_set = true;
   }
   if (p.ksplit < 1) { p.ksplit = 1; p.kper = p.kblocks; }
+  p.prefetch = pre ? 0 : 1;
   p.div_ksplit.set(p.ksplit);
   p.div_tiles_n.set(p.tiles_n);
   p.div_wo.set(p.Wo > 0 ? p.Wo : 1);
@@ -2267,6 +2342,7 @@ int run_halo(const HaloPlan& hp, const DotProblem& d, int64_t Cp, const uint16_t
   p.groups_per_chunk = p.Kh * (p.Kw / hp.tg);
   p.ph = static_cast<int>(d.ph_lo); p.pw = static_cast<int>(d.pw_lo);
   p.sa_stages = hp.sa; p.sb_stages = hp.sb; p.b_resident = hp.resident;
+  p.prefetch = pre ? 0 : 1;
   p.a_bytes = static_cast<uint32_t>(kBK * 2 * hp.Wb * hp.RB);
   p.b_bytes = static_cast<uint32_t>(hp.tg * (hp.bn / hp.ctas) * kBK * 2);
   p.div_tiles_n.set(p.tiles_n);
