@@ -1496,8 +1496,6 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  pdl_wait();
-  pdl_launch_dependents();
 
   const int npx = static_cast<int>(p.seg_bytes >> (p.cp_log2 + 1));   // pixels of a run
   const int epx = p.channels_last ? p.C : 1;                          // elements per pixel in one raw copy
@@ -1511,8 +1509,9 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
   const int nnew_later = min(p.Kh, p.Sh);           // rows a tile adds (the first tile adds all Kh)
   const int w_first = static_cast<int>(seg) * (kBM * p.Sw) - p.pw;   // input column of run pixel 0
   const int w_lo = max(w_first, 0), w_hi = min(w_first + npx, p.W);
-  // raw copies of tile t into raw stage r: lane i takes copy i = (new row, raw segment); called by warp 0
-  auto copy_tile = [&](int t, uint32_t r) {
+  // raw copies of tile t into raw stage r: lane i takes copy i = (new row, raw segment); called by warp 0.
+  // With `only_prefetch` the same stretches are merely requested into L2 (before the dependency wait).
+  auto copy_tile = [&](int t, uint32_t r, bool only_prefetch) {
     uint32_t j_l, c_l;
     p.div_nseg.divmod(static_cast<uint32_t>(lane), j_l, c_l);
     const int nnew = t == 0 ? p.Kh : nnew_later;
@@ -1526,6 +1525,12 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
       a0 = b0 & ~static_cast<int64_t>(15);                              // whole 16-byte pieces around the stretch;
       size = static_cast<uint32_t>(((b1 + 15) & ~static_cast<int64_t>(15)) - a0);   // the tensor's byte count is a multiple of 16
     }
+    if (only_prefetch) {
+      if (size)
+        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<uint64_t>(x) + static_cast<uint64_t>(a0)),
+                     "r"(size) : "memory");
+      return;
+    }
     const uint32_t total = __reduce_add_sync(0xffffffffu, size);
     if (lane == 0) mbar_expect_tx(bar_rfull + 8 * r, total);
     __syncwarp();
@@ -1533,7 +1538,19 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
       bulk_copy_g2s(r_base + r * p.raw_stage_bytes + j_l * p.raw_row_bytes + c_l * p.raw_seg_bytes,
                     reinterpret_cast<const unsigned char*>(x) + a0, size, bar_rfull + 8 * r);
   };
-  if (warp == 0 && ntiles > 0) copy_tile(0, 0);   // in flight while the block arranges the weights
+  // while the predecessor drains: the rows of the first two tiles and the weights on their way into L2
+  if (warp == 0) {
+    for (int t = 0; t < min(ntiles, 2); ++t) copy_tile(t, 0, true);
+  } else if (warp == 1) {
+    const uint32_t wbytes = (static_cast<uint32_t>(p.w_elems) * 2u) & ~15u, piece = ((wbytes / 32u) + 15u) & ~15u;
+    const uint32_t at = static_cast<uint32_t>(lane) * piece;
+    if (piece && at < wbytes)
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(reinterpret_cast<uint64_t>(wt) + at),
+                   "r"(min(piece, wbytes - at)) : "memory");
+  }
+  pdl_wait();
+  pdl_launch_dependents();
+  if (warp == 0 && ntiles > 0) copy_tile(0, 0, false);   // in flight while the block arranges the weights
 
   // ---- weights into operand order [kh][K chunk j][row o < bn][8 elements]: element kw * cp + c of filter row
   // kh sits at (j, i) = ((kw * cp + c) / 8, (kw * cp + c) % 8), zeros elsewhere.  The weight tensor is first
@@ -1580,7 +1597,7 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
     uint32_t r = 1 % static_cast<uint32_t>(p.raw_stages), ph = p.raw_stages == 1 ? 1u : 0u;
     for (int t = 1; t < ntiles; ++t) {
       if (!mbar_wait(bar_rempty + 8 * r, ph ^ 1u, abort_flag)) break;
-      copy_tile(t, r);
+      copy_tile(t, r, false);
       if (++r == static_cast<uint32_t>(p.raw_stages)) { r = 0; ph ^= 1u; }
     }
   } else if (warp >= 6) {
