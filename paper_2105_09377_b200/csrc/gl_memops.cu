@@ -974,10 +974,18 @@ __global__ void __launch_bounds__(kThreads) item_max(const float* __restrict__ i
 }
 
 __global__ void __launch_bounds__(kThreads) relu_vec(const float4* __restrict__ in, float4* __restrict__ out, int64_t n4) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  // while the predecessor drains, the lines of this thread's first trip are requested into L2 (a prefetch consumes
+  // nothing; a line the predecessor still writes is updated in L2, where all writes meet)
+  {
+    const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (i + j * stride < n4) asm volatile("prefetch.global.L2 [%0];" ::"l"(in + i + j * stride) : "memory");
+  }
   pdl_wait();
   pdl_launch_dependents();
   // four independent 16-byte loads in flight per thread
-  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += 4 * stride) {
     float4 v[4];
 #pragma unroll
