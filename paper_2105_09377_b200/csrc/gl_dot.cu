@@ -189,9 +189,28 @@ __global__ void __launch_bounds__(256) nchw_prepass(const uint16_t* __restrict__
                                                     const uint16_t* __restrict__ w, uint16_t* __restrict__ ws,
                                                     const PrepassParams p) {
   extern __shared__ uint16_t pre_smem[];
+  int b = blockIdx.x;
+  // While the predecessor drains, an activation block requests the lines of its loads into L2 (a prefetch
+  // consumes nothing; a line that is still being written is updated in L2, where all writes meet).
+  if (b < p.x_blocks) {
+    const int pt0 = static_cast<int>(fdiv(static_cast<uint32_t>(b), p.by_tiles_c));
+    const int c00 = (b - pt0 * p.tiles_c) * 64;
+    const int npix0 = p.Hs * p.Ws;
+    const int64_t HW0 = static_cast<int64_t>(p.H) * p.W;
+    // one line per (channel, 32-pixel stretch): thread t takes channel t / 4 and stretch t % 4 of the tile's 64
+    // pixels (for strided windows the stretch covers Sw times as many input pixels: two lines)
+    const int ch = threadIdx.x >> 2, part = threadIdx.x & 3;
+    const int64_t gp = static_cast<int64_t>(pt0) * 64 + 16 * part;
+    if (gp < p.total_pix && c00 + ch < p.C) {
+      const int64_t n = p.fast ? static_cast<int64_t>(fdiv(static_cast<uint32_t>(gp), p.by_npix)) : gp / npix0;
+      const int pix = static_cast<int>(gp - n * npix0);
+      const int hs = static_cast<int>(fdiv(static_cast<uint32_t>(pix), p.by_Ws)), wsx = pix - hs * p.Ws;
+      const uint16_t* at = x + (n * p.C + c00 + ch) * HW0 + static_cast<int64_t>(hs) * p.Sh * p.W + wsx * p.Sw;
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(at) : "memory");
+    }
+  }
   pdl_wait();
   pdl_launch_dependents();
-  int b = blockIdx.x;
   if (b >= p.x_blocks) {
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     if (wid >= p.wwarps) return;
