@@ -1431,6 +1431,7 @@ struct RowRunParams {
   int64_t O;
   int relu;
   int out_bf16;   // results rounded to bf16 (O a multiple of 8)
+  int out_nchw;   // results stored as (N, O, H', W'): squeeze + transpose (0 3 1 2) of Fig. 2a fused
   int C, H, W, Ho, Wo, Sh, Sw, Kh, Kw, ph, pw;
   int cp_log2;                  // pixels are widened to 8 / Sw = 2^cp_log2 channels
   int channels_last;            // items (H,W,C) / (Kh,Kw,C), else (C,H,W) / (C,Kh,Kw)
@@ -1735,7 +1736,7 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
       const uint32_t row = img * static_cast<uint32_t>(p.Ho) + static_cast<uint32_t>(ho0 + t);   // output row of the (N*Ho, Wo, O) view
       if (!mbar_wait(bar_tfull + 8 * acc, aph, abort_flag)) { ok = false; break; }
       tc_fence_after();
-      const int cstep = p.out_bf16 ? 64 : 32;   // a staged row is 128 bytes: 32 fp32 or 64 bf16 columns
+      const int cstep = (p.out_bf16 && !p.out_nchw) ? 64 : 32;   // a staged row is 128 bytes: 32 fp32 or 64 bf16 columns
 #pragma unroll 1
       for (int c = 0; c < p.bn; c += cstep) {
         if (c >= p.O) break;   // uniform across the warp
@@ -1744,6 +1745,34 @@ conv_rowrun(const uint16_t* __restrict__ x, const uint16_t* __restrict__ wt,
         if (p.relu) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(fmaxf(__uint_as_float(r[i]), 0.f));
+        }
+        if (p.out_nchw) {
+          // squeeze + transpose fused: the 32 pixels x 32 channels block is parked channel-major (a lane writes
+          // its pixel's value into every channel row: 32 lanes = one contiguous row piece, no bank conflict)
+          // and leaves as one box {32 pixels, 1 row, 32 channels, 1 image} of the (W', H', O, N) view
+          const uint32_t buf = epi_base + q * 4096;
+          if (leader) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+          __syncwarp();
+          if (p.out_bf16) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              asm volatile("st.shared.b16 [%0], %1;" ::"r"(buf + i * 64 + lane * 2), "h"(f32_to_bf16(__uint_as_float(r[i]))) : "memory");
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              asm volatile("st.shared.b32 [%0], %1;" ::"r"(buf + i * 128 + lane * 4), "r"(r[i]) : "memory");
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (leader) {   // pixels past W' and channels past O are clipped
+            asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];" ::"l"(
+                             reinterpret_cast<uint64_t>(&map_c)),
+                         "r"(static_cast<int>(seg) * kBM + q * 32), "r"(ho0 + t), "r"(c), "r"(static_cast<int>(img)), "r"(buf)
+                         : "memory");
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          }
+          ++chunk_it;
+          continue;
         }
         if (p.out_bf16) {
 #pragma unroll
@@ -1984,6 +2013,19 @@ bool encode_result_rows(CUtensorMap* m, float* base, int64_t rows, int64_t Wo, i
   return encode_tiled_cached(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE);
 }
 
+// Result of the fused squeeze + transpose, (N, O, H', W') viewed as (W', H', O, N): boxes of 32 pixels of one
+// output row x 32 channels, stored channel-major and un-swizzled.
+bool encode_result_nchw(CUtensorMap* m, float* base, int64_t N, int64_t O, int64_t Ho, int64_t Wo, bool bf16) {
+  const cuuint64_t es = bf16 ? 2 : 4;
+  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(Wo), static_cast<cuuint64_t>(Ho), static_cast<cuuint64_t>(O),
+                              static_cast<cuuint64_t>(N)};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(Wo) * es, static_cast<cuuint64_t>(Ho * Wo) * es,
+                                 static_cast<cuuint64_t>(O * Ho * Wo) * es};
+  const cuuint32_t box[4] = {32, 1, 32, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return encode_tiled_cached(m, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, base, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE);
+}
+
 // Row-window activations (N*Hp, Wpa, Cp): dimension 1 walks output columns with a stride of
 // Sw*Cp elements, shorter than the 64 elements of dimension 0 (the windows overlap).
 bool encode_rowwin(CUtensorMap* m, const void* base, int64_t rows, int64_t Wo, int64_t Wpa, int64_t Cp, int64_t Sw) {
@@ -2174,7 +2216,9 @@ ConvPlan plan_conv(const DotProblem& d, uint32_t flags) {
                     d.Kh * d.Kw * pl.Cp < (1ll << 31);
   pl.tc = fits && ((d.M + 127) / 128) * ((d.O + 63) / 64) < (1ll << 28);
   pl.prepass = !d.channels_last || pl.Cp != d.C;
-  if (pl.tc && !(flags & GL_OUT_NCHW) && (d.Sw == 1 || d.Sw == 2 || d.Sw == 4 || d.Sw == 8) && d.C <= 8 / d.Sw &&
+  // (with the fused squeeze + transpose the result rows are runs of W' pixels: whole 16-byte pieces)
+  if (pl.tc && (!(flags & GL_OUT_NCHW) || (d.Wo * ((flags & GL_OUT_BF16) ? 2 : 4)) % 16 == 0) &&
+      (d.Sw == 1 || d.Sw == 2 || d.Sw == 4 || d.Sw == 8) && d.C <= 8 / d.Sw &&
       d.O % ((flags & GL_OUT_BF16) ? 8 : 4) == 0 && d.O <= 128 && d.Kh <= 16 && d.Wo < (1ll << 24) &&
       d.N * d.Ho * ((d.Wo + kBM - 1) / kBM) < (1ll << 31) &&
       (d.N * d.C * d.H * d.W) % 8 == 0 &&                    // raw rows are copied as whole 16-byte pieces
@@ -2563,7 +2607,7 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
   if (pl.rowrun) {
     RowRunParams rp;
     std::memset(&rp, 0, sizeof(rp));
-    rp.O = d.O; rp.relu = relu; rp.out_bf16 = out_bf16;
+    rp.O = d.O; rp.relu = relu; rp.out_bf16 = out_bf16; rp.out_nchw = out_nchw;
     rp.C = static_cast<int>(d.C); rp.H = static_cast<int>(d.H); rp.W = static_cast<int>(d.W);
     rp.Ho = static_cast<int>(d.Ho); rp.Wo = static_cast<int>(d.Wo);
     rp.Sh = static_cast<int>(d.Sh); rp.Sw = static_cast<int>(d.Sw);
@@ -2597,7 +2641,9 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     rp.div_segs.set(rp.segs);
     rp.div_ho.set(d.Ho);
     CUtensorMap mc;
-    if (!encode_result_rows(&mc, dst, d.N * d.Ho, d.Wo, d.O, out_bf16 != 0)) return GL_ERR_CUDA;
+    if (out_nchw ? !encode_result_nchw(&mc, dst, d.N, d.O, d.Ho, d.Wo, out_bf16 != 0)
+                 : !encode_result_rows(&mc, dst, d.N * d.Ho, d.Wo, d.O, out_bf16 != 0))
+      return GL_ERR_CUDA;
     const int smem = 1024 + kRunEpiBytes + static_cast<int>((rp.b_bytes + 127u) & ~127u) +
                      rp.ring * static_cast<int>(rp.slot_bytes) + rp.raw_stages * static_cast<int>(rp.raw_stage_bytes) + 256;
     static bool attr_set_dev[64] = {false};

@@ -573,6 +573,41 @@ def test_full_size_conv_fused_squeeze_transpose(gl, cfg, layout):
     assert np.array_equal(out.tensor.cpu().numpy(), ref.transpose(0, 3, 1, 2))
 
 
+FEW_CHANNEL_NCHW = [
+    # n, c, h, w, o, k, stride, pad: few input channels, so the row-strip kernel takes them
+    (2, 3, 38, 40, 24, 7, 2, 3),      # W' = 20: fp32 rows are whole 16-byte pieces, bf16 rows are not (other kernel)
+    (2, 3, 30, 64, 40, 7, 2, 3),      # W' = 32, 40 filters: second channel box clipped at O
+    (1, 4, 20, 288, 16, 3, 2, 1),     # W' = 144: two pixel segments per row, the second ragged
+    (3, 8, 9, 16, 128, 3, 1, 1),      # stride 1, 8 channels, all 128 accumulator columns
+    (2, 1, 17, 48, 8, 5, 1, 2),       # one channel, 5x5
+]
+
+
+@pytest.mark.parametrize("layout", ["nchw", "nhwc"])
+@pytest.mark.parametrize("case", FEW_CHANNEL_NCHW)
+def test_few_channel_conv_fused_squeeze_transpose(gl, case, layout):
+    # Fig. 2a's whole program, (N,C,H,W) in and (N,O,H',W') out, on stem-like shapes, fp32 and bf16 results
+    n, c, h, w, o, k, s, pad = case
+    x = synth.uniform_int(47, 1, (n, c, h, w), -3, 3)
+    wt = synth.uniform_int(47, 2, (o, c, k, k), -3, 3)
+    ref = _conv_ref(x, wt, (s, s), (pad, pad)).transpose(0, 3, 1, 2)
+    if layout == "nhwc":
+        xa = gl.AccessPattern(to_bf16_device(np.ascontiguousarray(x.transpose(0, 2, 3, 1))), 1)
+        wa = gl.AccessPattern(to_bf16_device(np.ascontiguousarray(wt.transpose(0, 2, 3, 1))), 1)
+        spec = gl.windows_spec((k, k, c), (s, s, 1), (pad, pad, 0), (pad, pad, 0))
+    else:
+        xa, wa = gl.AccessPattern(to_bf16_device(x), 1), gl.AccessPattern(to_bf16_device(wt), 1)
+        spec = gl.windows_spec((c, k, k), (1, s, s), (0, pad, pad), (0, pad, pad))
+    for flags in (0, gl.GL_EPILOGUE_RELU, gl.GL_OUT_BF16, gl.GL_OUT_BF16 | gl.GL_EPILOGUE_RELU):
+        out = gl.gl_cartesian_dot(xa, spec, wa, flags=flags | gl.GL_OUT_NCHW)
+        _ok(gl)
+        assert tuple(out.tensor.shape) == ref.shape
+        want = np.maximum(ref, 0.0) if flags & gl.GL_EPILOGUE_RELU else ref
+        if flags & gl.GL_OUT_BF16:
+            want = _bf16(want)
+        assert np.array_equal(out.tensor.float().cpu().numpy().astype(np.float64), want), "flags=%d" % flags
+
+
 @pytest.mark.parametrize("cfg", FULL_CONVS, ids=[c.name for c in FULL_CONVS])
 def test_full_size_conv_bf16_results(gl, cfg):
     # GL_OUT_BF16 at full size: the exact integer sums rounded once to the nearest-even bf16
