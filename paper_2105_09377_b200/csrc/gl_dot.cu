@@ -614,7 +614,42 @@ struct TcParams {
   // kRowWin only: one tile = (up to) 128 outputs of one output row
   int Hp, segs;           // padded input rows per image; 128-wide segments per output row
   FastDiv div_segs, div_ho;
+  // Pairs only: tiles of two widths.  When the tile count is not a multiple of the resident pairs the last
+  // wave is partly empty; replacing some BN-wide tiles by half-wide ones evens the pairs' loads out.  Row band
+  // tm holds w(tm) = wA (tm < bA) or wA - 1 wide tiles from column 0 on, then half-wide tiles up to O.  Units
+  // count the wide tiles of all bands first (n_wide of them), then the half-wide ones (nA per band for
+  // tm < bA, nA + 2 per later band).
+  int mix, n_wide, wA, bA, nA;
 };
+
+struct TileAt { int tm, n0, width; };
+
+// Work unit (without the K-split index) -> row band, first column and width of its tile.
+template <int BN>
+__device__ __forceinline__ TileAt decode_tile(const TcParams& p, uint32_t t) {
+  TileAt at;
+  if (!p.mix) {
+    uint32_t tm, tn;
+    p.div_tiles_n.divmod(t, tm, tn);
+    at.tm = static_cast<int>(tm); at.n0 = static_cast<int>(tn) * BN; at.width = BN;
+    return at;
+  }
+  const int u = static_cast<int>(t);
+  if (u < p.n_wide) {
+    const int first = p.bA * p.wA;
+    int j;
+    if (u < first) { at.tm = u / p.wA; j = u - at.tm * p.wA; }
+    else { const int v = u - first, w = p.wA - 1; at.tm = v / w; j = v - at.tm * w; at.tm += p.bA; }
+    at.n0 = j * BN; at.width = BN;
+    return at;
+  }
+  const int v = u - p.n_wide, first = p.bA * p.nA;
+  int j;
+  if (v < first) { at.tm = v / p.nA; j = v - at.tm * p.nA; at.n0 = p.wA * BN + j * (BN / 2); }
+  else { const int x = v - first, n = p.nA + 2; at.tm = x / n; j = x - at.tm * n; at.tm += p.bA; at.n0 = (p.wA - 1) * BN + j * (BN / 2); }
+  at.width = BN / 2;
+  return at;
+}
 
 // A stage holds G K-blocks of 64 (G A sub-tiles, then G B sub-tiles) behind one pair of barriers.
 // OCC = blocks per SM the configuration is sized for (2 only for BN <= 128: TMEM has 512 columns).
@@ -690,22 +725,25 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
   else __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int num_tiles = p.tiles_m * p.tiles_n * p.ksplit;   // work units (p.tiles_m counts 128*CTAS-row tiles)
+  // work units (p.tiles_m counts 128*CTAS-row tiles)
+  const int num_tiles = p.mix ? p.n_wide + p.bA * p.nA + (p.tiles_m - p.bA) * (p.nA + 2) : p.tiles_m * p.tiles_n * p.ksplit;
   const int unit0 = static_cast<int>(blockIdx.x) / CTAS, unit_step = static_cast<int>(gridDim.x) / CTAS;
   // while the predecessor drains: the operands of this block's first unit (at most 4 K blocks of it) on their
   // way into L2
   if (p.prefetch && (MODE == kDense || MODE == kIm2col) && (warp == 0 || warp == 6) && unit0 < num_tiles) {
     if (elect_one()) {
-      uint32_t t, ks, tm, tn;
+      uint32_t t, ks;
       p.div_ksplit.divmod(static_cast<uint32_t>(unit0), t, ks);
-      p.div_tiles_n.divmod(t, tm, tn);
+      const TileAt at = decode_tile<BN>(p, t);
       const int kb_begin = static_cast<int>(ks) * p.kper, kb_end = min(min(p.kblocks, kb_begin + p.kper), kb_begin + 4);
-      const int m0 = (static_cast<int>(tm) * CTAS + static_cast<int>(rank)) * kBM;
-      const int n0 = static_cast<int>(tn) * BN + static_cast<int>(rank) * (BN / CTAS);
+      const int m0 = (at.tm * CTAS + static_cast<int>(rank)) * kBM;
+      const int n0 = at.n0 + static_cast<int>(rank) * (at.width / CTAS);
+      constexpr int kBoxesB = CTAS == 2 ? 2 : 1;   // pairs: B boxes are BN/4 rows high
       if (MODE == kDense) {
         for (int kb = kb_begin; kb < kb_end; ++kb) {
           if (warp == 0) tma_prefetch_2d(&map_a, kb * kBK, m0);
-          else tma_prefetch_2d(&map_b, kb * kBK, n0);
+          else
+            for (int h = 0; h < kBoxesB; ++h) tma_prefetch_2d(&map_b, kb * kBK, n0 + h * (BN / 4));
         }
       } else {
         uint32_t im, rem, ho, wo;
@@ -718,7 +756,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
             tma_prefetch_im2col(&map_a, cc * kBK, static_cast<int>(wo) * p.Sw - p.pw, static_cast<int>(ho) * p.Sh - p.ph,
                                 static_cast<int>(im), static_cast<uint16_t>(kw), static_cast<uint16_t>(kh));
           else
-            tma_prefetch_2d(&map_b, (kh * p.Kw + kw) * p.Cp + cc * kBK, n0);
+            for (int h = 0; h < kBoxesB; ++h) tma_prefetch_2d(&map_b, (kh * p.Kw + kw) * p.Cp + cc * kBK, n0 + h * (BN / 4));
           if (++cc == p.cchunks) { cc = 0; if (++kw == p.Kw) { kw = 0; ++kh; } }
         }
       }
@@ -739,13 +777,16 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
       uint32_t s = 0, ph = 0;   // ring slot and its phase, advanced by hand (no division in this loop)
       bool ok = true;
       for (int u = unit0; u < num_tiles && ok; u += unit_step) {
-        uint32_t t, ks, tm, tn;
+        uint32_t t, ks;
         p.div_ksplit.divmod(static_cast<uint32_t>(u), t, ks);
-        p.div_tiles_n.divmod(t, tm, tn);
+        const TileAt at = decode_tile<BN>(p, t);
+        const uint32_t tm = static_cast<uint32_t>(at.tm);
         const int kb_begin = static_cast<int>(ks) * p.kper, kb_end = min(p.kblocks, kb_begin + p.kper);
-        // this block's 128 rows of A and its BN/CTAS rows of B
-        const int m0 = (static_cast<int>(tm) * CTAS + static_cast<int>(rank)) * kBM;
-        const int n0 = static_cast<int>(tn) * BN + static_cast<int>(rank) * (BN / CTAS);
+        // this block's 128 rows of A and its share of the tile's rows of B (pairs fetch B in boxes of BN/4 rows:
+        // two per K block for a full-width tile, one for a half-width tile)
+        const int m0 = (at.tm * CTAS + static_cast<int>(rank)) * kBM;
+        const int n0 = at.n0 + static_cast<int>(rank) * (at.width / CTAS);
+        const int b_bytes = CTAS == 2 ? (at.width == BN ? Cfg::kStageB : Cfg::kStageB / 2) : Cfg::kStageB;
         int wbase = 0, hbase = 0, img = 0;
         if (MODE == kRowWin) {
           if (load_a) {   // tile -> (output row, segment) -> first padded input row
@@ -776,7 +817,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
           const uint32_t full = CTAS == 2 ? map_to_cta(bar_full + 8 * s, 0) : bar_full + 8 * s;
           const uint32_t stage = tiles + s * Cfg::kStage;
           const int nsub = min(G, kb_end - kb0);
-          if (rank == 0 && leader) mbar_expect_tx(bar_full + 8 * s, nsub * CTAS * (load_a ? Cfg::kStageA : Cfg::kStageB));
+          if (rank == 0 && leader) mbar_expect_tx(bar_full + 8 * s, nsub * CTAS * (load_a ? Cfg::kStageA : b_bytes));
 #pragma unroll 1
           for (int j = 0; j < nsub; ++j) {
             const int kb = kb0 + j;
@@ -785,13 +826,19 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
             if (CTAS == 2) {
               if (MODE == kDense) {
                 if (load_a) tma_load_2d_pair(sa, &map_a, kb * kBK, m0, full);
-                else tma_load_2d_pair(sb, &map_b, kb * kBK, n0, full);
+                else {
+                  tma_load_2d_pair(sb, &map_b, kb * kBK, n0, full);
+                  if (at.width == BN) tma_load_2d_pair(sb + Cfg::kStageB / 2, &map_b, kb * kBK, n0 + BN / 4, full);
+                }
               } else {
                 if (load_a)
                   tma_load_im2col_pair(sa, &map_a, cc * kBK, wbase, hbase, img, static_cast<uint16_t>(kw),
                                        static_cast<uint16_t>(kh), full);
-                else
-                  tma_load_2d_pair(sb, &map_b, (kh * p.Kw + kw) * p.Cp + cc * kBK, n0, full);
+                else {
+                  const int kx = (kh * p.Kw + kw) * p.Cp + cc * kBK;
+                  tma_load_2d_pair(sb, &map_b, kx, n0, full);
+                  if (at.width == BN) tma_load_2d_pair(sb + Cfg::kStageB / 2, &map_b, kx, n0 + BN / 4, full);
+                }
               }
             } else if (MODE == kDense) {
               if (load_a) tma_load_2d(sa, &map_a, kb * kBK, m0, full);
@@ -834,7 +881,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
     // ---------------- MMA issuer ----------------
     if (rank == 0) {
       const bool leader = elect_one();   // the loop is warp-uniform; this lane issues the MMAs and commits
-      constexpr uint32_t idesc = make_idesc(kBM * CTAS, BN);
+      constexpr uint32_t idesc_wide = make_idesc(kBM * CTAS, BN), idesc_half = make_idesc(kBM * CTAS, BN / 2);
       const uint64_t desc_a0 = (MODE == kIm2colGranule) ? make_desc(tiles, kBM * 16, 128, 0) : make_desc(tiles, 16, 1024, 2);
       const uint64_t desc_b0 = (MODE == kIm2colGranule) ? make_desc(tiles + G * Cfg::kStageA, BN * 16, 128, 0)
                                                         : make_desc(tiles + G * Cfg::kStageA, 16, 1024, 2);
@@ -844,6 +891,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
         const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
         uint32_t t, ks;
         p.div_ksplit.divmod(static_cast<uint32_t>(u), t, ks);
+        const uint32_t idesc = (CTAS == 2 && p.mix && static_cast<int>(t) >= p.n_wide) ? idesc_half : idesc_wide;
         const int kb_begin = static_cast<int>(ks) * p.kper, kb_end = min(p.kblocks, kb_begin + p.kper);
         if (!mbar_wait(bar_tempty + 8 * acc, aph ^ 1u, abort_flag)) { ok = false; break; }
         tc_fence_after();
@@ -896,11 +944,12 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
     const uint32_t stage_buf = epi_base + q * (Cfg::kEpiBufs * 4096);   // this warp's 32 rows x 128 bytes tiles
     for (int u = unit0; u < num_tiles && ok; u += unit_step, ++tile_it) {
       const uint32_t acc = tile_it & 1u, aph = (tile_it >> 1) & 1u;
-      uint32_t t, ks, tmu, tnu;
+      uint32_t t, ks;
       p.div_ksplit.divmod(static_cast<uint32_t>(u), t, ks);
-      p.div_tiles_n.divmod(t, tmu, tnu);
+      const TileAt at = decode_tile<BN>(p, t);
+      uint32_t tmu = static_cast<uint32_t>(at.tm);
       if (CTAS == 2) tmu = tmu * CTAS + rank;   // this block's 128 rows of the pair's tile
-      const int tm = static_cast<int>(tmu), tn = static_cast<int>(tnu);
+      const int tm = static_cast<int>(tmu);
       if (!mbar_wait(bar_tfull + 8 * acc, aph, abort_flag)) { ok = false; break; }
       tc_fence_after();
       int64_t m = static_cast<int64_t>(tm) * kBM + q * 32 + lane;
@@ -924,8 +973,8 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
       // bf16 results through TMA stores go 64 columns at a time (128 bytes per row, as 32 fp32 columns do)
       const int cstep = (p.out_bf16 && p.tma_store) ? 64 : 32;
 #pragma unroll 1
-      for (int c = 0; c < BN; c += cstep) {
-        const int64_t n0 = static_cast<int64_t>(tn) * BN + c;
+      for (int c = 0; c < at.width; c += cstep) {
+        const int64_t n0 = static_cast<int64_t>(at.n0) + c;
         if (n0 >= p.O) break;   // uniform across the warp
         uint32_t r[32];
         tc_load_32cols(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * BN + c, r);
@@ -2042,6 +2091,35 @@ bool encode_rowwin(CUtensorMap* m, const void* base, int64_t rows, int64_t Wo, i
 using PreLaunch = std::function<int()>;
 inline int run_pre(const PreLaunch& pre) { return pre ? pre() : GL_OK; }
 
+// Pairs: how many full-width tiles to keep so that, with units dealt out in turn (wide ones first), the most
+// loaded pair has as little as possible.  Loads count half-width columns: a wide tile is 2, a half-wide tile 1.
+// Sets p->mix and its fields when that beats all-wide tiles; returns the number of work units.
+int plan_tile_mix(TcParams* p, int bn, int pairs) {
+  const int bands = p->tiles_m, all_wide = bands * p->tiles_n;
+  const int cu = static_cast<int>((p->O + bn / 2 - 1) / (bn / 2));   // half-wide columns per band
+  if (pairs < 1 || cu < 2) return all_wide;
+  const int old_span = 2 * ((all_wide + pairs - 1) / pairs);
+  const int64_t units = static_cast<int64_t>(bands) * cu;
+  const int span = static_cast<int>((units + pairs - 1) / pairs);
+  const int wide = static_cast<int>(std::min<int64_t>(static_cast<int64_t>(pairs) * (span / 2), static_cast<int64_t>(bands) * (cu / 2)));
+  const int64_t narrow = units - 2 * static_cast<int64_t>(wide);
+  // dealing in turn: pair q gets wide tiles q, q + pairs, ...; the half-wide ones carry on from pair wide % pairs
+  int worst = 0;
+  for (int q = 0; q < pairs; ++q) {
+    const int nw = wide / pairs + (q < wide % pairs ? 1 : 0);
+    const int64_t first = ((q - wide % pairs) % pairs + pairs) % pairs;
+    const int nn = narrow > first ? static_cast<int>((narrow - first + pairs - 1) / pairs) : 0;
+    worst = std::max(worst, 2 * nw + nn);
+  }
+  if (worst >= old_span || wide < 1) return all_wide;
+  p->mix = 1;
+  p->n_wide = wide;
+  p->wA = (wide + bands - 1) / bands;
+  p->bA = wide - bands * (p->wA - 1);          // bands with wA wide tiles; the rest have wA - 1
+  p->nA = cu - 2 * p->wA;
+  return wide + static_cast<int>(narrow);
+}
+
 template <int BN, int MODE, int G, int OCC, int CTAS = 1>
 int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams p, cudaStream_t st, const PreLaunch& pre) {
   using Cfg = TcCfg<BN, G, OCC, CTAS>;
@@ -2096,7 +2174,9 @@ int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams
   } else {
     mc = ma;   // unused by the kernel; any valid map
   }
-  const int tiles = p.tiles_m * p.tiles_n * p.ksplit;
+  int tiles = p.tiles_m * p.tiles_n * p.ksplit;
+  p.mix = 0;
+  if (CTAS == 2 && p.ksplit == 1) tiles = plan_tile_mix(&p, BN, std::min(max_pairs_dev[dev], num_sms() / 2));
   if (const int rc = run_pre(pre)) return rc;
   if (CTAS == 2) {
     const int pairs = std::min(tiles, std::min(max_pairs_dev[dev], num_sms() / 2));
@@ -2111,7 +2191,8 @@ int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams
 }
 
 // Wide tiles of a large problem are bound by operand traffic from L2 to the SMs; a pair of blocks
-// sharing a 256x256 tile loads a third less per flop.  (The B tensor map then has boxes of bn/2 rows.)
+// sharing a 256x256 tile loads a third less per flop.  (The B tensor map then has boxes of bn/4 rows: two per
+// block and K block for a full-width tile, one for a half-width tile.)
 bool use_pair(int mode, int bn, const TcParams& p) {
   return bn == 256 && (mode == kDense || mode == kIm2col) && p.ksplit <= 1 && p.tiles_m >= 2;
 }
@@ -2596,7 +2677,7 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     p.K = d.K;
     p.kblocks = static_cast<int>((d.K + kBK - 1) / kBK);
     if (!encode_kmajor_sw128(&ma, pa, d.M, d.K, kBM) ||
-        !encode_kmajor_sw128(&mb, pb, d.O, d.K, use_pair(kDense, bn, p) ? bn / 2 : bn))
+        !encode_kmajor_sw128(&mb, pb, d.O, d.K, use_pair(kDense, bn, p) ? bn / 4 : bn))
       return GL_ERR_CUDA;
     return finish(launch_tc_bn<kDense>(bn, ma, mb, dst, p, st, PreLaunch()));
   }
@@ -2754,7 +2835,7 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     p.K = Cp;
     p.kblocks = static_cast<int>((Cp + kBK - 1) / kBK);
     if (!encode_kmajor_sw128(&ma, x, d.M, Cp, kBM) ||
-        !encode_kmajor_sw128(&mb, wt, d.O, Cp, use_pair(kDense, bn, p) ? bn / 2 : bn))
+        !encode_kmajor_sw128(&mb, wt, d.O, Cp, use_pair(kDense, bn, p) ? bn / 4 : bn))
       return GL_ERR_CUDA;
     return finish(launch_tc_bn<kDense>(bn, ma, mb, dst, p, st, pre));
   }
@@ -2769,7 +2850,7 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     p.cchunks = static_cast<int>((Cp + kBK - 1) / kBK);
     p.kblocks = static_cast<int>(taps) * p.cchunks;
     if (!encode_im2col(&ma, x, d, Cp, kBK, true) ||
-        !encode_kmajor_sw128(&mb, wt, d.O, p.K, use_pair(kIm2col, bn, p) ? bn / 2 : bn))
+        !encode_kmajor_sw128(&mb, wt, d.O, p.K, use_pair(kIm2col, bn, p) ? bn / 4 : bn))
       return GL_ERR_CUDA;
     return finish(launch_tc_bn<kIm2col>(bn, ma, mb, dst, p, st, pre));
   }

@@ -365,8 +365,9 @@ def test_dense_integer_bit_exact(gl, m, o, k):
 
 
 # Problems large enough for 256-wide tiles, which run on pairs of blocks sharing a 256x256 tile:
-# an odd number of 128-row tiles (the last pair has an empty half), ragged edges in both directions.
-DENSE_PAIRED = [(2600, 1930, 200), (4001, 1100, 136), (2305, 2309, 72)]
+# an odd number of 128-row tiles (the last pair has an empty half), ragged edges in both directions.  The tile
+# counts are not multiples of the resident pairs, so part of each result is computed as half-width tiles.
+DENSE_PAIRED = [(2600, 1930, 200), (4001, 1100, 136), (2305, 2309, 72), (2560, 3900, 72)]
 
 
 @pytest.mark.parametrize("m,o,k", DENSE_PAIRED)
