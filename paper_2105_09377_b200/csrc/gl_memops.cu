@@ -959,6 +959,68 @@ __global__ void __launch_bounds__(256) window_max_3x3s2(const float* __restrict_
   }
 }
 
+// The same pooling on 2-byte planes (rows that are multiples of eight values): a thread owns eight input
+// columns (four outputs) of one strip of R output rows.  bf16 values are compared as the floats they stand for
+// (a shift), so the maximum is exact.
+struct Pool3s2H {
+  int H, W, Ho, Wo, strips, w8;
+  int64_t items;   // planes * strips * w8
+  FastDiv by_w8, by_strips;
+};
+
+__device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
+__device__ __forceinline__ uint32_t bf16_pack_exact(float lo, float hi) {   // both already bf16 values
+  return (__float_as_uint(lo) >> 16) | (__float_as_uint(hi) & 0xFFFF0000u);
+}
+
+template <int R>
+__global__ void __launch_bounds__(256) window_max_3x3s2_bf16(const uint16_t* __restrict__ in, uint16_t* __restrict__ out,
+                                                              const Pool3s2H p, float fill) {
+  const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  if (t >= p.items) { pdl_wait(); pdl_launch_dependents(); return; }
+  uint32_t rest, j, plane, strip;
+  p.by_w8.divmod(static_cast<uint32_t>(t), rest, j);
+  p.by_strips.divmod(rest, plane, strip);
+  const uint16_t* src = in + static_cast<int64_t>(plane) * p.H * p.W;
+  uint16_t* dst = out + static_cast<int64_t>(plane) * p.Ho * p.Wo;
+  const int y0 = static_cast<int>(strip) * R;
+  pdl_wait();
+  pdl_launch_dependents();
+  uint4 v[2 * R + 1];
+  float left[2 * R + 1];
+  const uint32_t fill2 = bf16_pack_exact(fill, fill);
+#pragma unroll
+  for (int i = 0; i < 2 * R + 1; ++i) {
+    const int h = 2 * y0 - 1 + i;
+    if (h >= 0 && h < p.H) {
+      const uint16_t* row = src + (int64_t)h * p.W + 8 * j;
+      v[i] = *reinterpret_cast<const uint4*>(row);
+      left[i] = j > 0 ? bf16_lo(row[-1]) : fill;
+    } else {
+      v[i] = make_uint4(fill2, fill2, fill2, fill2);
+      left[i] = fill;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < R; ++i) {
+    const int y = y0 + i;
+    if (y < p.Ho) {
+      float o0 = -INFINITY, o1 = -INFINITY, o2 = -INFINITY, o3 = -INFINITY;
+#pragma unroll
+      for (int d = 0; d < 3; ++d) {
+        const uint4 w = v[2 * i + d];
+        const float x1 = bf16_hi(w.x), x3 = bf16_hi(w.y), x5 = bf16_hi(w.z);
+        o0 = fmaxf(o0, fmaxf(fmaxf(left[2 * i + d], bf16_lo(w.x)), x1));
+        o1 = fmaxf(o1, fmaxf(fmaxf(x1, bf16_lo(w.y)), x3));
+        o2 = fmaxf(o2, fmaxf(fmaxf(x3, bf16_lo(w.z)), x5));
+        o3 = fmaxf(o3, fmaxf(fmaxf(x5, bf16_lo(w.w)), bf16_hi(w.w)));
+      }
+      *reinterpret_cast<uint2*>(dst + (int64_t)y * p.Wo + 4 * j) = make_uint2(bf16_pack_exact(o0, o1), bf16_pack_exact(o2, o3));
+    }
+  }
+}
+
 // reduceMax of whole items (no windows): one warp per item.
 __global__ void __launch_bounds__(kThreads) item_max(const float* __restrict__ in, float* __restrict__ out,
                                                       int64_t items, int64_t item) {
@@ -1338,6 +1400,24 @@ int gl_compute_reduce_max(const gl_ap* in, const gl_windows* w, gl_ap* out, void
     gl_shape_windows(in, w, &A);
     const float fill = w->pad_kind == GL_PAD_NEG_INF ? -INFINITY : 0.0f;
     const int64_t nwin = numel(want);
+    if (w->wshape[0] == 3 && w->wshape[1] == 3 && w->stride[0] == 2 && w->stride[1] == 2 && w->pad_lo[0] == 1 &&
+        w->pad_lo[1] == 1 && in->shape[nb + 1] % 8 == 0 && in->shape[nb] < (1 << 20) && in->shape[nb + 1] < (1 << 20) &&
+        A.shape[nb + 1] * 2 == in->shape[nb + 1]) {
+      constexpr int kRows = 2;
+      Pool3s2H t;
+      t.H = (int)in->shape[nb]; t.W = (int)in->shape[nb + 1];
+      t.Ho = (int)A.shape[nb]; t.Wo = (int)A.shape[nb + 1];
+      t.strips = (t.Ho + kRows - 1) / kRows;
+      t.w8 = t.W / 8;
+      t.items = prod(in->shape, 0, nb) * t.strips * t.w8;
+      if (t.items < (1ll << 31)) {
+        t.by_w8 = make_fastdiv(t.w8);
+        t.by_strips = make_fastdiv(t.strips);
+        return launch_pdl(window_max_3x3s2_bf16<kRows>, dim3(static_cast<unsigned>((t.items + 255) / 256)), dim3(256), 0, st, 1,
+                          static_cast<const uint16_t*>(in->data), static_cast<uint16_t*>(out->data), t, fill) == cudaSuccess
+                   ? GL_OK : GL_ERR_CUDA;
+      }
+    }
     if (in->shape[nb] < (1 << 20) && in->shape[nb + 1] < (1 << 20) && w->wshape[0] < 1024 && w->wshape[1] < 1024 &&
         w->stride[0] < 1024 && w->stride[1] < 1024) {
       PoolTile t;

@@ -195,7 +195,8 @@ def test_channels_last_max_pool(gl, n, h, w, c, k, s, pd, dtype):
 
 
 @pytest.mark.parametrize("shape,k,s,pd", [((2, 3, 9, 8), (3, 3), (2, 2), (1, 1)), ((1, 5, 16, 24), (8, 8), (8, 8), (0, 0)),
-                                          ((3, 2, 7, 11), (2, 3), (1, 2), (0, 1))])
+                                          ((3, 2, 7, 11), (2, 3), (1, 2), (0, 1)), ((2, 2, 14, 16), (3, 3), (2, 2), (1, 1)),
+                                          ((1, 3, 33, 40), (3, 3), (2, 2), (1, 1)), ((2, 5, 112, 112), (3, 3), (2, 2), (1, 1))])
 def test_bf16_plane_max_pool(gl, shape, k, s, pd):
     x = synth.bf16_round(synth.uniform(13, 1, shape, -1.0, 1.0) - 2.0)
     ref = brute.maxpool(x, k, s, ((pd[0], pd[0]), (pd[1], pd[1])))
