@@ -809,6 +809,62 @@ __global__ void __launch_bounds__(kThreads) window_max_hwc(const uint4* __restri
   }
 }
 
+// The same with the window shape fixed at compile time: all KH*KW pieces are requested before the first maximum
+// is taken (addresses of border cells are clamped into the image and their values replaced by `fill`), so a
+// thread has KH*KW loads in flight instead of one chain of load, compare, next address.
+template <bool BF16, int KH, int KW>
+__global__ void __launch_bounds__(kThreads) window_max_hwc_fixed(const uint4* __restrict__ in, uint4* __restrict__ out,
+                                                                  const PoolHwc p, float fill) {
+  const int64_t e0 = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  const bool live = e0 < p.total;
+  uint32_t pix, v, row, wo, n, ho;
+  p.by_cv.divmod(static_cast<uint32_t>(live ? e0 : 0), pix, v);
+  p.by_Wo.divmod(pix, row, wo);
+  p.by_Ho.divmod(row, n, ho);
+  const uint4* img = in + static_cast<int64_t>(n) * p.H * p.W * p.cv + v;
+  pdl_wait();
+  pdl_launch_dependents();
+  if (!live) return;
+  uint4 q[KH * KW];
+  bool inside[KH * KW];
+#pragma unroll
+  for (int dy = 0; dy < KH; ++dy) {
+#pragma unroll
+    for (int dx = 0; dx < KW; ++dx) {
+      const int h = static_cast<int>(ho) * p.Sh + dy - p.ph, w = static_cast<int>(wo) * p.Sw + dx - p.pw;
+      inside[dy * KW + dx] = h >= 0 && h < p.H && w >= 0 && w < p.W;
+      const int hc = min(max(h, 0), p.H - 1), wc = min(max(w, 0), p.W - 1);
+      q[dy * KW + dx] = img[(static_cast<int64_t>(hc) * p.W + wc) * p.cv];
+    }
+  }
+  float best[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) best[i] = -INFINITY;
+#pragma unroll
+  for (int t = 0; t < KH * KW; ++t) {
+    const uint32_t qq[4] = {q[t].x, q[t].y, q[t].z, q[t].w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (BF16) {
+        best[2 * i] = fmaxf(best[2 * i], inside[t] ? bf16_bits_to_float(qq[i] & 0xFFFFu) : fill);
+        best[2 * i + 1] = fmaxf(best[2 * i + 1], inside[t] ? __uint_as_float(qq[i] & 0xFFFF0000u) : fill);
+      } else {
+        best[i] = fmaxf(best[i], inside[t] ? __uint_as_float(qq[i]) : fill);
+      }
+    }
+  }
+  uint4 r;
+  if (BF16) {
+    r.x = (__float_as_uint(best[0]) >> 16) | (__float_as_uint(best[1]) & 0xFFFF0000u);
+    r.y = (__float_as_uint(best[2]) >> 16) | (__float_as_uint(best[3]) & 0xFFFF0000u);
+    r.z = (__float_as_uint(best[4]) >> 16) | (__float_as_uint(best[5]) & 0xFFFF0000u);
+    r.w = (__float_as_uint(best[6]) >> 16) | (__float_as_uint(best[7]) & 0xFFFF0000u);
+  } else {
+    r = make_uint4(__float_as_uint(best[0]), __float_as_uint(best[1]), __float_as_uint(best[2]), __float_as_uint(best[3]));
+  }
+  out[e0] = r;
+}
+
 // 2D windows + reduceMax, tiled: one block owns TH output rows of one plane.  It
 // stages the (TH-1)*Sh+Kh input rows it needs (border cells hold the fill value)
 // with 128-bit loads, then every thread reduces whole windows out of shared
@@ -1019,6 +1075,51 @@ __global__ void __launch_bounds__(256) window_max_3x3s2_bf16(const uint16_t* __r
       *reinterpret_cast<uint2*>(dst + (int64_t)y * p.Wo + 4 * j) = make_uint2(bf16_pack_exact(o0, o1), bf16_pack_exact(o2, o3));
     }
   }
+}
+
+// 2-byte planes whose windows are eight columns wide, eight apart and unpadded in W (rows of a multiple of
+// eight values): every window row is one aligned 16-byte piece.  A thread owns one window; its Kh pieces are
+// requested eight at a time (rows outside the plane: address clamped, value replaced by `fill`).
+struct PoolRow8 {
+  int H, W, Kh, Sh, ph, Ho, Wo;
+  int64_t total;   // planes * Ho * Wo
+  FastDiv by_Wo, by_Ho;
+};
+
+__global__ void __launch_bounds__(kThreads) window_max_rows8_bf16(const uint16_t* __restrict__ in, uint16_t* __restrict__ out,
+                                                                   const PoolRow8 p, float fill) {
+  const int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  const bool live = e < p.total;
+  uint32_t row, wo, plane, ho;
+  p.by_Wo.divmod(static_cast<uint32_t>(live ? e : 0), row, wo);
+  p.by_Ho.divmod(row, plane, ho);
+  const uint16_t* src = in + static_cast<int64_t>(plane) * p.H * p.W + 8 * wo;
+  pdl_wait();
+  pdl_launch_dependents();
+  if (!live) return;
+  float best = -INFINITY;
+  const int h0 = static_cast<int>(ho) * p.Sh - p.ph;
+  for (int d0 = 0; d0 < p.Kh; d0 += 8) {
+    uint4 q[8];
+#pragma unroll
+    for (int d = 0; d < 8; ++d) {
+      const int h = min(max(h0 + d0 + d, 0), p.H - 1);
+      q[d] = *reinterpret_cast<const uint4*>(src + static_cast<int64_t>(h) * p.W);
+    }
+#pragma unroll
+    for (int d = 0; d < 8; ++d) {
+      const int h = h0 + d0 + d;
+      if (d0 + d < p.Kh) {
+        float m = fill;
+        if (h >= 0 && h < p.H) {
+          m = fmaxf(fmaxf(fmaxf(bf16_lo(q[d].x), bf16_hi(q[d].x)), fmaxf(bf16_lo(q[d].y), bf16_hi(q[d].y))),
+                    fmaxf(fmaxf(bf16_lo(q[d].z), bf16_hi(q[d].z)), fmaxf(bf16_lo(q[d].w), bf16_hi(q[d].w))));
+        }
+        best = fmaxf(best, m);
+      }
+    }
+  }
+  out[e] = static_cast<uint16_t>(__float_as_uint(best) >> 16);
 }
 
 // reduceMax of whole items (no windows): one warp per item.
@@ -1382,6 +1483,15 @@ int gl_compute_reduce_max(const gl_ap* in, const gl_windows* w, gl_ap* out, void
         t.by_Wo = make_fastdiv(t.Wo);
         t.by_Ho = make_fastdiv(t.Ho);
         const float fill = w->pad_kind == GL_PAD_NEG_INF ? -INFINITY : 0.0f;
+        if (t.split_log2 == 0 && t.Kh == 3 && t.Kw == 3 && (t.total + kThreads - 1) / kThreads <= 0x7FFFFFFF) {
+          const dim3 fgrid(static_cast<unsigned>((t.total + kThreads - 1) / kThreads));
+          const cudaError_t ferr =
+              bf16 ? launch_pdl(window_max_hwc_fixed<true, 3, 3>, fgrid, dim3(kThreads), 0, st, 1,
+                                static_cast<const uint4*>(in->data), static_cast<uint4*>(out->data), t, fill)
+                   : launch_pdl(window_max_hwc_fixed<false, 3, 3>, fgrid, dim3(kThreads), 0, st, 1,
+                                static_cast<const uint4*>(in->data), static_cast<uint4*>(out->data), t, fill);
+          return ferr == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+        }
         const dim3 grid(grid_for(t.total, kThreads));
         const cudaError_t err =
             bf16 ? launch_pdl(window_max_hwc<true>, grid, dim3(kThreads), 0, st, 1, static_cast<const uint4*>(in->data),
@@ -1417,6 +1527,20 @@ int gl_compute_reduce_max(const gl_ap* in, const gl_windows* w, gl_ap* out, void
                           static_cast<const uint16_t*>(in->data), static_cast<uint16_t*>(out->data), t, fill) == cudaSuccess
                    ? GL_OK : GL_ERR_CUDA;
       }
+    }
+    if (w->wshape[1] == 8 && w->stride[1] == 8 && w->pad_lo[1] == 0 && in->shape[nb + 1] % 8 == 0 &&
+        A.shape[nb + 1] * 8 <= in->shape[nb + 1] && w->wshape[0] <= 64 && w->stride[0] < 1024 && w->pad_lo[0] < 1024 &&
+        in->shape[nb] < (1 << 20) && in->shape[nb + 1] < (1 << 20) && nwin < (1ll << 31)) {
+      PoolRow8 t;
+      t.H = (int)in->shape[nb]; t.W = (int)in->shape[nb + 1];
+      t.Kh = (int)w->wshape[0]; t.Sh = (int)w->stride[0]; t.ph = (int)w->pad_lo[0];
+      t.Ho = (int)A.shape[nb]; t.Wo = (int)A.shape[nb + 1];
+      t.total = nwin;
+      t.by_Wo = make_fastdiv(t.Wo);
+      t.by_Ho = make_fastdiv(t.Ho);
+      return launch_pdl(window_max_rows8_bf16, dim3(static_cast<unsigned>((nwin + kThreads - 1) / kThreads)), dim3(kThreads), 0, st,
+                        1, static_cast<const uint16_t*>(in->data), static_cast<uint16_t*>(out->data), t, fill) == cudaSuccess
+                 ? GL_OK : GL_ERR_CUDA;
     }
     if (in->shape[nb] < (1 << 20) && in->shape[nb + 1] < (1 << 20) && w->wshape[0] < 1024 && w->wshape[1] < 1024 &&
         w->stride[0] < 1024 && w->stride[1] < 1024) {

@@ -196,7 +196,9 @@ def test_channels_last_max_pool(gl, n, h, w, c, k, s, pd, dtype):
 
 @pytest.mark.parametrize("shape,k,s,pd", [((2, 3, 9, 8), (3, 3), (2, 2), (1, 1)), ((1, 5, 16, 24), (8, 8), (8, 8), (0, 0)),
                                           ((3, 2, 7, 11), (2, 3), (1, 2), (0, 1)), ((2, 2, 14, 16), (3, 3), (2, 2), (1, 1)),
-                                          ((1, 3, 33, 40), (3, 3), (2, 2), (1, 1)), ((2, 5, 112, 112), (3, 3), (2, 2), (1, 1))])
+                                          ((1, 3, 33, 40), (3, 3), (2, 2), (1, 1)), ((2, 5, 112, 112), (3, 3), (2, 2), (1, 1)),
+                                          ((2, 3, 13, 32), (4, 8), (3, 8), (1, 0)), ((3, 4, 56, 56), (8, 8), (8, 8), (0, 0)),
+                                          ((1, 2, 40, 16), (20, 8), (20, 8), (0, 0))])
 def test_bf16_plane_max_pool(gl, shape, k, s, pd):
     x = synth.bf16_round(synth.uniform(13, 1, shape, -1.0, 1.0) - 2.0)
     ref = brute.maxpool(x, k, s, ((pd[0], pd[0]), (pd[1], pd[1])))
