@@ -328,15 +328,18 @@ def detail_workloads(device, peaks):
         chain_entry(layout)                       # Fig. 2a + relu + Fig. 2c + Fig. 2b composed, per item layout
     for cfg in (synth.MEM_IM2COL, synth.MEM_TRANSPOSE, synth.MEM_MAXPOOL, synth.MEM_RELU, synth.MEM_PAD):
         entry(cfg, "")
-    # a plain device-to-device copy of the pad workload's size, for scale: what a 52 MB operator can reach at all
-    # between two launches (torch's copy kernel, not one of this library's; a reference row, not a result)
-    n_f32 = synth.MEM_PAD.algorithmic_bytes // 8
-    srcs = [torch.empty(n_f32, dtype=torch.float32, device=device).normal_() for _ in range(6)]
-    dsts = [torch.empty_like(t) for t in srcs]
-    med, best = time_graph([lambda a=a, b=b: b.copy_(a) for a, b in zip(srcs, dsts)], 20, device)
-    out.append({"workload": "reference_copy_%dMB" % (n_f32 * 8 // 1000000), "layout": "torch copy_, same bytes as pad_w1",
-                "us": med * 1e6, "gbs": n_f32 * 8 / med / 1e9, "frac_hbm_peak": n_f32 * 8 / med / 1e9 / peaks["hbm_gbs"]})
-    del srcs, dsts
+    # plain device-to-device copies of the memory-bound workloads' sizes, for scale: what an operator that moves so
+    # many bytes can reach at all between two launches (torch's copy kernel, not one of this library's; reference
+    # rows, not results)
+    for cfg, label in ((synth.MEM_PAD, "pad_w1"), (synth.MEM_RELU, "relu_4096x4096"), (synth.MEM_IM2COL, "im2col")):
+        n_f32 = cfg.algorithmic_bytes // 8
+        sets = 6 if n_f32 * 8 < 100e6 else 3
+        srcs = [torch.empty(n_f32, dtype=torch.float32, device=device).normal_() for _ in range(sets)]
+        dsts = [torch.empty_like(t) for t in srcs]
+        med, best = time_graph([lambda a=a, b=b: b.copy_(a) for a, b in zip(srcs, dsts)], 20, device)
+        out.append({"workload": "reference_copy_%dMB" % (n_f32 * 8 // 1000000), "layout": "torch copy_, same bytes as %s" % label,
+                    "us": med * 1e6, "gbs": n_f32 * 8 / med / 1e9, "frac_hbm_peak": n_f32 * 8 / med / 1e9 / peaks["hbm_gbs"]})
+        del srcs, dsts
     # host cost of a plain call (no CUDA graph) on a small convolution: planning, tensor maps (cached per
     # argument list after the first call) and the launch
     from paper_2105_09377_b200 import binding as gl

@@ -1015,6 +1015,52 @@ __global__ void __launch_bounds__(256) window_max_3x3s2(const float* __restrict_
   }
 }
 
+// The same with the (plane, strip, column group) items dealt to threads one by one, so that every lane of a warp
+// has work whatever the row length (rows of 28 column groups leave four lanes of a warp-per-strip layout idle).
+template <int R>
+__global__ void __launch_bounds__(256) window_max_3x3s2_flat(const float* __restrict__ in, float* __restrict__ out,
+                                                              const Pool3s2 p, int64_t items, FastDiv by_w4, float fill) {
+  const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  const bool live = t < items;
+  uint32_t rest, j, plane, strip;
+  by_w4.divmod(static_cast<uint32_t>(live ? t : 0), rest, j);
+  p.by_strips.divmod(rest, plane, strip);
+  const float* src = in + static_cast<int64_t>(plane) * p.H * p.W;
+  float* dst = out + static_cast<int64_t>(plane) * p.Ho * p.Wo;
+  const int y0 = static_cast<int>(strip) * R;
+  pdl_wait();
+  pdl_launch_dependents();
+  if (!live) return;
+  float4 v[2 * R + 1];
+  float left[2 * R + 1];
+#pragma unroll
+  for (int i = 0; i < 2 * R + 1; ++i) {
+    const int h = 2 * y0 - 1 + i;
+    if (h >= 0 && h < p.H) {
+      const float* row = src + (int64_t)h * p.W + 4 * j;
+      v[i] = *reinterpret_cast<const float4*>(row);
+      left[i] = j > 0 ? row[-1] : fill;
+    } else {
+      v[i] = make_float4(fill, fill, fill, fill);
+      left[i] = fill;
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < R; ++i) {
+    const int y = y0 + i;
+    if (y < p.Ho) {
+      float o0 = -INFINITY, o1 = -INFINITY;
+#pragma unroll
+      for (int d = 0; d < 3; ++d) {
+        const float4 w = v[2 * i + d];
+        o0 = fmaxf(o0, fmaxf(fmaxf(left[2 * i + d], w.x), w.y));
+        o1 = fmaxf(o1, fmaxf(fmaxf(w.y, w.z), w.w));
+      }
+      *reinterpret_cast<float2*>(dst + (int64_t)y * p.Wo + 2 * j) = make_float2(o0, o1);
+    }
+  }
+}
+
 // The same pooling on 2-byte planes (rows that are multiples of eight values): a thread owns eight input
 // columns (four outputs) of one strip of R output rows.  bf16 values are compared as the floats they stand for
 // (a shift), so the maximum is exact.
@@ -1581,6 +1627,11 @@ int gl_compute_reduce_max(const gl_ap* in, const gl_windows* w, gl_ap* out, void
     t.w4 = t.W / 4;
     t.units = prod(in->shape, 0, na) * t.strips;
     t.by_strips = make_fastdiv(t.strips);
+    const int64_t items = t.units * t.w4;
+    if (t.w4 % 32 != 0 && items < (1ll << 31)) {
+      return launch_pdl(window_max_3x3s2_flat<kRows>, dim3(static_cast<unsigned>((items + 255) / 256)), dim3(256), 0, st, 1, src, dst,
+                        t, items, make_fastdiv(t.w4), fill) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+    }
     const int64_t blocks = (t.units + 7) / 8;
     if (blocks <= 0x7FFFFFFF) {
       return launch_pdl(window_max_3x3s2<kRows>, dim3(static_cast<unsigned>(blocks)), dim3(32, 8), 0, st, 1, src, dst, t,
