@@ -590,7 +590,7 @@ constexpr int kBM = 128;
 constexpr int kBK = 64;          // bf16 elements per K block = one 128-byte swizzle row
 constexpr int kTcThreads = 224;  // warp 0 TMA (A), warp 1 MMA + TMEM, warps 2-5 epilogue, warp 6 TMA (B)
 
-enum AMode { kDense = 0, kIm2col = 1, kIm2colGranule = 2, kRowWin = 3 };
+enum AMode { kDense = 0, kIm2col = 1, kIm2colGranule = 2, kRowWin = 3, kChwPix = 4 };
 
 struct TcParams {
   int64_t M, O, K;        // K as laid out in B (for conv: Kh*Kw*Cp)
@@ -620,7 +620,13 @@ struct TcParams {
   // count the wide tiles of all bands first (n_wide of them), then the half-wide ones (nA per band for
   // tm < bA, nA + 2 per later band).
   int mix, n_wide, wA, bA, nA;
+  // kChwPix only: 1x1 windows over (C,H,W) items read where they are.  A tile is two output rows of one image in
+  // a pitch of 64 pixels: tensor-memory lane m = 64 * j + w is input pixel (row (2 * ti + j) * Sh, column w).
+  int pix_tpi, pix_w;     // tiles per image = ceil(Ho / 2); input width (w >= pix_w: zero fill, dropped)
+  FastDiv div_pix_tpi;
 };
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int c, int w, int h, int n, uint32_t bar);
 
 struct TileAt { int tm, n0, width; };
 
@@ -674,6 +680,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
        const __grid_constant__ CUtensorMap map_c, float* __restrict__ out, const TcParams p) {
   using Cfg = TcCfg<BN, G, OCC, CTAS>;
   static_assert(CTAS == 1 || (CTAS == 2 && (MODE == kDense || MODE == kIm2col)), "pairs: dense and im2col tiles only");
+  static_assert(MODE != kChwPix || (CTAS == 1 && G == 1), "pixel-major A: one K block per stage, single blocks");
   static_assert(Cfg::kStages >= 2, "ring too shallow");
   extern __shared__ unsigned char smem_raw[];
   // operand tiles need 1024-byte alignment for the 128-byte swizzle
@@ -796,6 +803,13 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
             wbase = static_cast<int>(seg) * kBM;
             hbase = static_cast<int>(im) * p.Hp + static_cast<int>(ho) * p.Sh;
           }
+        } else if (MODE == kChwPix) {
+          if (load_a) {   // tile -> (image, pair of output rows)
+            uint32_t im, ti;
+            p.div_pix_tpi.divmod(tm, im, ti);
+            img = static_cast<int>(im);
+            hbase = static_cast<int>(ti) * 2;
+          }
         } else if (MODE != kDense && load_a) {
           uint32_t im, rem, ho, wo;
           p.div_howo.divmod(static_cast<uint32_t>(m0), im, rem);
@@ -847,6 +861,15 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
               // K block kb = filter row kb: 128 output columns x 64 values of padded input row hbase + kb
               if (load_a) tma_load_3d(sa, &map_a, 0, wbase, hbase + kb, full);
               else tma_load_2d(sb, &map_b, kb * kBK, n0, full);
+            } else if (MODE == kChwPix) {
+              // A arrives pixel-major: a box is 64 channels x one input row of 64 pixels (128 bytes per channel),
+              // the tile's two rows 8 KB apart; pixels past the row's end read as zeros
+              if (load_a) {
+                tma_load_4d(sa, &map_a, 0, hbase * p.Sh, kb * kBK, img, full);
+                tma_load_4d(sa + Cfg::kStageA / 2, &map_a, 0, (hbase + 1) * p.Sh, kb * kBK, img, full);
+              } else {
+                tma_load_2d(sb, &map_b, kb * kBK, n0, full);
+              }
             } else if (MODE == kIm2col) {
               if (load_a)
                 tma_load_im2col(sa, &map_a, cc * kBK, wbase, hbase, img, static_cast<uint16_t>(kw),
@@ -881,8 +904,14 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
     // ---------------- MMA issuer ----------------
     if (rank == 0) {
       const bool leader = elect_one();   // the loop is warp-uniform; this lane issues the MMAs and commits
-      constexpr uint32_t idesc_wide = make_idesc(kBM * CTAS, BN), idesc_half = make_idesc(kBM * CTAS, BN / 2);
-      const uint64_t desc_a0 = (MODE == kIm2colGranule) ? make_desc(tiles, kBM * 16, 128, 0) : make_desc(tiles, 16, 1024, 2);
+      // (pixel-major A: bit 15 of the instruction descriptor = A is MN-major)
+      constexpr uint32_t idesc_wide = make_idesc(kBM * CTAS, BN) | (MODE == kChwPix ? (1u << 15) : 0u),
+                         idesc_half = make_idesc(kBM * CTAS, BN / 2);
+      // MN-major A with the 128-byte swizzle: 64 pixels of one channel per 128-byte row, 8 channels per 1024-byte
+      // group (SBO), the next 64 pixels LBO bytes further on
+      const uint64_t desc_a0 = (MODE == kIm2colGranule) ? make_desc(tiles, kBM * 16, 128, 0)
+                               : (MODE == kChwPix)      ? make_desc(tiles, Cfg::kStageA / 2, 1024, 2)
+                                                        : make_desc(tiles, 16, 1024, 2);
       const uint64_t desc_b0 = (MODE == kIm2colGranule) ? make_desc(tiles + G * Cfg::kStageA, BN * 16, 128, 0)
                                                         : make_desc(tiles + G * Cfg::kStageA, 16, 1024, 2);
       uint32_t s = 0, ph = 0, tile_it = 0;
@@ -908,7 +937,7 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
             if (j < nsub) {
 #pragma unroll
               for (int k = 0; k < kBK / 16; ++k) {
-                constexpr int kStepA = (MODE == kIm2colGranule) ? 2 * (kBM * 16) : 32;
+                constexpr int kStepA = (MODE == kIm2colGranule) ? 2 * (kBM * 16) : (MODE == kChwPix ? 16 * 128 : 32);
                 constexpr int kStepB = (MODE == kIm2colGranule) ? 2 * (BN * 16) : 32;
                 const uint64_t da = da0 + ((j * Cfg::kStageA + k * kStepA) >> 4);
                 const uint64_t db = db0 + ((j * Cfg::kStageB + k * kStepB) >> 4);
@@ -960,6 +989,14 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
         const int wloc = static_cast<int>(oseg) * kBM + q * 32 + lane;
         m = static_cast<int64_t>(orow) * p.Wo + wloc;
         m_ok = wloc < p.Wo;
+      }
+      if (MODE == kChwPix) {
+        uint32_t im, ti;
+        p.div_pix_tpi.divmod(tmu, im, ti);
+        const int mloc = q * 32 + lane, w = mloc & 63, hh = static_cast<int>(ti) * 2 + (mloc >> 6);
+        const int ow = w >> (p.Sw - 1);   // Sw is 1 or 2
+        m = (static_cast<int64_t>(im) * p.Ho + hh) * p.Wo + ow;
+        m_ok = hh < p.Ho && w < p.pix_w && (w & (p.Sw - 1)) == 0 && ow < p.Wo;
       }
       const int64_t row_at = (static_cast<int64_t>(ks) * p.M + m) * p.O;   // partial plane ks (0 without a K split)
       float* row = out + row_at;
@@ -2162,11 +2199,12 @@ int launch_tc(const CUtensorMap& ma, const CUtensorMap& mb, float* out, TcParams
   p.div_wo.set(p.Wo > 0 ? p.Wo : 1);
   p.div_howo.set(p.Wo > 0 ? static_cast<int64_t>(p.Wo) * p.Ho : 1);
   CUtensorMap mc;
-  p.tma_store = (p.O % (p.out_bf16 ? 8 : 4) == 0 && !p.out_nchw) ? 1 : 0;
+  p.tma_store = (p.O % (p.out_bf16 ? 8 : 4) == 0 && !p.out_nchw && MODE != kChwPix) ? 1 : 0;
   if (MODE == kRowWin) {
     p.div_segs.set(p.segs);
     p.div_ho.set(p.Ho);
   }
+  if (MODE == kChwPix) p.div_pix_tpi.set(p.pix_tpi);
   if (p.tma_store) {
     const bool ok = MODE == kRowWin ? encode_result_rows(&mc, out, p.M / p.Wo, p.Wo, p.O, p.out_bf16 != 0)
                                     : encode_result(&mc, out, p.M, p.O, p.ksplit, p.out_bf16 != 0);
@@ -2283,6 +2321,9 @@ struct ConvPlan {
   // (C,H,W) items with 1x1 unpadded windows: the copy holds only the pixels the windows touch and is
   // then the [N*H'*W', Cp] matrix of a plain matrix product
   bool as_matrix = false;
+  // (C,H,W) items with 1x1 unpadded windows whose rows the TMA unit can fetch (W a multiple of 8, at most 64): read
+  // in place as a pixel-major (MN-major) A operand, no copy at all
+  bool pixmajor = false;
   bool rowrun = false;
   int rr_cp = 0, rr_ksteps = 0, rr_bn = 0, rr_stages = 0, rr_raw_stages = 0, rr_nseg = 0;
   uint32_t rr_seg = 0, rr_slot = 0, rr_b_bytes = 0, rr_raw_seg = 0;
@@ -2335,6 +2376,13 @@ ConvPlan plan_conv(const DotProblem& d, uint32_t flags) {
     pl.Wpa = (pl.Wpa + d.Sw - 1) / d.Sw * d.Sw;
     pl.x_bytes = round_up(static_cast<size_t>(d.N * pl.Hp * pl.Wpa * pl.Cp) * 2, 1024);
     pl.w_bytes = round_up(static_cast<size_t>(d.O * d.Kh * kBK) * 2, 1024);
+    return pl;
+  }
+  pl.pixmajor = pl.tc && !d.channels_last && d.Kh == 1 && d.Kw == 1 && d.ph_lo == 0 && d.ph_hi == 0 && d.pw_lo == 0 &&
+                d.pw_hi == 0 && !(flags & GL_OUT_NCHW) && d.C % 8 == 0 && d.C >= kBK && d.W % 8 == 0 && d.W <= 64 &&
+                (d.Sw == 1 || d.Sw == 2) && d.N * ((d.Ho + 1) / 2) < (1ll << 30);
+  if (pl.pixmajor) {
+    pl.prepass = false;
     return pl;
   }
   pl.as_matrix = pl.tc && !d.channels_last && d.Kh == 1 && d.Kw == 1 && d.ph_lo == 0 && d.ph_hi == 0 && d.pw_lo == 0 &&
@@ -2425,6 +2473,18 @@ bool encode_halo_box(CUtensorMap* m, const void* base, const DotProblem& d, int6
   const cuuint64_t strides[3] = {static_cast<cuuint64_t>(Cp) * 2, static_cast<cuuint64_t>(d.W * Cp) * 2,
                                  static_cast<cuuint64_t>(d.H * d.W * Cp) * 2};
   const cuuint32_t box[4] = {kBK, static_cast<cuuint32_t>(Wb), static_cast<cuuint32_t>(RB), 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return encode_tiled_cached(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+}
+
+// (C,H,W) items as (W, H, C, N): one box = 64 pixels of one input row x 64 channels, landing channel by channel
+// (128 bytes of pixels each): the MN-major A operand of 1x1 windows.  Pixels past W and channels past C read as zeros.
+bool encode_chw_rows(CUtensorMap* m, const void* base, const DotProblem& d) {
+  const cuuint64_t dims[4] = {static_cast<cuuint64_t>(d.W), static_cast<cuuint64_t>(d.H), static_cast<cuuint64_t>(d.C),
+                              static_cast<cuuint64_t>(d.N)};
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(d.W) * 2, static_cast<cuuint64_t>(d.H * d.W) * 2,
+                                 static_cast<cuuint64_t>(d.C * d.H * d.W) * 2};
+  const cuuint32_t box[4] = {64, 1, kBK, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   return encode_tiled_cached(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
 }
@@ -2646,7 +2706,7 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
   const size_t pre_bytes = (d.conv && pl.prepass) ? pl.x_bytes + pl.w_bytes : 0;
   HaloPlan hp;
   if (d.conv) hp = plan_halo(d, pl, flags);
-  const bool split_mode = (!d.conv || (!pl.rowwin && pl.Cp >= kBK)) && !out_nchw && !hp.ok;
+  const bool split_mode = (!d.conv || (!pl.rowwin && pl.Cp >= kBK)) && !out_nchw && !hp.ok && !pl.pixmajor;
   const int64_t kblocks_all = !d.conv ? (d.K + kBK - 1) / kBK : d.Kh * d.Kw * ((pl.Cp + kBK - 1) / kBK);
   TilePlan tp = plan_tiles(d.M, d.O, kblocks_all, split_mode);
   if (tp.ksplit > 1 && (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 1023u) ||
@@ -2743,6 +2803,20 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     auto kernel = d.C == 3 ? (d.channels_last ? conv_rowrun<3, 1> : conv_rowrun<3, 0>) : conv_rowrun<0, 0>;
     return launch_pdl(kernel, dim3(static_cast<unsigned>(grid)), dim3(kRunThreads), static_cast<size_t>(smem), st, 1,
                       pa, pb, mc, rp) == cudaSuccess ? GL_OK : GL_ERR_CUDA;
+  }
+  if (pl.pixmajor) {
+    // 1x1 windows of (C,H,W) items: A tiles come straight from the items, pixel-major; the weights (O, C, 1, 1)
+    // already are the [O, C] matrix.  With Sw = 2 the odd pixels of a row are multiplied too and dropped.
+    p.K = d.C;
+    p.kblocks = static_cast<int>((d.C + kBK - 1) / kBK);
+    p.Sh = static_cast<int>(d.Sh); p.Sw = static_cast<int>(d.Sw);
+    p.Ho = static_cast<int>(d.Ho); p.Wo = static_cast<int>(d.Wo);
+    p.pix_w = static_cast<int>(d.W);
+    p.pix_tpi = static_cast<int>((d.Ho + 1) / 2);
+    p.tiles_m = static_cast<int>(d.N * p.pix_tpi);
+    p.tiles_n = static_cast<int>((d.O + 127) / 128);
+    if (!encode_chw_rows(&ma, pa, d) || !encode_kmajor_sw128(&mb, pb, d.O, d.C, 128)) return GL_ERR_CUDA;
+    return launch_tc<128, kChwPix, 1, 1>(ma, mb, dst, p, st, PreLaunch());
   }
   if (pl.prepass) {
     const size_t need = pl.x_bytes + pl.w_bytes;

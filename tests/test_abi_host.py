@@ -184,7 +184,9 @@ def test_scratch_sizes_follow_the_layout_rules(gl):
     assert need((32, 128, 28, 28), (128, 128, 3, 3), spec) == up(32 * 28 * 28 * 128 * 2) + up(128 * 9 * 128 * 2)
     # (C,H,W) items, 1x1 stride 2, no pad: only the pixels the windows touch, weights [O, C]
     spec = gl.windows_spec((256, 1, 1), (1, 2, 2))
-    assert need((32, 256, 56, 56), (128, 256, 1, 1), spec) == up(32 * 28 * 28 * 256 * 2) + up(128 * 256 * 2)
+    assert need((8, 256, 30, 30), (128, 256, 1, 1), spec) == up(8 * 15 * 15 * 256 * 2) + up(128 * 256 * 2)
+    # ... unless the rows are ones the TMA unit can fetch (W a multiple of 8, at most 64): read in place, no copy
+    assert need((32, 256, 56, 56), (128, 256, 1, 1), spec) == 0
     # RGB stem, stride 2, either item layout: both operands are read where they are, nothing is copied
     for shape, wshape, spec in (((32, 3, 224, 224), (64, 3, 7, 7), gl.windows_spec((3, 7, 7), (1, 2, 2), (0, 3, 3), (0, 3, 3))),
                                 ((32, 224, 224, 3), (64, 7, 7, 3), gl.windows_spec((7, 7, 3), (2, 2, 1), (3, 3, 0), (3, 3, 0)))):

@@ -457,6 +457,12 @@ CONV_1X1_CHW = [
     (1, 200, 7, 7, 260, 1, 1),     # C not a multiple of 64, O spans tiles
     (2, 128, 10, 10, 64, 2, 2),
     (1, 2048, 7, 7, 64, 1, 1),     # one tile, 32 K blocks: the contraction is split and summed by the second kernel
+    # rows the TMA unit can fetch (W a multiple of 8, at most 64): read in place as a pixel-major operand, no copy
+    (2, 64, 6, 8, 16, 1, 1),
+    (3, 72, 9, 16, 40, 2, 2),      # C = 72: second K block mostly zero fill; odd H'
+    (1, 128, 5, 64, 130, 1, 1),    # full 64-pixel rows, two column tiles, O not a multiple of 4
+    (2, 64, 7, 24, 8, 3, 2),       # row stride 3
+    (2, 256, 12, 56, 128, 2, 2),
 ]
 
 
@@ -469,6 +475,11 @@ def test_conv_1x1_chw_items_bit_exact(gl, case):
     got = _conv_gpu(gl, x, wt, (sh, sw), (0, 0), channels_last=False)
     assert got.shape == ref.shape
     assert np.array_equal(got.astype(np.float64), ref)
+    got = _conv_gpu(gl, x, wt, (sh, sw), (0, 0), channels_last=False, flags=gl.GL_EPILOGUE_RELU)
+    assert np.array_equal(got.astype(np.float64), np.maximum(ref, 0.0))
+    if o % 8 == 0:
+        got = _conv_gpu(gl, x, wt, (sh, sw), (0, 0), channels_last=False, flags=gl.GL_OUT_BF16)
+        assert np.array_equal(np.asarray(got, dtype=np.float64), _bf16(ref))
     # with the fused squeeze + transpose the same items take the general window path
     out = gl.gl_cartesian_dot(gl.AccessPattern(to_bf16_device(x), 1), gl.windows_spec((c, 1, 1), (1, sh, sw)),
                               gl.AccessPattern(to_bf16_device(wt), 1), flags=gl.GL_OUT_NCHW)
