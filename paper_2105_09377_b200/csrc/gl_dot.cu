@@ -622,7 +622,9 @@ struct TcParams {
   int mix, n_wide, wA, bA, nA;
   // kChwPix only: 1x1 windows over (C,H,W) items read where they are.  A tile is two output rows of one image in
   // a pitch of 64 pixels: tensor-memory lane m = 64 * j + w is input pixel (row (2 * ti + j) * Sh, column w).
+  // With unit strides the image is one run of H*W pixels instead (pix_flat): a tile is 128 consecutive pixels.
   int pix_tpi, pix_w;     // tiles per image = ceil(Ho / 2); input width (w >= pix_w: zero fill, dropped)
+  int pix_flat, pix_hw;   // flat form: tiles per image = ceil(H*W / 128)
   FastDiv div_pix_tpi;
 };
 
@@ -865,8 +867,13 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
               // A arrives pixel-major: a box is 64 channels x one input row of 64 pixels (128 bytes per channel),
               // the tile's two rows 8 KB apart; pixels past the row's end read as zeros
               if (load_a) {
-                tma_load_4d(sa, &map_a, 0, hbase * p.Sh, kb * kBK, img, full);
-                tma_load_4d(sa + Cfg::kStageA / 2, &map_a, 0, (hbase + 1) * p.Sh, kb * kBK, img, full);
+                if (p.pix_flat) {   // hbase = 2 * tile index: 64-pixel pieces hbase and hbase + 1 of the image
+                  tma_load_3d(sa, &map_a, hbase * 64, kb * kBK, img, full);
+                  tma_load_3d(sa + Cfg::kStageA / 2, &map_a, (hbase + 1) * 64, kb * kBK, img, full);
+                } else {
+                  tma_load_4d(sa, &map_a, 0, hbase * p.Sh, kb * kBK, img, full);
+                  tma_load_4d(sa + Cfg::kStageA / 2, &map_a, 0, (hbase + 1) * p.Sh, kb * kBK, img, full);
+                }
               } else {
                 tma_load_2d(sb, &map_b, kb * kBK, n0, full);
               }
@@ -997,6 +1004,11 @@ dot_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtens
         const int ow = w >> (p.Sw - 1);   // Sw is 1 or 2
         m = (static_cast<int64_t>(im) * p.Ho + hh) * p.Wo + ow;
         m_ok = hh < p.Ho && w < p.pix_w && (w & (p.Sw - 1)) == 0 && ow < p.Wo;
+        if (p.pix_flat) {
+          const int pixel = static_cast<int>(ti) * kBM + mloc;
+          m = static_cast<int64_t>(im) * p.pix_hw + pixel;
+          m_ok = pixel < p.pix_hw;
+        }
       }
       const int64_t row_at = (static_cast<int64_t>(ks) * p.M + m) * p.O;   // partial plane ks (0 without a K split)
       float* row = out + row_at;
@@ -2379,8 +2391,10 @@ ConvPlan plan_conv(const DotProblem& d, uint32_t flags) {
     return pl;
   }
   pl.pixmajor = pl.tc && !d.channels_last && d.Kh == 1 && d.Kw == 1 && d.ph_lo == 0 && d.ph_hi == 0 && d.pw_lo == 0 &&
-                d.pw_hi == 0 && !(flags & GL_OUT_NCHW) && d.C % 8 == 0 && d.C >= kBK && d.W % 8 == 0 && d.W <= 64 &&
-                (d.Sw == 1 || d.Sw == 2) && d.N * ((d.Ho + 1) / 2) < (1ll << 30);
+                d.pw_hi == 0 && !(flags & GL_OUT_NCHW) && d.C % 8 == 0 && d.C >= kBK &&
+                ((d.Sh == 1 && d.Sw == 1 && (d.H * d.W) % 8 == 0 && d.H * d.W < (1ll << 30)) ||   // one run of H*W pixels
+                 (d.W % 8 == 0 && d.W <= 64 && (d.Sw == 1 || d.Sw == 2))) &&                     // row by row
+                d.N * ((d.Ho + 1) / 2) < (1ll << 30);
   if (pl.pixmajor) {
     pl.prepass = false;
     return pl;
@@ -2487,6 +2501,15 @@ bool encode_chw_rows(CUtensorMap* m, const void* base, const DotProblem& d) {
   const cuuint32_t box[4] = {64, 1, kBK, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   return encode_tiled_cached(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, base, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
+}
+
+// The same items as (H*W, C, N) when the windows touch every pixel: one box = 64 consecutive pixels x 64 channels.
+bool encode_chw_flat(CUtensorMap* m, const void* base, const DotProblem& d) {
+  const cuuint64_t dims[3] = {static_cast<cuuint64_t>(d.H * d.W), static_cast<cuuint64_t>(d.C), static_cast<cuuint64_t>(d.N)};
+  const cuuint64_t strides[2] = {static_cast<cuuint64_t>(d.H * d.W) * 2, static_cast<cuuint64_t>(d.C * d.H * d.W) * 2};
+  const cuuint32_t box[3] = {64, kBK, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return encode_tiled_cached(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
 }
 
 // Weights (O, Kh, Kw, Cp) viewed as (64 channels, O, chunk, tap): one box = BN rows x 64 channels of
@@ -2812,10 +2835,13 @@ int gl_cartesian_dot(const gl_ap* a0, const gl_windows* w, const gl_ap* a1, gl_a
     p.Sh = static_cast<int>(d.Sh); p.Sw = static_cast<int>(d.Sw);
     p.Ho = static_cast<int>(d.Ho); p.Wo = static_cast<int>(d.Wo);
     p.pix_w = static_cast<int>(d.W);
-    p.pix_tpi = static_cast<int>((d.Ho + 1) / 2);
+    p.pix_flat = (d.Sh == 1 && d.Sw == 1 && (d.H * d.W) % 8 == 0) ? 1 : 0;
+    p.pix_hw = static_cast<int>(d.H * d.W);
+    p.pix_tpi = static_cast<int>(p.pix_flat ? (d.H * d.W + kBM - 1) / kBM : (d.Ho + 1) / 2);
     p.tiles_m = static_cast<int>(d.N * p.pix_tpi);
     p.tiles_n = static_cast<int>((d.O + 127) / 128);
-    if (!encode_chw_rows(&ma, pa, d) || !encode_kmajor_sw128(&mb, pb, d.O, d.C, 128)) return GL_ERR_CUDA;
+    if (!(p.pix_flat ? encode_chw_flat(&ma, pa, d) : encode_chw_rows(&ma, pa, d)) || !encode_kmajor_sw128(&mb, pb, d.O, d.C, 128))
+      return GL_ERR_CUDA;
     return launch_tc<128, kChwPix, 1, 1>(ma, mb, dst, p, st, PreLaunch());
   }
   if (pl.prepass) {

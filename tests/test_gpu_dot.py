@@ -463,6 +463,10 @@ CONV_1X1_CHW = [
     (1, 128, 5, 64, 130, 1, 1),    # full 64-pixel rows, two column tiles, O not a multiple of 4
     (2, 64, 7, 24, 8, 3, 2),       # row stride 3
     (2, 256, 12, 56, 128, 2, 2),
+    (2, 64, 9, 16, 24, 2, 1),      # rows skipped, every pixel of a row used
+    # unit strides and H*W a multiple of 8: the image as one run of pixels
+    (2, 64, 10, 12, 16, 1, 1),     # H*W = 120: one ragged tile per image
+    (1, 128, 28, 28, 64, 1, 1),    # 784 pixels: 6 tiles + 16 pixels
 ]
 
 
