@@ -467,6 +467,10 @@ CONV_1X1_CHW = [
     # unit strides and H*W a multiple of 8: the image as one run of pixels
     (2, 64, 10, 12, 16, 1, 1),     # H*W = 120: one ragged tile per image
     (1, 128, 28, 28, 64, 1, 1),    # 784 pixels: 6 tiles + 16 pixels
+    # H*W a multiple of 4 only: planes the TMA unit cannot address, back to the layout copy
+    (2, 64, 6, 6, 24, 1, 1),
+    (3, 128, 14, 14, 72, 1, 1),    # 196 pixels: 128 + 68
+    (1, 192, 10, 18, 136, 1, 1),   # three K blocks, two column tiles
 ]
 
 
