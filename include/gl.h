@@ -200,9 +200,11 @@ GL_API int gl_compute_reduce_sum(const gl_ap* in, gl_ap* out, void* stream);
  * taken in an unspecified order.  `workspace` must hold at least
  * gl_cartesian_dot_workspace() bytes (it may be NULL when that is 0) and must be
  * 1024-byte aligned; its contents are scratch.  Few-channel convolutions (at most
- * 8 / Sw channels, the RGB stem) and channels-last items with a channel count
- * that is a multiple of 8 need none: the kernels read both operands where they
- * are.  Encoded tensor maps are kept per argument list, so a repeated call on the
+ * 8 / Sw channels, the RGB stem), channels-last items with a channel count that is
+ * a multiple of 8, and 1x1 unpadded windows over (C,H,W) items whose rows the TMA
+ * unit can address (C a multiple of 8 and at least 64; unit strides with H*W a
+ * multiple of 8, or W a multiple of 8 up to 64 with a column stride of 1 or 2) need
+ * none: the kernels read both operands where they are.  Encoded tensor maps are kept per argument list, so a repeated call on the
  * same buffers skips the driver's encoding.  The kernels are launched with programmatic
  * stream serialisation: their set-up may run while the preceding kernel of the stream
  * drains, and they wait for its completion before their first access to memory. */
