@@ -285,13 +285,18 @@ __global__ void __launch_bounds__(kThreads) pad_rows_flat(const uint32_t* __rest
     const uint32_t o = static_cast<uint32_t>(pc) << 2;         // total < 2^31
     uint32_t r = d_out == 1 ? o : (__umulhi(o, mul) >> shift);
     int c = static_cast<int>(o - r * static_cast<uint32_t>(d_out));
+    // all four loads go out before the first select: border cells read a clamped address and are replaced
     uint32_t v[4];
+    bool inside[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const int x = c - lo;
-      v[i] = (x >= 0 && x < d_in) ? in[static_cast<int64_t>(r) * d_in + x] : fill;
+      inside[i] = x >= 0 && x < d_in;
+      v[i] = in[static_cast<int64_t>(r) * d_in + min(max(x, 0), d_in - 1)];
       if (++c == d_out) { c = 0; ++r; }
     }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) v[i] = inside[i] ? v[i] : fill;
     reinterpret_cast<uint4*>(out)[pc] = make_uint4(v[0], v[1], v[2], v[3]);
   }
   // the last total % 4 elements
