@@ -159,8 +159,10 @@ class ClockSampler:
 # reference arm: the CPU checker, as it stands
 # --------------------------------------------------------------------------
 
-def cpu_baseline_dense(target_seconds: float = 12.0):
-    """Times oracle.brute.rowdot on a sample of rows of the 4096^3 workload."""
+def cpu_baseline_dense(target_seconds: float = 12.0, gpu_result=None):
+    """Times oracle.brute.rowdot on a sample of rows of the 4096^3 workload.  With `gpu_result` (the device's
+    [M, O] result of the same seeded inputs, relu applied, as the end-to-end leg brought it back) the sampled rows
+    are also compared: max |g - r| / max(|r|, rms(r)), the metric and inputs of the parity tests."""
     import numpy as np
     from oracle import brute
     from paper_2105_09377_b200 import synth
@@ -171,16 +173,23 @@ def cpu_baseline_dense(target_seconds: float = 12.0):
     for _ in range(3):                        # grow the sample until it takes a fair share of the target
         idx = np.arange(rows, dtype=np.int64)
         t0 = time.perf_counter()
-        brute.rowdot(a, b, idx)
+        ref = brute.rowdot(a, b, idx)
         dt = max(time.perf_counter() - t0, 1e-4)
         if rows >= case.m or dt >= target_seconds / 3:
             break
         rows = int(min(case.m, max(rows * 2, rows * target_seconds / dt)))
         rows -= rows % 8
     flops = 2.0 * rows * case.o * case.k
-    return {"value": flops / dt / 1e12, "unit": "TFLOP/s", "cores": brute.num_threads(), "kind": "oracle",
-            "sample": "rows 0..%d of A (of %d) against all %d rows of B, float64 accumulate, %.1f s" % (rows - 1, case.m, case.o, dt),
-            "seconds": dt, "rows": rows}
+    res = {"value": flops / dt / 1e12, "unit": "TFLOP/s", "cores": brute.num_threads(), "kind": "oracle",
+           "sample": "rows 0..%d of A (of %d) against all %d rows of B, float64 accumulate, %.1f s" % (rows - 1, case.m, case.o, dt),
+           "seconds": dt, "rows": rows}
+    if gpu_result is not None:
+        want = np.maximum(np.asarray(ref, dtype=np.float64), 0.0)
+        got = np.asarray(gpu_result[:want.shape[0]], dtype=np.float64)
+        rms = float(np.sqrt(np.mean(want * want))) or 1.0
+        res["max_rel_err"] = float(np.max(np.abs(got - want) / np.maximum(np.abs(want), rms)))
+        res["max_rel_err_of"] = "the device's result rows 0..%d against the oracle's, tolerance of the parity tests 2e-3" % (want.shape[0] - 1)
+    return res
 
 
 def run_reference(args):
@@ -296,17 +305,20 @@ def detail_workloads(device, peaks):
         del runs
         torch.cuda.empty_cache()
 
-    def entry(cfg, layout, bf16_out=False):
+    def entry(cfg, layout, bf16_out=False, nchw_out=False):
         from paper_2105_09377_b200 import binding as gl
         nsets = max(2, int((2 * L2_BYTES + cfg.algorithmic_bytes - 1) // cfg.algorithmic_bytes))
         nsets = min(nsets, 32)
         calls, flops, nbytes = [], 0.0, 0
         for _ in range(nsets):
-            c, flops, nbytes = rw.build_call(cfg, layout, device, None, gl.GL_OUT_BF16 if bf16_out else 0)
+            c, flops, nbytes = rw.build_call(cfg, layout, device, None,
+                                             (gl.GL_OUT_BF16 if bf16_out else 0) | (gl.GL_OUT_NCHW if nchw_out else 0))
             calls.append(c)
         if bf16_out:                     # results written as 2-byte elements
             nbytes -= cfg.n * cfg.ho * cfg.wo * cfg.o * 2
             layout = layout + "+bf16out"
+        if nchw_out:                     # Fig. 2a as written: (C,H,W) items in, (N,O,H',W') out
+            layout = layout + "+nchwout"
         med, best = time_graph(calls, 20, device)
         e = {"workload": cfg.name, "us": med * 1e6, "us_best": best * 1e6, "gbs": nbytes / med / 1e9,
              "frac_hbm_peak": nbytes / med / 1e9 / peaks["hbm_gbs"], "buffer_sets": nsets}
@@ -324,6 +336,8 @@ def detail_workloads(device, peaks):
     entry(synth.CONV_SWEEP_3X3[0], "rewritten")   # the materialised im2col form of Section 5.3, for comparison
     for cfg in (synth.CONV_SWEEP_3X3[0], synth.CONV_STRIDED_1X1[0], synth.CONV_STRIDED_1X1[1]):
         entry(cfg, "nhwc", bf16_out=True)         # the two bandwidth-bound shapes with bf16 results
+    for cfg in (synth.CONV_SWEEP_3X3[0], synth.CONV_STRIDED_1X1[0]):
+        entry(cfg, "nchw", nchw_out=True)         # the whole program of Fig. 2a, squeeze + transpose fused
     for layout in ("nhwc", "nchw"):
         chain_entry(layout)                       # Fig. 2a + relu + Fig. 2c + Fig. 2b composed, per item layout
     for cfg in (synth.MEM_IM2COL, synth.MEM_TRANSPOSE, synth.MEM_MAXPOOL, synth.MEM_RELU, synth.MEM_PAD):
@@ -531,7 +545,7 @@ def run_gpu(args):
         "gpu_launches": args.steps, "clocks": clocks,
     }
     if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline_dense(args.cpu_seconds)
+        line["cpu_baseline"] = cpu_baseline_dense(args.cpu_seconds, gpu_result=o_pin[(e2e_steps - 1) % 2].numpy())
     if world == 1 and args.detail:
         line["detail_columns"] = ["workload", "layout", "us", "TFLOP/s", "GB/s (algorithmic)", "fraction of binding roofline"]
         line["detail"] = compact_rows(detail_workloads(device, peaks))

@@ -70,6 +70,8 @@ def build_call(cfg, layout: str, device, batch=None, flags=0):
             spec = gl.windows_spec((cfg.c, cfg.kh, cfg.kw), (1, cfg.stride, cfg.stride), (0, cfg.pad, cfg.pad), (0, cfg.pad, cfg.pad))
         xa, wa = gl.AccessPattern(_bf16(x, device), 1), gl.AccessPattern(_bf16(wt, device), 1)
         out = gl.output_like(gl.gl_shape_cartesian_dot(x.shape, 1, spec, wt.shape, 1), device)
+        if flags & gl.GL_OUT_NCHW:      # Fig. 2a's whole program: squeeze + transpose (0 3 1 2) fused, ((N,O,H',W'),())
+            out = gl.AccessPattern(torch.empty((cfg.n, cfg.o, cfg.ho, cfg.wo), dtype=torch.float32, device=device), 4)
         if flags & gl.GL_OUT_BF16:      # results stored as bf16: half the bytes written
             out = gl.AccessPattern(out.tensor.to(torch.bfloat16), out.access_ndim)
         need = gl.gl_cartesian_dot_workspace(xa, spec, wa, flags)
