@@ -387,6 +387,51 @@ def test_dense_paired_tiles_bit_exact(gl, m, o, k):
         assert bool((sentinel[:4] == -7.0).all()) and bool((sentinel[m + 4:] == -7.0).all())
 
 
+GUARDED_CONVS = [
+    # n, c, h, w, o, k, stride, pad, channels_last, flags: one case per kernel family
+    (2, 128, 28, 28, 128, 3, 1, 1, True, 0),       # resident windows on block pairs
+    (2, 64, 20, 20, 64, 3, 1, 1, True, 0),         # resident windows, two blocks per SM
+    (2, 3, 40, 40, 64, 7, 2, 3, True, 0),          # few channels read in place, channels-last
+    (2, 3, 40, 40, 64, 7, 2, 3, False, 1),         # ... (C,H,W) items, fused squeeze + transpose
+    (2, 64, 12, 16, 40, 1, 2, 0, False, 0),        # pixel-major 1x1 windows
+    (2, 72, 9, 9, 40, 3, 1, 1, False, 0),          # layout copies + im2col-mode tiles
+    (1, 512, 7, 7, 64, 3, 1, 1, True, 0),          # K split: partial planes in the workspace
+    (2, 12, 10, 12, 8, 3, 1, 1, False, 0),         # row-window copies
+]
+
+
+@pytest.mark.parametrize("case", GUARDED_CONVS, ids=lambda c: "x".join(map(str, c)))
+def test_conv_writes_only_its_result_and_its_workspace(gl, case):
+    # guard bands around the result and behind the workspace must keep their fill; the result must be right
+    n, c, h, w, o, k, s_, pad, cl, nchw = case
+    flags = gl.GL_OUT_NCHW if nchw else 0
+    x = synth.uniform_int(48, 1, (n, c, h, w), -3, 3)
+    wt = synth.uniform_int(48, 2, (o, c, k, k), -3, 3)
+    ref = _conv_ref(x, wt, (s_, s_), (pad, pad))
+    if cl:
+        xa = gl.AccessPattern(to_bf16_device(np.ascontiguousarray(x.transpose(0, 2, 3, 1))), 1)
+        wa = gl.AccessPattern(to_bf16_device(np.ascontiguousarray(wt.transpose(0, 2, 3, 1))), 1)
+        spec = gl.windows_spec((k, k, c), (s_, s_, 1), (pad, pad, 0), (pad, pad, 0))
+    else:
+        xa, wa = gl.AccessPattern(to_bf16_device(x), 1), gl.AccessPattern(to_bf16_device(wt), 1)
+        spec = gl.windows_spec((c, k, k), (1, s_, s_), (0, pad, pad), (0, pad, pad))
+    ho, wo = ref.shape[1], ref.shape[2]
+    count, band = n * ho * wo * o, 4096
+    buf = torch.full((count + 2 * band,), -7.0, device="cuda")
+    shape = (n, o, ho, wo) if nchw else ((n, ho, wo, 1, o) if cl else (n, 1, ho, wo, o))
+    out = gl.AccessPattern(buf[band:band + count].view(shape), 4 if nchw else 5)
+    need = gl.gl_cartesian_dot_workspace(xa, spec, wa, flags)
+    ws = torch.full((need + 1024 + band,), 0xAB, dtype=torch.uint8, device="cuda")
+    first = (ws.data_ptr() + 1023) // 1024 * 1024 - ws.data_ptr()
+    gl.gl_cartesian_dot(xa, spec, wa, out=out, flags=flags, workspace=ws[:first + need] if need else None)
+    _ok(gl)
+    got = buf[band:band + count].view(shape).cpu().numpy().astype(np.float64)
+    want = ref.transpose(0, 3, 1, 2) if nchw else (ref[:, :, :, None] if cl else ref[:, None])
+    assert np.array_equal(got, want)
+    assert bool((buf[:band] == -7.0).all()) and bool((buf[band + count:] == -7.0).all())
+    assert bool((ws[first + need:] == 0xAB).all()) and bool((ws[:first] == 0xAB).all())
+
+
 def test_conv_paired_tiles_bit_exact(gl):
     # 161 row tiles x one 256-wide column tile: the im2col loads of both blocks of a pair
     n, c, h, w, o = 5, 64, 64, 64, 200
