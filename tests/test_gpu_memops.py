@@ -244,3 +244,56 @@ def test_output_metadata_is_checked(gl):
     with pytest.raises(gl.GlError) as e:
         gl.gl_compute_relu(gl.AccessPattern(x.to(torch.bfloat16), 1))
     assert e.value.code == 2
+
+
+def _guarded(shape, dtype, band=2048):
+    """A result tensor of `shape` inside a larger buffer whose guard bands hold -7."""
+    count = int(np.prod(shape))
+    buf = torch.full((count + 2 * band,), -7.0, device="cuda", dtype=dtype)
+    return buf, buf[band:band + count].view(shape), band, count
+
+
+def _bands_intact(buf, band, count):
+    return bool((buf[:band] == -7.0).all()) and bool((buf[band + count:] == -7.0).all())
+
+
+def test_memory_bound_operators_write_only_their_results(gl):
+    # every operator writes into the middle of a buffer whose guard bands must keep their fill; ragged shapes
+    x = synth.uniform(14, 1, (3, 5, 13, 18), -1.0, 1.0) - 2.0
+    xa = gl.AccessPattern(to_f32_device(x), 1)
+    # im2col
+    spec = gl.windows_spec((5, 3, 3), (1, 1, 1), (0, 1, 1), (0, 1, 1))
+    first = gl.gl_access_windows(xa, spec)
+    buf, view, band, count = _guarded(tuple(first.tensor.shape), torch.float32)
+    gl.gl_access_windows(xa, spec, out=gl.AccessPattern(view, first.access_ndim))
+    assert gl.gl_poll_device_status() == 0 and torch.equal(view, first.tensor) and _bands_intact(buf, band, count)
+    # transpose
+    first = gl.gl_access_transpose(xa, (0, 2, 3, 1))
+    buf, view, band, count = _guarded(tuple(first.tensor.shape), torch.float32)
+    gl.gl_access_transpose(xa, (0, 2, 3, 1), out=gl.AccessPattern(view, first.access_ndim))
+    assert gl.gl_poll_device_status() == 0 and torch.equal(view, first.tensor) and _bands_intact(buf, band, count)
+    assert np.array_equal(view.cpu().numpy(), x.transpose(0, 2, 3, 1).astype(np.float32))
+    # pad of the innermost dimension
+    first = gl.gl_access_pad(xa, 3, 1, 1)
+    buf, view, band, count = _guarded(tuple(first.tensor.shape), torch.float32)
+    gl.gl_access_pad(xa, 3, 1, 1, out=gl.AccessPattern(view, first.access_ndim))
+    assert gl.gl_poll_device_status() == 0 and torch.equal(view, first.tensor) and _bands_intact(buf, band, count)
+    assert np.array_equal(view.cpu().numpy(), np.pad(x, ((0, 0), (0, 0), (0, 0), (1, 1))).astype(np.float32))
+    # max pooling, fp32 planes (3x3 stride 2: rows of four column groups and a half) and bf16 planes
+    xp = synth.uniform(14, 2, (3, 5, 14, 24), -1.0, 1.0) - 2.0
+    pool = gl.windows_spec((3, 3), (2, 2), (1, 1), (1, 1), gl.GL_PAD_NEG_INF)
+    ref = brute.maxpool(xp.astype(np.float32), (3, 3), (2, 2), ((1, 1), (1, 1)))
+    buf, view, band, count = _guarded(ref.shape, torch.float32)
+    nd = gl.gl_compute_reduce_max(gl.AccessPattern(to_f32_device(xp), 2), pool).access_ndim
+    gl.gl_compute_reduce_max(gl.AccessPattern(to_f32_device(xp), 2), pool, out=gl.AccessPattern(view, nd))
+    assert gl.gl_poll_device_status() == 0 and np.array_equal(view.cpu().numpy(), ref) and _bands_intact(buf, band, count)
+    xb = synth.bf16_round(xp)
+    refb = brute.maxpool(xb, (3, 3), (2, 2), ((1, 1), (1, 1)))
+    buf, view, band, count = _guarded(refb.shape, torch.bfloat16)
+    gl.gl_compute_reduce_max(gl.AccessPattern(to_bf16_device(xb), 2), pool, out=gl.AccessPattern(view, nd))
+    assert gl.gl_poll_device_status() == 0 and np.array_equal(view.float().cpu().numpy(), refb) and _bands_intact(buf, band, count)
+    # relu
+    buf, view, band, count = _guarded(x.shape, torch.float32)
+    gl.gl_compute_relu(xa, out=gl.AccessPattern(view, 1))
+    assert gl.gl_poll_device_status() == 0 and _bands_intact(buf, band, count)
+    assert np.array_equal(view.cpu().numpy(), np.maximum(x, 0.0).astype(np.float32))
